@@ -1,0 +1,274 @@
+"""CPU oracle for the TriSpec verify pass — TEST INFRASTRUCTURE, not a product path.
+
+Plain, slow, fp64 numpy restatement of what the verification pass computes, written from
+the paper's definitions. It shares no code with the CUDA path and must only be used by the
+tests, the smoke check and the benchmark's CPU-baseline leg.
+
+What each function follows:
+  build_tree_mask  tree attention mask of a draft tree (Figure 4, "attention mask updates";
+                   tree configuration of Section 4.1): a node sees its ancestors and itself.
+  verify_attn      the attention of one parallel verification pass (Eq. 2 / Eq. 5): every
+                   tree node attends to the whole committed context plus the tree keys its
+                   mask row allows; plain softmax(q k / sqrt(D)) v.
+  lmhead_stats     per-position softmax distribution p_i in R^V (Eq. 5) reduced to the
+                   quantities the rule needs: top_1(p), top_2(p) (Eq. 8), argmax token x_i^(p)
+                   (greedy form of Eq. 6) and p_i(x_i^(d)) for each drafted child.
+  accept_scan      greedy acceptance s_i (Eq. 6), acceptance length tau_a (Eq. 7), margin
+                   predicate g (Eq. 8), trusted prefix tau_m (Eq. 9) and the routing cases
+                   (i)/(ii) of "Adaptive Verification Routing" / Algorithm 1; TARGET mode is
+                   the "standard left-to-right acceptance rule" applied after Eq. 10.
+
+Readings of the paper taken here (the paper states the rule for a chain of k tokens):
+  * Tree rule = the chain rule applied along the path the greedy matches select; the margin
+    test at a node precedes the child match (if g = 0 at depth j then tau_m = j and, all
+    earlier tokens having matched, tau_a >= j: case (ii)).
+  * top_2 is the largest entry among indices other than the arg-max (two equal maxima give
+    margin 0). Ties resolve to the lowest vocabulary index; duplicate sibling tokens resolve
+    to the lowest node index.
+  * Parity of the tree rule is pinned by brute force over all root-to-leaf paths in the tests;
+    the end-to-end behaviour of the paper's models (acceptance lengths, speedups) is
+    "parity unpinned": it needs the paper's models and datasets.
+"""
+from __future__ import annotations
+
+from typing import Dict, Iterable, Optional, Sequence, Tuple
+
+import numpy as np
+
+MODE_PROXY = 0
+MODE_TARGET = 1
+
+
+def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> float64 values (exact)."""
+    u = np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------------------
+# tree mask (Figure 4; Section 4.1 tree configuration)
+# ----------------------------------------------------------------------------------------
+def build_tree_mask(parent: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """mask[b][i] has bit j set iff j is an ancestor of i or j == i; depth[b][i] = number of
+    edges from the root. parent[b][0] = -1 and parent[b][i] < i; T <= 64."""
+    parent = np.asarray(parent)
+    B, T = parent.shape
+    assert T <= 64
+    mask = np.zeros((B, T), dtype=np.uint64)
+    depth = np.zeros((B, T), dtype=np.int32)
+    for b in range(B):
+        for i in range(T):
+            bits = 0
+            steps = 0
+            p = i
+            while p >= 0:
+                bits |= (1 << p)
+                p = int(parent[b, p])
+                steps += 1
+            mask[b, i] = np.uint64(bits)
+            depth[b, i] = steps - 1
+    return mask, depth
+
+
+# ----------------------------------------------------------------------------------------
+# verification attention (Eq. 2 / Eq. 5: one parallel pass over the drafted tokens)
+# ----------------------------------------------------------------------------------------
+def _context_kv(cache_bits: np.ndarray, b: int, kvh: int, L: int,
+                block_table: Optional[np.ndarray], block_size: int) -> np.ndarray:
+    """[L][D] fp64 keys or values of sequence b, KV head kvh. Contiguous cache is
+    [B][Lmax][Hkv][D]; a paged pool is [num_blocks][block][Hkv][D] and token t lives in block
+    block_table[b][t // block], slot t % block."""
+    if block_table is None:
+        return bf16_to_f64(cache_bits[b, :L, kvh, :])
+    t = np.arange(L)
+    blk = block_table[b, t // block_size]
+    return bf16_to_f64(cache_bits[blk, t % block_size, kvh, :])
+
+
+def verify_attn(q: np.ndarray, k_tree: np.ndarray, v_tree: np.ndarray, mask: np.ndarray,
+                k_cache: np.ndarray, v_cache: np.ndarray, ctx_len: np.ndarray, scale: float,
+                block_table: Optional[np.ndarray] = None, block_size: int = 64,
+                seqs: Optional[Iterable[int]] = None,
+                samples: Optional[Sequence[Tuple[int, int, int]]] = None):
+    """o[b][i][h] = sum_j softmax_j(scale * q[b][i][h] . k_j) v_j over the visible keys j:
+    all ctx_len[b] context positions and the tree nodes whose bit is set in mask[b][i].
+    KV head of query head h is h // (Hq // Hkv).
+
+    Returns (o float64 [B][T][Hq][D], lse float64 [B][Hq][T]); entries that were not asked for
+    (seqs / samples restrict the work) are NaN. `samples` is a list of (b, i, h)."""
+    B, T, Hq, D = q.shape
+    Hkv = k_tree.shape[2]
+    G = Hq // Hkv
+    o = np.full((B, T, Hq, D), np.nan)
+    lse = np.full((B, Hq, T), np.nan)
+    if samples is None:
+        bs = range(B) if seqs is None else list(seqs)
+        todo = {}
+        for b in bs:
+            for g in range(Hkv):
+                todo[(b, g)] = [(i, h) for h in range(g * G, (g + 1) * G) for i in range(T)]
+    else:
+        todo = {}
+        for (b, i, h) in samples:
+            todo.setdefault((int(b), int(h) // G), []).append((int(i), int(h)))
+    for (b, g), items in todo.items():
+        L = int(ctx_len[b])
+        Kc = _context_kv(k_cache, b, g, L, block_table, block_size)
+        Vc = _context_kv(v_cache, b, g, L, block_table, block_size)
+        Kt = bf16_to_f64(k_tree[b, :, g, :])
+        Vt = bf16_to_f64(v_tree[b, :, g, :])
+        for (i, h) in items:
+            qi = bf16_to_f64(q[b, i, h, :])
+            vis = [j for j in range(T) if (int(mask[b, i]) >> j) & 1]
+            s = np.concatenate([Kc @ qi, Kt[vis] @ qi]) * scale
+            m = s.max()
+            e = np.exp(s - m)
+            den = e.sum()
+            p = e / den
+            o[b, i, h, :] = p[:L] @ Vc + p[L:] @ Vt[vis]
+            lse[b, h, i] = m + np.log(den)
+    return o, lse
+
+
+# ----------------------------------------------------------------------------------------
+# LM-head softmax statistics (Eq. 5 distributions; top_1/top_2 of Eq. 8)
+# ----------------------------------------------------------------------------------------
+STAT_F = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft")
+STAT_I = ("top1_idx", "top2_idx")
+
+
+def row_logits(h_row_bits: np.ndarray, W64: np.ndarray, logit_scale: float) -> np.ndarray:
+    """z_v = logit_scale * <h, W_v> for every vocabulary entry v (fp64)."""
+    return logit_scale * (W64 @ bf16_to_f64(h_row_bits))
+
+
+def lmhead_stats(h: np.ndarray, W: np.ndarray, parent: np.ndarray, tok: np.ndarray,
+                 logit_scale: float, seqs: Optional[Iterable[int]] = None,
+                 W64: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """Per row r = (b, node): p = softmax(z) over the vocabulary, reduced to
+    max z, lse = log sum exp z, the largest entry (top1_val, top1_idx; ties -> lowest index),
+    the largest entry among the other indices (top2_val, top2_idx), p_top1, p_top2; and for
+    each child node c the logit of its drafted token in its parent's row (draft_logit[b][c])
+    and the probability p_draft[b][c] = p_{parent(c)}(tok[c]). Entries of node 0 in
+    draft_logit / p_draft are NaN. h is [B][T][d] bf16 bits, W is [V][d] bf16 bits.
+    All outputs are [B][T]; rows of sequences not in `seqs` are NaN / -1."""
+    B, T, d = h.shape
+    if W64 is None:
+        W64 = bf16_to_f64(W)
+    out = {k: np.full((B, T), np.nan) for k in STAT_F}
+    out.update({k: np.full((B, T), -1, dtype=np.int64) for k in STAT_I})
+    for b in (range(B) if seqs is None else seqs):
+        for r in range(T):
+            z = row_logits(h[b, r], W64, logit_scale)
+            m = z.max()
+            lse = m + np.log(np.exp(z - m).sum())
+            i1 = int(np.argmax(z))                 # first occurrence = lowest index
+            z_wo = z.copy()
+            z_wo[i1] = -np.inf
+            i2 = int(np.argmax(z_wo))
+            out["max"][b, r] = m
+            out["lse"][b, r] = lse
+            out["top1_val"][b, r] = z[i1]
+            out["top2_val"][b, r] = z[i2]
+            out["top1_idx"][b, r] = i1
+            out["top2_idx"][b, r] = i2
+            out["p_top1"][b, r] = np.exp(z[i1] - lse)
+            out["p_top2"][b, r] = np.exp(z[i2] - lse)
+            for c in range(1, T):
+                if int(parent[b, c]) == r:
+                    out["draft_logit"][b, c] = z[int(tok[b, c])]
+                    out["p_draft"][b, c] = np.exp(z[int(tok[b, c])] - lse)
+    return out
+
+
+# ----------------------------------------------------------------------------------------
+# acceptance scan (Eq. 6-9, routing cases (i)/(ii), Algorithm 1)
+# ----------------------------------------------------------------------------------------
+def accept_scan(p_top1: np.ndarray, p_top2: np.ndarray, top1_idx: np.ndarray,
+                parent: np.ndarray, tok: np.ndarray, lam: float, mode: int = MODE_PROXY,
+                active: Optional[np.ndarray] = None,
+                start_node: Optional[np.ndarray] = None,
+                near_eps: float = 1e-3) -> Dict[str, np.ndarray]:
+    """Greedy walk of each draft tree.
+
+    At the current node (position i+1 of the chain formulas, i = tokens accepted so far):
+      PROXY mode: if top_1(p) - top_2(p) < lambda the position is untrusted: tau_m = i, and as
+        every earlier token matched tau_a >= tau_m: case (ii), accept x_{1:tau_m}, escalate.
+      Otherwise look for the child whose drafted token equals the arg-max token (s_{i+1} = 1):
+        none -> tau_a = i < tau_m: case (i), approve, bonus = arg-max token of this node;
+        found -> accept it and move there.
+      TARGET mode: the same without the margin test (never escalates).
+
+    Outputs per sequence: accept_len, escalate (0/1), bonus_tok (-1 if escalated), path
+    [B][T] (accepted node ids in order, -1 padded), last_node, near_thr (number of visited
+    positions with |margin - lambda| < near_eps; PROXY mode only); plus n_escalated and
+    esc_index (ascending sequence ids that escalated, -1 padded). Inactive sequences get
+    accept_len 0, escalate 0, bonus -1, last_node -1.
+    """
+    parent = np.asarray(parent)
+    B, T = parent.shape
+    res = {
+        "accept_len": np.zeros(B, dtype=np.int32),
+        "escalate": np.zeros(B, dtype=np.uint8),
+        "bonus_tok": np.full(B, -1, dtype=np.int32),
+        "path": np.full((B, T), -1, dtype=np.int32),
+        "last_node": np.full(B, -1, dtype=np.int32),
+        "near_thr": np.zeros(B, dtype=np.int32),
+    }
+    for b in range(B):
+        if active is not None and not active[b]:
+            continue
+        cur = 0 if start_node is None else int(start_node[b])
+        n = 0
+        while True:
+            if mode == MODE_PROXY:
+                margin = float(p_top1[b, cur]) - float(p_top2[b, cur])
+                if abs(margin - lam) < near_eps:
+                    res["near_thr"][b] += 1
+                if not (margin >= lam):
+                    res["escalate"][b] = 1
+                    break
+            nxt = -1
+            for c in range(cur + 1, T):
+                if int(parent[b, c]) == cur and int(tok[b, c]) == int(top1_idx[b, cur]):
+                    nxt = c
+                    break
+            if nxt < 0:
+                res["bonus_tok"][b] = int(top1_idx[b, cur])
+                break
+            res["path"][b, n] = nxt
+            n += 1
+            cur = nxt
+        res["accept_len"][b] = n
+        res["last_node"][b] = cur
+    esc = np.nonzero(res["escalate"])[0].astype(np.int32)
+    res["n_escalated"] = np.int32(len(esc))
+    res["esc_index"] = np.full(B, -1, dtype=np.int32)
+    res["esc_index"][:len(esc)] = esc
+    return res
+
+
+# ----------------------------------------------------------------------------------------
+# the whole pass
+# ----------------------------------------------------------------------------------------
+def verify(inp: Dict[str, np.ndarray], scale: float, logit_scale: float, lam: float,
+           mode: int = MODE_PROXY, block_size: int = 64, with_attention: bool = True):
+    """Mask -> attention -> LM-head statistics -> acceptance scan, on the arrays produced by
+    the input generator. Only sequences listed in inp["seq_index"] (all if None) are verified."""
+    parent, tok = inp["parent"], inp["tok"]
+    B = parent.shape[0]
+    seqs = list(range(B)) if inp.get("seq_index") is None else [int(s) for s in inp["seq_index"]]
+    active = np.zeros(B, dtype=np.uint8)
+    active[seqs] = 1
+    mask, depth = build_tree_mask(parent)
+    out = {"mask": mask, "depth": depth}
+    if with_attention:
+        o, lse = verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], mask, inp["k_cache"],
+                             inp["v_cache"], inp["ctx_len"], scale,
+                             block_table=inp.get("block_table"), block_size=block_size, seqs=seqs)
+        out["o"], out["attn_lse"] = o, lse
+    st = lmhead_stats(inp["h"], inp["W"], parent, tok, logit_scale, seqs=seqs)
+    out["stats"] = st
+    out["scan"] = accept_scan(st["p_top1"], st["p_top2"], st["top1_idx"], parent, tok, lam,
+                              mode=mode, active=active)
+    return out
