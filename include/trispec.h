@@ -1,0 +1,182 @@
+/*
+ * trispec.h — C ABI of the B200 (sm_100a) verify pass of TriSpec, ternary speculative
+ * decoding with a lightweight proxy verifier.
+ *
+ * One verification pass scores a draft tree of T = k + 1 nodes per sequence (node 0 is the
+ * last committed token, whose output distribution is p_1 of Eq. 2 / Eq. 5; nodes 1..k are the
+ * k drafted tokens). The pass is:
+ *   1. trispec_build_tree_mask  ancestor mask of the draft tree (Figure 4, Section 4.1)
+ *   2. trispec_verify_attn      GQA attention of the tree tokens over the committed KV cache
+ *                               and the tree's own keys under that mask (Eq. 2 / Eq. 5)
+ *   3. trispec_lmhead_stats     LM head fused with per-position softmax statistics: max,
+ *                               log-sum-exp, top_1 / top_2 (Eq. 8), p(drafted token) (Eq. 6)
+ *   4. trispec_accept_scan      acceptance length tau_a (Eq. 7), trusted prefix tau_m (Eq. 9)
+ *                               and routing: approve or escalate (cases (i)/(ii), Algorithm 1)
+ *   trispec_verify              the four in order on one stream.
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless a comment says
+ *     "host". The library never frees or retains caller memory past the call.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream). No call synchronises the device.
+ *   - Return value: 0 (TRISPEC_OK) or a trispec_status error. Argument errors are detected
+ *     on the host before anything is launched. No exceptions, no output on stdout/stderr.
+ *   - bf16 tensors are passed as `const void*` (16-bit patterns). D (head dim) must be 128,
+ *     T <= 64, Hq / Hkv in {1, 2, 4, 8, 16}.
+ *   - Rows of per-node arrays are indexed row = b * T + node.
+ *   - `dev_status` (optional, int32 on the device, caller zeroes it): receives a non-zero
+ *     code if a bounded device-side wait gave up; the kernels never trap.
+ */
+#ifndef TRISPEC_H_
+#define TRISPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TRISPEC_OK = 0,
+  TRISPEC_ERR_INVALID_ARG = 1,     /* null pointer, non-positive size, misaligned pointer */
+  TRISPEC_ERR_UNSUPPORTED = 2,     /* D != 128, T > 64, unsupported group size, ... */
+  TRISPEC_ERR_WORKSPACE = 3,       /* workspace_bytes smaller than the *_workspace() query */
+  TRISPEC_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed */
+  TRISPEC_ERR_DEVICE_TIMEOUT = 5   /* value written to dev_status by a bounded wait */
+} trispec_status;
+
+#define TRISPEC_MODE_PROXY 0   /* margin rule of Eq. 8-9 applied (proxy verifier) */
+#define TRISPEC_MODE_TARGET 1  /* plain left-to-right acceptance (target verifier, after Eq. 10) */
+
+#define TRISPEC_KV_CONTIGUOUS 0 /* k_cache, v_cache: [B][Lmax][Hkv][D] */
+#define TRISPEC_KV_PAGED 1      /* pool [num_blocks][block_size][Hkv][D] + block_table */
+
+const char* trispec_status_string(int status);
+
+/* Number of the library's own kernels launched on this process since load (host counter). */
+long long trispec_launch_count(void);
+
+/* ---------------------------------------------------------------------------------------
+ * 1. Tree mask (Figure 4 "attention mask updates"; draft tree of Section 4.1).
+ *    parent [B][T] int32: parent[b][0] = -1, 0 <= parent[b][i] < i.
+ *    mask   [B][T] uint64: bit j of mask[b][i] is 1 iff j is an ancestor of i or j == i.
+ *    depth  [B][T] int32 : edges from the root (may be NULL).
+ *    Malformed parents (>= i or < -1) are not dereferenced: the row gets mask 0 and depth -1.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int B, T;
+  const int32_t* parent;
+  uint64_t* mask;
+  int32_t* depth;
+} trispec_tree_args;
+int trispec_build_tree_mask(const trispec_tree_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 2. Verification attention (the attention of the parallel verification pass, Eq. 2 / 5).
+ *    o[b][i][h] = sum_j softmax_j(scale * q[b][i][h] . k_j) v_j over all ctx_len[b] context
+ *    keys plus the tree keys j with bit j set in mask[b][i]; KV head of h is h / (Hq/Hkv).
+ *    q [B][T][Hq][D], k_tree/v_tree [B][T][Hkv][D], o [B][T][Hq][D]: bf16.
+ *    kv_layout CONTIGUOUS: k_cache/v_cache [B][Lmax][Hkv][D] bf16.
+ *    kv_layout PAGED: pool [num_blocks][block_size=64][Hkv][D]; token t of sequence b is in
+ *      block block_table[b][t / 64] (int32 [B][max_blocks_per_seq]), slot t % 64.
+ *    ctx_len [B] int32, 0 <= ctx_len[b] <= Lmax (contiguous) or 64 * max_blocks_per_seq.
+ *    seq_index (optional, int32 [B_active], device): only these sequences are computed;
+ *      NULL = all B (then B_active is ignored).
+ *    lse (optional) f32 [B][Hq][T]: log-sum-exp of the scaled scores.
+ *    workspace: device scratch of at least trispec_verify_attn_workspace(a) bytes,
+ *      256-byte aligned; contents are undefined before and after the call.
+ *    Pointers of bf16 tensors must be 16-byte aligned.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int B, T, Hq, Hkv, D;
+  float scale;
+  const void *q, *k_tree, *v_tree;
+  int kv_layout;
+  const void *k_cache, *v_cache;
+  int Lmax, num_blocks, block_size, max_blocks_per_seq;
+  const int32_t *block_table, *ctx_len;
+  const uint64_t* mask;
+  const int32_t* seq_index;
+  int B_active;
+  void* o;
+  float* lse;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+} trispec_attn_args;
+size_t trispec_verify_attn_workspace(const trispec_attn_args* a);
+int trispec_verify_attn(const trispec_attn_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 3. LM-head softmax statistics (distributions p_i in R^V of Eq. 5; top_1, top_2 of Eq. 8).
+ *    z[r][v] = logit_scale * <h[r], W[v]>; no [rows x V] logits are written to memory.
+ *    Per row r = b*T + node (all arrays [B*T]):
+ *      max, lse = log sum_v exp z; (top1_val, top1_idx) largest entry, (top2_val, top2_idx)
+ *      largest entry among the other indices (ties -> lowest index);
+ *      p_top1 = exp(top1_val - lse), p_top2 likewise.
+ *    Per CHILD node c >= 1: draft_logit[b*T+c] = z[b*T+parent[c]][tok[c]] and
+ *      p_draft = exp(draft_logit - lse[parent row]); entries of node 0 are NaN.
+ *    h [B*T][d] bf16, W [V][d] bf16 (row-major, 16-byte aligned, d % 64 == 0).
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  float *max, *lse, *top1_val, *top2_val, *p_top1, *p_top2;
+  int32_t *top1_idx, *top2_idx;
+  float *draft_logit, *p_draft;
+} trispec_stats;
+
+typedef struct {
+  int B, T, d, V;
+  float logit_scale;
+  const void *h, *W;
+  const int32_t *parent, *tok;
+  const int32_t* seq_index;  /* optional subset, as in trispec_attn_args */
+  int B_active;
+  trispec_stats out;
+  void* workspace;           /* >= trispec_lmhead_stats_workspace(a) bytes, 256-byte aligned */
+  size_t workspace_bytes;
+  int32_t* dev_status;
+} trispec_lmhead_args;
+size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a);
+int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 4. Acceptance scan (Eq. 6 greedy form, Eq. 7, Eq. 8, Eq. 9, routing cases (i)/(ii),
+ *    Algorithm 1). Per sequence, walking from start_node (root if NULL):
+ *      PROXY mode: if p_top1 - p_top2 < lambda at the current node -> escalate (case (ii),
+ *      the accepted tokens so far are x_{1:tau_m}); else the child whose token equals
+ *      top1_idx is accepted and the walk continues; no such child -> approve (case (i)),
+ *      bonus_tok = top1_idx of the current node. TARGET mode: no margin test.
+ *    active (optional uint8 [B]): sequences with 0 are skipped (outputs: accept_len 0,
+ *      escalate 0, bonus -1, last_node -1, path -1).
+ *    Outputs: accept_len, bonus_tok, last_node, near_thr int32 [B]; escalate uint8 [B];
+ *      path int32 [B][T] (accepted node ids in order, -1 padded);
+ *      near_thr = visited positions with |margin - lambda| < 1e-3 (PROXY mode);
+ *      n_escalated int32 [1]; esc_index int32 [B] ascending ids of escalated sequences,
+ *      -1 padded. near_thr, n_escalated and esc_index may be NULL (n_escalated and esc_index
+ *      only together).
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int B, T;
+  float lambda;
+  int mode;
+  const int32_t *parent, *tok;
+  trispec_stats in;          /* only p_top1, p_top2, top1_idx are read */
+  const uint8_t* active;
+  const int32_t* start_node;
+  int32_t *accept_len, *bonus_tok, *path, *last_node, *near_thr, *n_escalated, *esc_index;
+  uint8_t* escalate;
+} trispec_scan_args;
+int trispec_accept_scan(const trispec_scan_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Fused pass: the four calls above in order on `stream` (one verification round of
+ * Algorithm 1 for one verifier). `attn` may be NULL to skip attention.
+ * ------------------------------------------------------------------------------------- */
+int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
+                   const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRISPEC_H_ */

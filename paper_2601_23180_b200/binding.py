@@ -1,0 +1,231 @@
+"""ctypes binding of libtrispec.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams, nothing else);
+every step of the verify pass runs inside the library's kernels. Importing this module
+fails loudly when the library has not been built: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtrispec.so")
+
+MODE_PROXY = 0
+MODE_TARGET = 1
+KV_CONTIGUOUS = 0
+KV_PAGED = 1
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_23180_b200.build` "
+                      "(there is no CPU or PyTorch fallback for the verify pass)")
+_lib = C.CDLL(LIB_PATH)
+
+_vp, _i, _f, _sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
+
+
+class TreeArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("parent", _vp), ("mask", _vp), ("depth", _vp)]
+
+
+class AttnArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("Hq", _i), ("Hkv", _i), ("D", _i), ("scale", _f),
+                ("q", _vp), ("k_tree", _vp), ("v_tree", _vp), ("kv_layout", _i),
+                ("k_cache", _vp), ("v_cache", _vp), ("Lmax", _i), ("num_blocks", _i),
+                ("block_size", _i), ("max_blocks_per_seq", _i), ("block_table", _vp),
+                ("ctx_len", _vp), ("mask", _vp), ("seq_index", _vp), ("B_active", _i),
+                ("o", _vp), ("lse", _vp), ("workspace", _vp), ("workspace_bytes", _sz),
+                ("dev_status", _vp)]
+
+
+class Stats(C.Structure):
+    _fields_ = [(n, _vp) for n in ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2",
+                                   "top1_idx", "top2_idx", "draft_logit", "p_draft")]
+
+
+class LmheadArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("d", _i), ("V", _i), ("logit_scale", _f), ("h", _vp), ("W", _vp),
+                ("parent", _vp), ("tok", _vp), ("seq_index", _vp), ("B_active", _i), ("out", Stats),
+                ("workspace", _vp), ("workspace_bytes", _sz), ("dev_status", _vp)]
+
+
+class ScanArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("lam", _f), ("mode", _i), ("parent", _vp), ("tok", _vp),
+                ("stats", Stats), ("active", _vp), ("start_node", _vp), ("accept_len", _vp),
+                ("bonus_tok", _vp), ("path", _vp), ("last_node", _vp), ("near_thr", _vp),
+                ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
+
+
+_lib.trispec_status_string.restype = C.c_char_p
+_lib.trispec_status_string.argtypes = [_i]
+_lib.trispec_launch_count.restype = C.c_longlong
+_lib.trispec_build_tree_mask.argtypes = [C.POINTER(TreeArgs), _vp]
+_lib.trispec_verify_attn_workspace.restype = _sz
+_lib.trispec_verify_attn_workspace.argtypes = [C.POINTER(AttnArgs)]
+_lib.trispec_verify_attn.argtypes = [C.POINTER(AttnArgs), _vp]
+_lib.trispec_lmhead_stats_workspace.restype = _sz
+_lib.trispec_lmhead_stats_workspace.argtypes = [C.POINTER(LmheadArgs)]
+_lib.trispec_lmhead_stats.argtypes = [C.POINTER(LmheadArgs), _vp]
+_lib.trispec_accept_scan.argtypes = [C.POINTER(ScanArgs), _vp]
+_lib.trispec_verify.argtypes = [C.POINTER(TreeArgs), C.POINTER(AttnArgs), C.POINTER(LmheadArgs),
+                                C.POINTER(ScanArgs), _vp]
+
+EXPORTS = ["trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
+           "trispec_verify_attn_workspace", "trispec_verify_attn", "trispec_lmhead_stats_workspace",
+           "trispec_lmhead_stats", "trispec_accept_scan", "trispec_verify"]
+
+
+class TrispecError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"trispec error {code}: {_lib.trispec_status_string(code).decode()}")
+
+
+def _check(code: int):
+    if code != 0:
+        raise TrispecError(code)
+
+
+def _p(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def status_string(code: int) -> str:
+    return _lib.trispec_status_string(code).decode()
+
+
+def launch_count() -> int:
+    return int(_lib.trispec_launch_count())
+
+
+STAT_F32 = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft")
+STAT_I32 = ("top1_idx", "top2_idx")
+
+
+def alloc_stats(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
+    st = {k: torch.full((B, T), float("nan"), dtype=torch.float32, device=device) for k in STAT_F32}
+    st.update({k: torch.full((B, T), -1, dtype=torch.int32, device=device) for k in STAT_I32})
+    return st
+
+
+def _stats_struct(st: Dict[str, torch.Tensor]) -> Stats:
+    s = Stats()
+    for name, _ in Stats._fields_:
+        setattr(s, name, _p(st.get(name)))
+    return s
+
+
+# ------------------------------------------------------------------------------ argument builders
+def tree_args(parent: torch.Tensor, mask: torch.Tensor, depth: Optional[torch.Tensor]) -> TreeArgs:
+    B, T = parent.shape
+    return TreeArgs(B, T, _p(parent), _p(mask), _p(depth))
+
+
+def attn_args(q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, scale, o, workspace=None,
+              block_table=None, block_size=64, seq_index=None, lse=None, dev_status=None) -> AttnArgs:
+    B, T, Hq, D = q.shape
+    Hkv = k_tree.shape[2]
+    a = AttnArgs()
+    a.B, a.T, a.Hq, a.Hkv, a.D, a.scale = B, T, Hq, Hkv, D, float(scale)
+    a.q, a.k_tree, a.v_tree = _p(q), _p(k_tree), _p(v_tree)
+    a.k_cache, a.v_cache = _p(k_cache), _p(v_cache)
+    if block_table is None:
+        a.kv_layout, a.Lmax = KV_CONTIGUOUS, k_cache.shape[1]
+        a.num_blocks, a.block_size, a.max_blocks_per_seq = 0, 0, 0
+    else:
+        a.kv_layout, a.num_blocks = KV_PAGED, k_cache.shape[0]
+        a.block_size, a.max_blocks_per_seq = int(block_size), block_table.shape[1]
+        a.Lmax = a.block_size * a.max_blocks_per_seq
+    a.block_table, a.ctx_len, a.mask = _p(block_table), _p(ctx_len), _p(mask)
+    a.seq_index = _p(seq_index)
+    a.B_active = 0 if seq_index is None else int(seq_index.numel())
+    a.o, a.lse = _p(o), _p(lse)
+    a.workspace = _p(workspace)
+    a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a.dev_status = _p(dev_status)
+    return a
+
+
+def lmhead_args(h, W, parent, tok, logit_scale, stats, workspace=None, seq_index=None,
+                dev_status=None) -> LmheadArgs:
+    B, T = parent.shape
+    a = LmheadArgs()
+    a.B, a.T, a.d, a.V, a.logit_scale = B, T, h.shape[-1], W.shape[0], float(logit_scale)
+    a.h, a.W, a.parent, a.tok = _p(h), _p(W), _p(parent), _p(tok)
+    a.seq_index = _p(seq_index)
+    a.B_active = 0 if seq_index is None else int(seq_index.numel())
+    a.out = _stats_struct(stats)
+    a.workspace = _p(workspace)
+    a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a.dev_status = _p(dev_status)
+    return a
+
+
+def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], active=None,
+              start_node=None) -> ScanArgs:
+    B, T = parent.shape
+    a = ScanArgs()
+    a.B, a.T, a.lam, a.mode = B, T, float(lam), int(mode)
+    a.parent, a.tok = _p(parent), _p(tok)
+    a.stats = _stats_struct(stats)
+    a.active, a.start_node = _p(active), _p(start_node)
+    for k in ("accept_len", "bonus_tok", "path", "last_node", "near_thr", "n_escalated", "esc_index", "escalate"):
+        setattr(a, k, _p(out.get(k)))
+    return a
+
+
+def alloc_scan_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
+    i32 = dict(dtype=torch.int32, device=device)
+    return {
+        "accept_len": torch.full((B,), -7, **i32), "bonus_tok": torch.full((B,), -7, **i32),
+        "path": torch.full((B, T), -7, **i32), "last_node": torch.full((B,), -7, **i32),
+        "near_thr": torch.full((B,), -7, **i32), "n_escalated": torch.full((1,), -7, **i32),
+        "esc_index": torch.full((B,), -7, **i32),
+        "escalate": torch.full((B,), 9, dtype=torch.uint8, device=device),
+    }
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(256, (nbytes + 255) // 256 * 256), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------------------ entry points
+def trispec_build_tree_mask(args: TreeArgs, stream=None):
+    _check(_lib.trispec_build_tree_mask(C.byref(args), _stream(stream)))
+
+
+def trispec_verify_attn_workspace(args: AttnArgs) -> int:
+    return int(_lib.trispec_verify_attn_workspace(C.byref(args)))
+
+
+def trispec_verify_attn(args: AttnArgs, stream=None):
+    _check(_lib.trispec_verify_attn(C.byref(args), _stream(stream)))
+
+
+def trispec_lmhead_stats_workspace(args: LmheadArgs) -> int:
+    return int(_lib.trispec_lmhead_stats_workspace(C.byref(args)))
+
+
+def trispec_lmhead_stats(args: LmheadArgs, stream=None):
+    _check(_lib.trispec_lmhead_stats(C.byref(args), _stream(stream)))
+
+
+def trispec_accept_scan(args: ScanArgs, stream=None):
+    _check(_lib.trispec_accept_scan(C.byref(args), _stream(stream)))
+
+
+def trispec_verify(tree: TreeArgs, attn: Optional[AttnArgs], lm: LmheadArgs, scan: ScanArgs, stream=None):
+    _check(_lib.trispec_verify(C.byref(tree), None if attn is None else C.byref(attn), C.byref(lm),
+                               C.byref(scan), _stream(stream)))

@@ -1,0 +1,401 @@
+// LM head fused with per-row softmax statistics (distributions p_i of Eq. 5 reduced to what
+// the margin rule of Eq. 8 and the acceptance test of Eq. 6 need). The [rows x V] logits
+// never reach global memory: each CTA streams a slice of the vocabulary through
+// tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) and its epilogue keeps, per row, a
+// running (max, sum of exponentials, top-1, top-2) in registers across all of its vocabulary
+// tiles. A small second kernel merges the per-slice partials and computes the drafted-token
+// probabilities.
+//
+// GEMM kernel layout
+//   M tile  = 128 rows = 2 sequence slots x 64 node slots (T <= 64; missing nodes are
+//             zero-filled by the TMA out-of-bounds rule, missing sequences are not loaded)
+//   N tile  = up to 256 vocabulary entries (one tcgen05.mma N), a multiple of 16
+//   K block = 64 bf16 = one 128-byte swizzle row; 4 MMAs of K = 16 per block
+//   warps 0-3: epilogue (one TMEM lane = one row per thread), warp 4: TMA producer,
+//   warp 5: MMA issuer and TMEM owner. Accumulators are double-buffered in TMEM
+//   (2 x 256 columns) so that the epilogue of tile i overlaps the MMAs of tile i + 1.
+//   CTA c works on M tile (c % n_mt) and vocabulary range (c / n_mt): CTAs that share a
+//   vocabulary range are neighbours and stream the same W tiles at the same time, so W is
+//   read from HBM once and re-hit in L2.
+#include <math.h>
+
+#include "host_common.h"
+#include "sm100.cuh"
+
+namespace trispec {
+
+constexpr int LM_BM = 128;
+constexpr int LM_BN = 256;
+constexpr int LM_BK = 64;
+constexpr int LM_STAGES = 4;
+constexpr int LM_A_BYTES = LM_BM * LM_BK * 2;   // 16 KB
+constexpr int LM_B_BYTES = LM_BN * LM_BK * 2;   // 32 KB
+constexpr int LM_BOX_BYTES = 64 * LM_BK * 2;    // one TMA box: 64 rows x 64 k
+constexpr int LM_STAGE_BYTES = LM_A_BYTES + LM_B_BYTES;
+constexpr int LM_THREADS = 192;
+constexpr int LM_SMEM_BYTES = LM_STAGES * LM_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct __align__(16) LmPartial {
+  float m, s, v1, v2;  // raw (unscaled) running max, sum of 2^((z-m)c), top-1 / top-2 raw logits
+  int i1, i2, pad0, pad1;
+};
+
+struct LmParams {
+  int T, d, V;
+  int n_seq;      // active sequences
+  int n_mt;       // M tiles = ceil(n_seq / 2)
+  int n_ranges;   // vocabulary ranges
+  float c;        // logit_scale * log2(e)
+  const int32_t* seq_index;
+  LmPartial* partial;  // [n_ranges][n_mt * 128]
+  int32_t* dev_status;
+};
+
+struct TileIter {
+  int u0, units, n_tiles;
+  __device__ TileIter(int V, int n_ranges, int r) {
+    const int V16 = (V + 15) >> 4;
+    u0 = static_cast<int>((static_cast<long long>(V16) * r) / n_ranges);
+    const int u1 = static_cast<int>((static_cast<long long>(V16) * (r + 1)) / n_ranges);
+    units = u1 - u0;
+    n_tiles = (units + 15) >> 4;
+  }
+  __device__ void tile(int t, int& n0, int& nw) const {
+    const int a = (units * t) / n_tiles, b = (units * (t + 1)) / n_tiles;
+    n0 = (u0 + a) << 4;
+    nw = (b - a) << 4;
+  }
+};
+
+__global__ void __launch_bounds__(LM_THREADS, 1)
+lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
+                   const LmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LM_STAGES * LM_STAGE_BYTES);
+  uint64_t* full_bar = bars;                      // [LM_STAGES]
+  uint64_t* empty_bar = bars + LM_STAGES;         // [LM_STAGES]
+  uint64_t* tmem_full = bars + 2 * LM_STAGES;     // [2]
+  uint64_t* tmem_empty = bars + 2 * LM_STAGES + 2;  // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LM_STAGES + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int mt = blockIdx.x % p.n_mt;
+  const int range = blockIdx.x / p.n_mt;
+  const TileIter tiles(p.V, p.n_ranges, range);
+  const int n_kb = p.d / LM_BK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < LM_STAGES; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 4); }
+    fence_mbar_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_h); prefetch_tmap(&tmap_w); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const int a0 = 2 * mt, a1 = 2 * mt + 1;
+      const int s0 = p.seq_index ? __ldg(p.seq_index + a0) : a0;
+      const bool has1 = a1 < p.n_seq;
+      const int s1 = has1 ? (p.seq_index ? __ldg(p.seq_index + a1) : a1) : 0;
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = 0; t < tiles.n_tiles; ++t) {
+        int n0, nw;
+        tiles.tile(t, n0, nw);
+        const int nbox = (nw + 63) >> 6;
+        const uint32_t tx = static_cast<uint32_t>((has1 ? 2 : 1) + nbox) * LM_BOX_BYTES;
+        for (int kb = 0; kb < n_kb; ++kb) {
+          mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
+          uint8_t* sa = smem + stage * LM_STAGE_BYTES;
+          uint8_t* sb = sa + LM_A_BYTES;
+          mbar_expect_tx(full_bar + stage, tx);
+          tma_load_3d(sa, &tmap_h, full_bar + stage, kb * LM_BK, 0, s0);
+          if (has1) tma_load_3d(sa + LM_BOX_BYTES, &tmap_h, full_bar + stage, kb * LM_BK, 0, s1);
+          for (int j = 0; j < nbox; ++j)
+            tma_load_2d(sb + j * LM_BOX_BYTES, &tmap_w, full_bar + stage, kb * LM_BK, n0 + 64 * j);
+          if (++stage == LM_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int t = 0; t < tiles.n_tiles; ++t) {
+        int n0, nw;
+        tiles.tile(t, n0, nw);
+        const int buf = t & 1;
+        mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * LM_BN);
+        const uint32_t idesc = idesc_bf16(LM_BM, nw, false, false);
+        for (int kb = 0; kb < n_kb; ++kb) {
+          mbar_wait(full_bar + stage, phase, p.dev_status);
+          tc_fence_after();
+          const uint32_t sa = base_u32 + stage * LM_STAGE_BYTES;
+          const uint64_t adesc = smem_desc_sw128(sa, 1024, 16);
+          const uint64_t bdesc = smem_desc_sw128(sa + LM_A_BYTES, 1024, 16);
+#pragma unroll
+          for (int k = 0; k < LM_BK / 16; ++k) {
+            // advancing 16 elements (32 bytes) along K inside the swizzle row: +2 in the
+            // 16-byte-granular start address field
+            tc_mma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
+          }
+          tc_commit(empty_bar + stage);
+          if (++stage == LM_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        tc_commit(tmem_full + buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3)
+    const int row = warp * 32 + lane;  // TMEM lane == row of the M tile
+    float m = -INFINITY, s = 0.f, v1 = -INFINITY, v2 = -INFINITY;
+    int i1 = -1, i2 = -1;
+    const float c = p.c;
+    for (int t = 0; t < tiles.n_tiles; ++t) {
+      int n0, nw;
+      tiles.tile(t, n0, nw);
+      const int buf = t & 1;
+      mbar_wait(tmem_full + buf, (t >> 1) & 1u, p.dev_status);
+      tc_fence_after();
+      const int ncols = min(nw, p.V - n0);  // valid columns of this tile
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(buf * LM_BN);
+      for (int c0 = 0; c0 < ncols; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c0, r);
+        tc_wait_ld();
+        const int nv = ncols - c0;  // >= 1
+        float cmax = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float v = __uint_as_float(r[j]);
+          if (j >= nv) { v = -INFINITY; r[j] = __float_as_uint(v); }
+          cmax = fmaxf(cmax, v);
+        }
+        if (cmax > m) {
+          s *= ex2f((m - cmax) * c);
+          m = cmax;
+        }
+        const float mc = m * c;
+        float acc = 0.f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc += ex2f(fmaf(__uint_as_float(r[j]), c, -mc));
+        s += acc;
+        if (cmax > v2) {
+          const int col0 = n0 + c0;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float v = __uint_as_float(r[j]);
+            if (v > v1) { v2 = v1; i2 = i1; v1 = v; i1 = col0 + j; }
+            else if (v > v2) { v2 = v; i2 = col0 + j; }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tmem_empty + buf);
+    }
+    LmPartial out;
+    out.m = m; out.s = s; out.v1 = v1; out.v2 = v2; out.i1 = i1; out.i2 = i2; out.pad0 = 0; out.pad1 = 0;
+    p.partial[static_cast<size_t>(range) * (p.n_mt * LM_BM) + mt * LM_BM + row] = out;
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Merge of the per-range partials + drafted-token logits. One block per active sequence.
+// ---------------------------------------------------------------------------------------
+struct LmFinalizeParams {
+  int T, d, V, n_mt, n_ranges;
+  float scale, c;
+  const int32_t* seq_index;
+  const LmPartial* partial;
+  const uint16_t *h, *W;
+  const int32_t *parent, *tok;
+  trispec_stats out;
+};
+
+constexpr int LM_FIN_THREADS = 256;
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+__global__ void __launch_bounds__(LM_FIN_THREADS)
+lmhead_finalize_kernel(const LmFinalizeParams p) {
+  __shared__ float lse_s[64];
+  const int a = blockIdx.x;
+  const int seq = p.seq_index ? __ldg(p.seq_index + a) : a;
+  const int T = p.T;
+  const long long row0 = static_cast<long long>(seq) * T;
+  const int tid = threadIdx.x;
+  if (tid < T) {
+    const size_t prow = static_cast<size_t>(a) * 64 + tid;
+    const size_t stride = static_cast<size_t>(p.n_mt) * LM_BM;
+    float M = -INFINITY;
+    for (int r = 0; r < p.n_ranges; ++r) M = fmaxf(M, p.partial[r * stride + prow].m);
+    float S = 0.f, v1 = -INFINITY, v2 = -INFINITY;
+    int i1 = -1, i2 = -1;
+    // larger value first, lower index on ties
+    auto better = [](float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia >= 0 && (ib < 0 || ia < ib)); };
+    for (int r = 0; r < p.n_ranges; ++r) {
+      const LmPartial q = p.partial[r * stride + prow];
+      S += q.s * ex2f((q.m - M) * p.c);
+      const float cv[2] = {q.v1, q.v2};
+      const int ci[2] = {q.i1, q.i2};
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        if (ci[k] < 0) continue;
+        if (better(cv[k], ci[k], v1, i1)) { v2 = v1; i2 = i1; v1 = cv[k]; i1 = ci[k]; }
+        else if (better(cv[k], ci[k], v2, i2)) { v2 = cv[k]; i2 = ci[k]; }
+      }
+    }
+    const float lse = M * p.scale + logf(S);
+    const long long o = row0 + tid;
+    p.out.max[o] = M * p.scale;
+    p.out.lse[o] = lse;
+    p.out.top1_val[o] = v1 * p.scale;
+    p.out.top2_val[o] = v2 * p.scale;
+    p.out.top1_idx[o] = i1;
+    p.out.top2_idx[o] = i2;
+    p.out.p_top1[o] = expf(v1 * p.scale - lse);
+    p.out.p_top2[o] = expf(v2 * p.scale - lse);
+    lse_s[tid] = lse;
+    if (tid == 0) {
+      p.out.draft_logit[o] = __int_as_float(0x7fc00000);
+      p.out.p_draft[o] = __int_as_float(0x7fc00000);
+    }
+  }
+  __syncthreads();
+  // drafted-token logit z[parent(c)][tok[c]]: one warp per child, 16-byte loads
+  const int warp = tid >> 5, lane = tid & 31;
+  for (int cnode = 1 + warp; cnode < T; cnode += LM_FIN_THREADS / 32) {
+    const int par = __ldg(p.parent + row0 + cnode);
+    const int tk = __ldg(p.tok + row0 + cnode);
+    float dl = __int_as_float(0x7fc00000), pd = dl;
+    if (par >= 0 && par < cnode && tk >= 0 && tk < p.V) {
+      const uint4* hv = reinterpret_cast<const uint4*>(p.h + (row0 + par) * p.d);
+      const uint4* wv = reinterpret_cast<const uint4*>(p.W + static_cast<long long>(tk) * p.d);
+      float acc = 0.f;
+      for (int i = lane; i < p.d / 8; i += 32) {
+        const uint4 x = __ldg(hv + i), y = __ldg(wv + i);
+        acc = fmaf(bf16_lo(x.x), bf16_lo(y.x), acc); acc = fmaf(bf16_hi(x.x), bf16_hi(y.x), acc);
+        acc = fmaf(bf16_lo(x.y), bf16_lo(y.y), acc); acc = fmaf(bf16_hi(x.y), bf16_hi(y.y), acc);
+        acc = fmaf(bf16_lo(x.z), bf16_lo(y.z), acc); acc = fmaf(bf16_hi(x.z), bf16_hi(y.z), acc);
+        acc = fmaf(bf16_lo(x.w), bf16_lo(y.w), acc); acc = fmaf(bf16_hi(x.w), bf16_hi(y.w), acc);
+      }
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      dl = acc * p.scale;
+      pd = expf(dl - lse_s[par]);
+    }
+    if (lane == 0) {
+      p.out.draft_logit[row0 + cnode] = dl;
+      p.out.p_draft[row0 + cnode] = pd;
+    }
+  }
+}
+
+static int lm_plan(const trispec_lmhead_args* a, int* n_seq, int* n_mt, int* n_ranges) {
+  if (!a || a->B <= 0 || a->T <= 0 || a->d <= 0 || a->V <= 0) return TRISPEC_ERR_INVALID_ARG;
+  if (a->T > 64 || (a->d % LM_BK) != 0 || a->V < 2) return TRISPEC_ERR_UNSUPPORTED;
+  *n_seq = a->seq_index ? a->B_active : a->B;
+  if (*n_seq <= 0 || *n_seq > a->B) return TRISPEC_ERR_INVALID_ARG;
+  *n_mt = (*n_seq + 1) / 2;
+  const int sms = device_sm_count();
+  int r = sms / *n_mt;
+  if (r < 1) r = 1;
+  const int V16 = (a->V + 15) / 16;
+  if (r > V16) r = V16;
+  *n_ranges = r;
+  return TRISPEC_OK;
+}
+
+}  // namespace trispec
+
+extern "C" size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a) {
+  using namespace trispec;
+  int n_seq, n_mt, n_ranges;
+  if (lm_plan(a, &n_seq, &n_mt, &n_ranges) != TRISPEC_OK) return 0;
+  return static_cast<size_t>(n_ranges) * n_mt * LM_BM * sizeof(LmPartial);
+}
+
+extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) {
+  using namespace trispec;
+  int n_seq, n_mt, n_ranges;
+  int rc = lm_plan(a, &n_seq, &n_mt, &n_ranges);
+  if (rc != TRISPEC_OK) return rc;
+  if (!a->h || !a->W || !a->parent || !a->tok || !a->workspace) return TRISPEC_ERR_INVALID_ARG;
+  if (!aligned16(a->h) || !aligned16(a->W) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
+    return TRISPEC_ERR_INVALID_ARG;
+  if (!(a->logit_scale > 0.f) || !isfinite(a->logit_scale)) return TRISPEC_ERR_INVALID_ARG;
+  const trispec_stats& o = a->out;
+  if (!o.max || !o.lse || !o.top1_val || !o.top2_val || !o.p_top1 || !o.p_top2 || !o.top1_idx || !o.top2_idx ||
+      !o.draft_logit || !o.p_draft)
+    return TRISPEC_ERR_INVALID_ARG;
+  if (a->workspace_bytes < trispec_lmhead_stats_workspace(a)) return TRISPEC_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  CUtensorMap tm_h, tm_w;
+  {
+    const uint64_t dims[3] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->T), static_cast<uint64_t>(a->B)};
+    const uint64_t strides[2] = {static_cast<uint64_t>(a->d) * 2, static_cast<uint64_t>(a->d) * 2 * a->T};
+    const uint32_t box[3] = {LM_BK, 64, 1};
+    if (!encode_tmap_bf16(&tm_h, a->h, 3, dims, strides, box)) return TRISPEC_ERR_CUDA;
+  }
+  {
+    const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
+    const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
+    const uint32_t box[2] = {LM_BK, 64};
+    if (!encode_tmap_bf16(&tm_w, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    TRISPEC_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         LM_SMEM_BYTES));
+    attr_set = true;
+  }
+  LmParams p;
+  p.T = a->T; p.d = a->d; p.V = a->V;
+  p.n_seq = n_seq; p.n_mt = n_mt; p.n_ranges = n_ranges;
+  p.c = a->logit_scale * kLog2e;
+  p.seq_index = a->seq_index;
+  p.partial = static_cast<LmPartial*>(a->workspace);
+  p.dev_status = a->dev_status;
+  lmhead_gemm_kernel<<<n_mt * n_ranges, LM_THREADS, LM_SMEM_BYTES, st>>>(tm_h, tm_w, p);
+  count_launch();
+  TRISPEC_CUDA_OK(cudaGetLastError());
+
+  LmFinalizeParams f;
+  f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges;
+  f.scale = a->logit_scale; f.c = p.c;
+  f.seq_index = a->seq_index;
+  f.partial = p.partial;
+  f.h = static_cast<const uint16_t*>(a->h);
+  f.W = static_cast<const uint16_t*>(a->W);
+  f.parent = a->parent; f.tok = a->tok;
+  f.out = a->out;
+  lmhead_finalize_kernel<<<n_seq, LM_FIN_THREADS, 0, st>>>(f);
+  count_launch();
+  TRISPEC_CUDA_OK(cudaGetLastError());
+  return TRISPEC_OK;
+}

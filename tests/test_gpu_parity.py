@@ -1,0 +1,154 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs, element by element at sizes that span several tiles and ragged tails."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import trispec_oracle as orc
+from paper_2601_23180_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H():
+    import tests.gpu_helpers as h
+    return h
+
+
+# ------------------------------------------------------------------------------ tree mask
+@pytest.mark.parametrize("name", gen.CONFIG_ORDER)
+def test_tree_mask_bit_exact(H, name):
+    cfg = gen.CONFIGS[name]
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(cfg.B)])
+    mask, depth = H.run_tree_mask(H.i32_dev(parent))
+    ref_mask, ref_depth = orc.build_tree_mask(parent)
+    assert np.array_equal(mask.cpu().numpy().view(np.uint64), ref_mask)
+    assert np.array_equal(depth.cpu().numpy(), ref_depth)
+
+
+def test_tree_mask_edge_cases(H):
+    # single node; T = 64 chain (bit 63 set); malformed parents are flagged, not followed
+    for parent in (np.array([[-1]], dtype=np.int32), np.arange(-1, 63, dtype=np.int32)[None]):
+        mask, depth = H.run_tree_mask(H.i32_dev(parent))
+        ref_mask, ref_depth = orc.build_tree_mask(parent)
+        assert np.array_equal(mask.cpu().numpy().view(np.uint64), ref_mask)
+        assert np.array_equal(depth.cpu().numpy(), ref_depth)
+    bad = np.array([[-1, 0, 2, 1], [-1, 0, 0, 7]], dtype=np.int32)
+    mask, depth = H.run_tree_mask(H.i32_dev(bad))
+    m = mask.cpu().numpy()
+    assert m[0, 2] == 0 and depth[0, 2].item() == -1 and m[0, 1] == 3
+    assert m[1, 3] == 0 and depth[1, 3].item() == -1
+
+
+# ------------------------------------------------------------------------------ accept scan
+@pytest.mark.parametrize("mode", [gen.MODE_PROXY, gen.MODE_TARGET])
+@pytest.mark.parametrize("name,B", [("proxy_tree", 37), ("llama_tree", 16), ("tiny_chain", 5)])
+def test_scan_bit_exact_on_oracle_stats(H, name, B, mode):
+    cfg = gen.small_variant(gen.CONFIGS[name], B=B, V=2048, d=128, rho=0.3,
+                            logit_scale=3.6 / (0.02 * math.sqrt(128)))
+    inp = gen.make_inputs(cfg, with_attention=False)
+    st = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale)
+    # the scan decides in fp32: give both sides the same fp32 probabilities
+    st32 = {"p_top1": st["p_top1"].astype(np.float32), "p_top2": st["p_top2"].astype(np.float32),
+            "top1_idx": st["top1_idx"]}
+    active = (np.arange(B) % 5 != 3).astype(np.uint8)
+    for lam in (0.5, 0.0, 1.5):
+        ref = orc.accept_scan(st32["p_top1"].astype(np.float64), st32["p_top2"].astype(np.float64),
+                              st32["top1_idx"], inp["parent"], inp["tok"], lam, mode=mode, active=active)
+        got = H.run_scan(st32, inp["parent"], inp["tok"], lam, mode, active=active)
+        clean = ref["near_thr"] == 0
+        for k in ("accept_len", "escalate", "bonus_tok", "last_node", "path"):
+            assert np.array_equal(got[k][clean], ref[k][clean]), (k, lam)
+        assert np.array_equal(got["near_thr"], ref["near_thr"])
+        if clean.all():
+            assert got["n_escalated"][0] == ref["n_escalated"]
+            assert np.array_equal(got["esc_index"], ref["esc_index"])
+
+
+def test_scan_start_node_and_large_batch(H):
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=3000, V=512, d=64, rho=0.2,
+                            logit_scale=3.6 / (0.02 * 8.0))
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(cfg.B)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(cfg.B)])
+    g = np.random.default_rng(0)
+    # synthetic statistics: top-1 is a child's token with probability 0.7
+    top1 = np.zeros((cfg.B, cfg.T), dtype=np.int64)
+    for b in range(cfg.B):
+        for r in range(cfg.T):
+            kids = np.nonzero(parent[b] == r)[0]
+            top1[b, r] = tok[b, g.choice(kids)] if len(kids) and g.random() < 0.7 else g.integers(0, cfg.V)
+    p1 = g.uniform(0.4, 1.0, (cfg.B, cfg.T)).astype(np.float32)
+    p2 = (p1 * g.uniform(0.0, 0.5, (cfg.B, cfg.T))).astype(np.float32)
+    st = {"p_top1": p1, "p_top2": p2, "top1_idx": top1}
+    start = g.integers(0, 3, cfg.B).astype(np.int32)
+    for mode, sn in ((gen.MODE_PROXY, None), (gen.MODE_TARGET, start)):
+        ref = orc.accept_scan(p1.astype(np.float64), p2.astype(np.float64), top1, parent, tok, 0.5, mode=mode,
+                              start_node=sn)
+        got = H.run_scan(st, parent, tok, 0.5, mode, start_node=sn)
+        clean = ref["near_thr"] == 0
+        for k in ("accept_len", "escalate", "bonus_tok", "last_node", "path"):
+            assert np.array_equal(got[k][clean], ref[k][clean]), k
+        esc = np.nonzero(got["escalate"])[0]
+        assert got["n_escalated"][0] == len(esc)
+        assert np.array_equal(got["esc_index"][:len(esc)], esc) and (got["esc_index"][len(esc):] == -1).all()
+
+
+# ------------------------------------------------------------------------------ LM-head stats
+LM_CASES = [
+    # name, overrides: several M tiles, several vocabulary tiles per CTA, ragged vocabulary tail
+    ("tiny_chain", dict(V=5000, d=256)),
+    ("proxy_tree", dict(B=3, V=40011, d=512)),
+    ("proxy_tree", dict(B=5, V=151936 // 8, d=192, logit_scale=3.6 / (0.02 * math.sqrt(192)))),
+    ("target_escalated", dict(B=7, n_active=3, V=9000, d=320, logit_scale=3.6 / (0.02 * math.sqrt(320)))),
+    ("llama_tree", dict(B=2, V=128256 // 4, d=1024, logit_scale=3.6 / (0.02 * 32.0))),
+]
+
+
+@pytest.mark.parametrize("name,over", LM_CASES)
+def test_lmhead_stats_against_oracle(H, name, over):
+    over = dict(over)
+    if "logit_scale" not in over:
+        over["logit_scale"] = 3.6 / (0.02 * math.sqrt(over["d"]))
+    cfg = gen.small_variant(gen.CONFIGS[name], rho=0.2, **over)
+    inp = gen.make_inputs(cfg, with_attention=False)
+    dev = H.to_device(inp)
+    got = H.run_lmhead(dev, cfg)
+    seqs = list(range(cfg.B)) if inp["seq_index"] is None else [int(s) for s in inp["seq_index"]]
+    ref = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale, seqs=seqs)
+    n_tie = H.check_stats(got, ref, seqs, cfg.T)
+    assert n_tie <= 0.02 * len(seqs) * cfg.T + 2
+    # rows of sequences that were not asked for stay untouched
+    for b in range(cfg.B):
+        if b not in seqs:
+            assert np.isnan(got["lse"][b]).all() and (got["top1_idx"][b] == -1).all()
+
+
+def test_lmhead_tiny_vocab_and_argument_errors(H):
+    import torch
+    from paper_2601_23180_b200 import binding as ts
+    # V = 19 (one 32-wide tile with 13 masked columns), duplicated maximum -> margin exactly 0
+    cfg = gen.small_variant(gen.CONFIGS["tiny_chain"], V=19, d=64, logit_scale=2.0)
+    inp = gen.make_inputs(cfg, with_attention=False)
+    inp["W"][7] = inp["W"][3]
+    dev = H.to_device(inp)
+    got = H.run_lmhead(dev, cfg)
+    ref = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale)
+    for r in range(cfg.T):
+        assert abs(got["lse"][0, r] - ref["lse"][0, r]) < 1e-3
+        if ref["top1_idx"][0, r] == 3:
+            assert got["top1_idx"][0, r] == 3 and got["top2_idx"][0, r] == 7
+            assert got["p_top1"][0, r] == got["p_top2"][0, r]
+    # argument errors are reported before any launch
+    st = ts.alloc_stats(cfg.B, cfg.T)
+    a = ts.lmhead_args(dev["h"], dev["W"], dev["parent"], dev["tok"], cfg.logit_scale, st)
+    n0 = ts.launch_count()
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_lmhead_stats(a)            # no workspace
+    assert e.value.code == 1 and ts.launch_count() == n0
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    a.workspace, a.workspace_bytes = ws.data_ptr(), 256
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_lmhead_stats(a)            # workspace too small
+    assert e.value.code == 3 and ts.launch_count() == n0
