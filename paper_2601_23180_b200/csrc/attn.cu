@@ -1,3 +1,502 @@
+// Verification attention (the attention of the parallel verification pass, Eq. 2 / Eq. 5):
+// every draft-tree node attends to the whole committed context plus the tree keys its mask
+// row allows. Split-KV: one CTA handles (sequence, KV head, M tile, KV split) and writes an
+// unnormalised partial (O, m, l); a second kernel merges the splits.
+//
+// GQA packing: the G = Hq / Hkv query heads that share a KV head are stacked on the M axis,
+// row = node_local * G + head_in_group, so one K/V tile serves all of them. An M tile holds
+// NPT = min(128 / G, 64) nodes.
+//
+// Per 64-key tile:  S = Q K^T  (tcgen05.mma M=128, N=64, K=128, both operands K-major)
+//                   online softmax in registers, one TMEM lane (row) per thread, exp2 domain,
+//                   lazy rescaling of O (only when the running max grows by more than 2^8)
+//                   P (bf16) -> shared memory, O += P V (V is the MN-major B operand)
+// S is double-buffered in TMEM so that S(t+1) is computed while the softmax of tile t runs.
+// K/V tiles arrive by TMA (no multicast) through a 2-stage mbarrier ring; two CTAs fit on one
+// SM (shared memory ~111 KB, 256 TMEM columns each) and overlap each other's phases.
+#include <math.h>
+
 #include "host_common.h"
-extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) { (void)a; return 0; }
-extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) { (void)a; (void)stream; return TRISPEC_ERR_UNSUPPORTED; }
+#include "sm100.cuh"
+
+namespace trispec {
+
+constexpr int AT_BM = 128;      // rows per M tile
+constexpr int AT_BN = 64;       // keys per tile (= paged block size)
+constexpr int AT_D = 128;
+constexpr int AT_STAGES = 2;
+constexpr int AT_BOX_BYTES = 64 * 64 * 2;               // 64 rows x 64 elements
+constexpr int AT_Q_BYTES = AT_BM * AT_D * 2;            // 32 KB (2 boxes of 128 rows x 64)
+constexpr int AT_KV_STAGE_BYTES = 4 * AT_BOX_BYTES;     // K (2 boxes) + V (2 boxes) = 32 KB
+constexpr int AT_P_BYTES = AT_BM * AT_BN * 2;           // 16 KB
+constexpr int AT_THREADS = 192;
+constexpr int AT_SMEM_USED = AT_Q_BYTES + AT_STAGES * AT_KV_STAGE_BYTES + AT_P_BYTES + 128;
+// two CTAs per SM: 2 x (dynamic + 1 KB reserved) must fit 228 KB, which leaves 896 bytes of alignment slack
+constexpr int AT_SMEM_BYTES = AT_SMEM_USED + 896;
+constexpr int AT_TMEM_COLS = 256;                        // S0 [0,64) S1 [64,128) O [128,256)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;                // log2 units
+
+struct AttnParams {
+  int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split;
+  int paged, max_blocks_per_seq, num_blocks;
+  float scale_log2;
+  const int32_t *block_table, *ctx_len, *seq_index;
+  const uint64_t* mask;
+  float* part_o;    // [items][128][128]
+  float* part_ml;   // [items][128][2]
+  int32_t* dev_status;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+__global__ void __launch_bounds__(AT_THREADS, 2)
+verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                         const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kt,
+                         const __grid_constant__ CUtensorMap tm_vt, const AttnParams p) {
+  // ---- which work item
+  int idx = blockIdx.x;
+  const int mtile = idx % p.n_mt; idx /= p.n_mt;
+  const int split = idx % p.n_splits; idx /= p.n_splits;
+  const int g = idx % p.Hkv;
+  const int a = idx / p.Hkv;
+  const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
+  const int L = __ldg(p.ctx_len + b);
+  const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
+  const int last_split = max(0, (n_ctx_tiles + p.tiles_per_split - 1) / p.tiles_per_split - 1);
+  if (split > last_split) return;            // nothing to do: the merge kernel skips it too
+  const int t_begin = split * p.tiles_per_split;
+  const int t_end = min(n_ctx_tiles, t_begin + p.tiles_per_split);
+  const bool has_tree = (split == last_split);
+  const int n_tiles = (t_end - t_begin) + (has_tree ? 1 : 0);   // >= 1
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
+  if (base_u32 - smem_u32(smem_raw) > static_cast<uint32_t>(AT_SMEM_BYTES - AT_SMEM_USED)) {
+    if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 7);   // shared memory window misaligned
+    return;
+  }
+  uint8_t* sQ = smem;
+  uint8_t* sKV = smem + AT_Q_BYTES;
+  uint8_t* sP = sKV + AT_STAGES * AT_KV_STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + AT_P_BYTES);
+  uint64_t* q_bar = bars;            // 1
+  uint64_t* full_bar = bars + 1;     // [2]
+  uint64_t* empty_bar = bars + 3;    // [2]
+  uint64_t* s_bar = bars + 5;        // [2]
+  uint64_t* o_bar = bars + 7;        // 1
+  uint64_t* p_bar = bars + 8;        // 1, 128 arrivals
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(q_bar, 1);
+    for (int i = 0; i < AT_STAGES; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
+    mbar_init(s_bar, 1); mbar_init(s_bar + 1, 1); mbar_init(o_bar, 1); mbar_init(p_bar, 128);
+    fence_mbar_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(tmem_slot, AT_TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kt); prefetch_tmap(&tm_vt);
+      const int rows = p.NPT * p.G;
+      mbar_expect_tx(q_bar, static_cast<uint32_t>(rows) * AT_D * 2);
+      tma_load_4d(sQ, &tm_q, q_bar, 0, g * p.G, mtile * p.NPT, b);
+      tma_load_4d(sQ + AT_BM * 128, &tm_q, q_bar, 64, g * p.G, mtile * p.NPT, b);
+    }
+    int stage = 0;
+    uint32_t phase = 0;
+    int blk_cache = 0;
+    for (int i = 0; i < n_tiles; ++i) {
+      const bool tree = has_tree && (i == n_tiles - 1);
+      const int t = t_begin + i;
+      int blk = 0;
+      if (p.paged && !tree) {
+        // block ids are fetched 32 at a time by the whole warp
+        if ((i & 31) == 0) {
+          const int tt = t + lane;
+          int v = 0;
+          if (tt < t_end) v = __ldg(p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq + tt);
+          if (v < 0 || v >= p.num_blocks) {
+            if (tt < t_end && p.dev_status) atomicExch(p.dev_status, 6);   // bad block id: clamped
+            v = 0;
+          }
+          blk_cache = v;
+        }
+        blk = __shfl_sync(0xffffffffu, blk_cache, i & 31);
+      }
+      if (lane == 0) {
+        mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
+        uint8_t* sk = sKV + stage * AT_KV_STAGE_BYTES;
+        uint8_t* sv = sk + 2 * AT_BOX_BYTES;
+        mbar_expect_tx(full_bar + stage, AT_KV_STAGE_BYTES);
+        if (tree) {
+          tma_load_4d(sk, &tm_kt, full_bar + stage, 0, g, 0, b);
+          tma_load_4d(sk + AT_BOX_BYTES, &tm_kt, full_bar + stage, 64, g, 0, b);
+          tma_load_4d(sv, &tm_vt, full_bar + stage, 0, g, 0, b);
+          tma_load_4d(sv + AT_BOX_BYTES, &tm_vt, full_bar + stage, 64, g, 0, b);
+        } else {
+          const int c2 = p.paged ? 0 : t * AT_BN;
+          const int c3 = p.paged ? blk : b;
+          tma_load_4d(sk, &tm_k, full_bar + stage, 0, g, c2, c3);
+          tma_load_4d(sk + AT_BOX_BYTES, &tm_k, full_bar + stage, 64, g, c2, c3);
+          tma_load_4d(sv, &tm_v, full_bar + stage, 0, g, c2, c3);
+          tma_load_4d(sv + AT_BOX_BYTES, &tm_v, full_bar + stage, 64, g, c2, c3);
+        }
+      }
+      if (++stage == AT_STAGES) { stage = 0; phase ^= 1u; }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = idesc_bf16(AT_BM, AT_BN, false, false);
+      const uint32_t idesc_o = idesc_bf16(AT_BM, AT_D, false, true);
+      const uint32_t sQ_u = base_u32, sKV_u = base_u32 + AT_Q_BYTES, sP_u = sKV_u + AT_STAGES * AT_KV_STAGE_BYTES;
+      auto issue_pv = [&](int i) {
+        const int stage = i & 1;
+        const uint32_t sv = sKV_u + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < AT_BN / 16; ++kk) {
+          const uint64_t ad = smem_desc_sw128(sP_u + kk * 32, 1024, 16);
+          // V: MN-major, 64-dim blocks 8 KB apart (LBO), 8-key groups 1 KB apart (SBO)
+          const uint64_t bd = smem_desc_sw128(sv + kk * 2048, 1024, AT_BOX_BYTES);
+          tc_mma_ss(tmem_base + 128, ad, bd, idesc_o, (i | kk) != 0);
+        }
+        tc_commit(empty_bar + stage);
+        tc_commit(o_bar);
+      };
+      mbar_wait(q_bar, 0, p.dev_status);
+      for (int i = 0; i < n_tiles; ++i) {
+        const int stage = i & 1, buf = i & 1;
+        mbar_wait(full_bar + stage, (i >> 1) & 1u, p.dev_status);
+        tc_fence_after();
+        const uint32_t sk = sKV_u + stage * AT_KV_STAGE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < AT_D / 16; ++kk) {
+          const uint64_t ad = smem_desc_sw128(sQ_u + (kk >> 2) * (AT_BM * 128) + (kk & 3) * 32, 1024, 16);
+          const uint64_t bd = smem_desc_sw128(sk + (kk >> 2) * AT_BOX_BYTES + (kk & 3) * 32, 1024, 16);
+          tc_mma_ss(tmem_base + buf * AT_BN, ad, bd, idesc_s, kk != 0);
+        }
+        tc_commit(s_bar + buf);
+        if (i > 0) {
+          mbar_wait(p_bar, (i - 1) & 1u, p.dev_status);   // P(i-1) is in shared memory
+          tc_fence_after();
+          issue_pv(i - 1);
+        }
+      }
+      mbar_wait(p_bar, (n_tiles - 1) & 1u, p.dev_status);
+      tc_fence_after();
+      issue_pv(n_tiles - 1);
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax (warps 0-3)
+    const int row = warp * 32 + lane;
+    const int node = mtile * p.NPT + row / p.G;
+    const bool row_valid = (row < p.NPT * p.G) && (node < p.T);
+    const uint64_t mrow = row_valid ? __ldg(p.mask + static_cast<long long>(b) * p.T + node) : 0ull;
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    float m_ref = -INFINITY, l = 0.f;
+
+    for (int i = 0; i < n_tiles; ++i) {
+      const int stage = i & 1, buf = i & 1;
+      const bool tree = has_tree && (i == n_tiles - 1);
+      mbar_wait(s_bar + buf, (i >> 1) & 1u, p.dev_status);
+      tc_fence_after();
+      uint32_t sr[64];
+      {
+        uint32_t r0[32], r1[32];
+        tmem_ld32(tmem_base + lane_base + buf * AT_BN, r0);
+        tmem_ld32(tmem_base + lane_base + buf * AT_BN + 32, r1);
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { sr[j] = r0[j]; sr[32 + j] = r1[j]; }
+      }
+      // which keys of this tile does this row see
+      uint64_t vis;
+      int nvalid = AT_BN;
+      if (tree) {
+        vis = mrow;
+      } else {
+        nvalid = min(AT_BN, L - (t_begin + i) * AT_BN);
+        vis = (nvalid >= 64) ? ~0ull : ((1ull << nvalid) - 1ull);
+      }
+      float tmax = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 64; ++j) {
+        float v = __uint_as_float(sr[j]) * p.scale_log2;
+        if (!((vis >> j) & 1ull)) v = -INFINITY;
+        sr[j] = __float_as_uint(v);
+        tmax = fmaxf(tmax, v);
+      }
+      if (i > 0) {
+        mbar_wait(o_bar, (i - 1) & 1u, p.dev_status);   // P V of the previous tile is complete
+        tc_fence_after();
+      }
+      if (i == 0) {
+        m_ref = tmax;
+      } else {
+        const bool need = tmax > m_ref + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, need)) {
+          float f = 1.f;
+          if (need) { f = (m_ref == -INFINITY) ? 0.f : ex2f(m_ref - tmax); m_ref = tmax; l *= f; }
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_base + lane_base + 128 + c * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * f);
+            tmem_st32(tmem_base + lane_base + 128 + c * 32, o);
+          }
+          tc_wait_st();
+        }
+      }
+      const float mu = (m_ref == -INFINITY) ? 0.f : m_ref;
+      float lsum = 0.f;
+      uint8_t* prow = sP + row * 128;
+#pragma unroll
+      for (int cch = 0; cch < 8; ++cch) {
+        float e[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { e[j] = ex2f(__uint_as_float(sr[cch * 8 + j]) - mu); lsum += e[j]; }
+        uint4 pk;
+        pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]);
+        pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
+        *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk;
+      }
+      l += lsum;
+      if (nvalid < AT_BN) {
+        // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
+        uint8_t* sv = sKV + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
+        for (int e = threadIdx.x; e < (AT_BN - nvalid) * 16; e += 128) {
+          const int r = nvalid + (e >> 4), c16 = e & 15;
+          *reinterpret_cast<uint4*>(sv + (c16 >> 3) * AT_BOX_BYTES + r * 128 + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(p_bar);
+    }
+    // ---------------------------------------------------------------- epilogue
+    mbar_wait(o_bar, (n_tiles - 1) & 1u, p.dev_status);
+    tc_fence_after();
+    const size_t item = static_cast<size_t>(blockIdx.x);
+    float* po = p.part_o + (item * AT_BM + row) * AT_D;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      uint32_t o[32];
+      tmem_ld32(tmem_base + lane_base + 128 + c * 32, o);
+      tc_wait_ld();
+      if (row_valid) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4)
+          *reinterpret_cast<float4*>(po + c * 32 + j) =
+              make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
+                          __uint_as_float(o[j + 3]));
+      }
+    }
+    if (row_valid) {
+      float2 ml = make_float2(m_ref, l);
+      *reinterpret_cast<float2*>(p.part_ml + (item * AT_BM + row) * 2) = ml;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, AT_TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Merge of the KV splits: one warp per output row (sequence, node, query head).
+// ---------------------------------------------------------------------------------------
+struct AttnMergeParams {
+  int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split, n_seq;
+  const int32_t *ctx_len, *seq_index;
+  const float *part_o, *part_ml;
+  uint16_t* o;   // bf16 [B][T][Hq][128]
+  float* lse;    // [B][Hq][T] or null
+};
+
+__global__ void __launch_bounds__(256)
+verify_attn_merge_kernel(const AttnMergeParams p) {
+  const int lane = threadIdx.x & 31;
+  const long long w = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  const long long total = static_cast<long long>(p.n_seq) * p.T * p.Hq;
+  if (w >= total) return;
+  const int hq = static_cast<int>(w % p.Hq);
+  const int node = static_cast<int>((w / p.Hq) % p.T);
+  const int a = static_cast<int>(w / (static_cast<long long>(p.Hq) * p.T));
+  const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
+  const int g = hq / p.G, j = hq % p.G;
+  const int mtile = node / p.NPT;
+  const int row = (node % p.NPT) * p.G + j;
+  const int L = __ldg(p.ctx_len + b);
+  const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
+  const int n_valid = max(0, (n_ctx_tiles + p.tiles_per_split - 1) / p.tiles_per_split - 1) + 1;
+  const size_t item0 = ((static_cast<size_t>(a) * p.Hkv + g) * p.n_splits) * p.n_mt + mtile;
+  float M = -INFINITY;
+  for (int s = 0; s < n_valid; ++s) {
+    const size_t item = item0 + static_cast<size_t>(s) * p.n_mt;
+    M = fmaxf(M, __ldg(p.part_ml + (item * AT_BM + row) * 2));
+  }
+  float Lsum = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_valid; ++s) {
+    const size_t item = item0 + static_cast<size_t>(s) * p.n_mt;
+    const float2 ml = __ldg(reinterpret_cast<const float2*>(p.part_ml + (item * AT_BM + row) * 2));
+    const float wgt = (ml.x == -INFINITY) ? 0.f : ex2f(ml.x - M);
+    Lsum += ml.y * wgt;
+    const float4 v = __ldg(reinterpret_cast<const float4*>(p.part_o + (item * AT_BM + row) * AT_D) + lane);
+    acc.x = fmaf(v.x, wgt, acc.x); acc.y = fmaf(v.y, wgt, acc.y);
+    acc.z = fmaf(v.z, wgt, acc.z); acc.w = fmaf(v.w, wgt, acc.w);
+  }
+  const float inv = 1.f / Lsum;
+  uint2 out;
+  out.x = pack_bf16(acc.x * inv, acc.y * inv);
+  out.y = pack_bf16(acc.z * inv, acc.w * inv);
+  uint16_t* orow = p.o + ((static_cast<size_t>(b) * p.T + node) * p.Hq + hq) * AT_D;
+  *reinterpret_cast<uint2*>(orow + lane * 4) = out;
+  if (p.lse && lane == 0) p.lse[(static_cast<size_t>(b) * p.Hq + hq) * p.T + node] = (M + log2f(Lsum)) * kLn2;
+}
+
+struct AttnPlan {
+  int n_seq, G, NPT, n_mt, tiles_max, tiles_per_split, n_splits;
+  size_t items;
+};
+
+static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
+  if (!a || a->B <= 0 || a->T <= 0 || a->Hq <= 0 || a->Hkv <= 0) return TRISPEC_ERR_INVALID_ARG;
+  if (a->D != AT_D || a->T > 64 || a->Hq % a->Hkv != 0) return TRISPEC_ERR_UNSUPPORTED;
+  const int G = a->Hq / a->Hkv;
+  if (!(G == 1 || G == 2 || G == 4 || G == 8 || G == 16)) return TRISPEC_ERR_UNSUPPORTED;
+  int Lmax;
+  if (a->kv_layout == TRISPEC_KV_CONTIGUOUS) {
+    if (a->Lmax < 0) return TRISPEC_ERR_INVALID_ARG;
+    Lmax = a->Lmax;
+  } else if (a->kv_layout == TRISPEC_KV_PAGED) {
+    if (a->block_size != AT_BN) return TRISPEC_ERR_UNSUPPORTED;
+    if (a->max_blocks_per_seq <= 0 || a->num_blocks <= 0) return TRISPEC_ERR_INVALID_ARG;
+    Lmax = a->max_blocks_per_seq * AT_BN;
+  } else {
+    return TRISPEC_ERR_INVALID_ARG;
+  }
+  pl->n_seq = a->seq_index ? a->B_active : a->B;
+  if (pl->n_seq <= 0 || pl->n_seq > a->B) return TRISPEC_ERR_INVALID_ARG;
+  pl->G = G;
+  pl->NPT = (AT_BM / G < 64) ? AT_BM / G : 64;
+  pl->n_mt = (a->T + pl->NPT - 1) / pl->NPT;
+  pl->tiles_max = (Lmax + AT_BN - 1) / AT_BN;
+  const long long fixed = static_cast<long long>(pl->n_seq) * a->Hkv * pl->n_mt;
+  const long long target = static_cast<long long>(device_sm_count()) * 2 * 8;   // ~8 waves of 2 CTAs/SM
+  long long c = (static_cast<long long>(pl->tiles_max) * fixed + target - 1) / target;
+  if (c < 16) c = 16;
+  if (c > pl->tiles_max) c = pl->tiles_max > 0 ? pl->tiles_max : 1;
+  pl->tiles_per_split = static_cast<int>(c);
+  pl->n_splits = pl->tiles_max > 0 ? (pl->tiles_max + pl->tiles_per_split - 1) / pl->tiles_per_split : 1;
+  pl->items = static_cast<size_t>(fixed) * pl->n_splits;
+  if (pl->items > 0x7fffffffull) return TRISPEC_ERR_UNSUPPORTED;
+  return TRISPEC_OK;
+}
+
+}  // namespace trispec
+
+extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) {
+  using namespace trispec;
+  AttnPlan pl;
+  if (attn_plan(a, &pl) != TRISPEC_OK) return 0;
+  return pl.items * AT_BM * (AT_D + 2) * sizeof(float);
+}
+
+extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
+  using namespace trispec;
+  AttnPlan pl;
+  int rc = attn_plan(a, &pl);
+  if (rc != TRISPEC_OK) return rc;
+  if (!a->q || !a->k_tree || !a->v_tree || !a->ctx_len || !a->mask || !a->o || !a->workspace)
+    return TRISPEC_ERR_INVALID_ARG;
+  if (pl.tiles_max > 0 && (!a->k_cache || !a->v_cache)) return TRISPEC_ERR_INVALID_ARG;
+  if (a->kv_layout == TRISPEC_KV_PAGED && !a->block_table) return TRISPEC_ERR_INVALID_ARG;
+  if (!aligned16(a->q) || !aligned16(a->k_tree) || !aligned16(a->v_tree) || !aligned16(a->k_cache) ||
+      !aligned16(a->v_cache) || !aligned16(a->o) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
+    return TRISPEC_ERR_INVALID_ARG;
+  if (!(a->scale > 0.f) || !isfinite(a->scale)) return TRISPEC_ERR_INVALID_ARG;
+  if (a->workspace_bytes < trispec_verify_attn_workspace(a)) return TRISPEC_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  const uint64_t D = AT_D, Hq = a->Hq, Hkv = a->Hkv, T = a->T, B = a->B;
+  CUtensorMap tm_q, tm_k, tm_v, tm_kt, tm_vt;
+  {
+    const uint64_t dims[4] = {D, Hq, T, B};
+    const uint64_t str[3] = {D * 2, Hq * D * 2, T * Hq * D * 2};
+    const uint32_t box[4] = {64, static_cast<uint32_t>(pl.G), static_cast<uint32_t>(pl.NPT), 1};
+    if (!encode_tmap_bf16(&tm_q, a->q, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+  }
+  {
+    const uint64_t dims[4] = {D, Hkv, T, B};
+    const uint64_t str[3] = {D * 2, Hkv * D * 2, T * Hkv * D * 2};
+    const uint32_t box[4] = {64, 1, 64, 1};
+    if (!encode_tmap_bf16(&tm_kt, a->k_tree, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+    if (!encode_tmap_bf16(&tm_vt, a->v_tree, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+  }
+  if (pl.tiles_max > 0) {
+    uint64_t dims[4], str[3];
+    if (a->kv_layout == TRISPEC_KV_CONTIGUOUS) {
+      dims[0] = D; dims[1] = Hkv; dims[2] = a->Lmax; dims[3] = B;
+      str[0] = D * 2; str[1] = Hkv * D * 2; str[2] = static_cast<uint64_t>(a->Lmax) * Hkv * D * 2;
+    } else {
+      dims[0] = D; dims[1] = Hkv; dims[2] = AT_BN; dims[3] = a->num_blocks;
+      str[0] = D * 2; str[1] = Hkv * D * 2; str[2] = static_cast<uint64_t>(AT_BN) * Hkv * D * 2;
+    }
+    const uint32_t box[4] = {64, 1, 64, 1};
+    if (!encode_tmap_bf16(&tm_k, a->k_cache, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+    if (!encode_tmap_bf16(&tm_v, a->v_cache, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+  } else {
+    tm_k = tm_kt;   // never dereferenced: every sequence has zero context tiles
+    tm_v = tm_vt;
+  }
+  TRISPEC_CUDA_OK(cudaFuncSetAttribute(verify_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       AT_SMEM_BYTES));
+  AttnParams p;
+  p.T = a->T; p.Hq = a->Hq; p.Hkv = a->Hkv; p.G = pl.G; p.NPT = pl.NPT; p.n_mt = pl.n_mt;
+  p.n_splits = pl.n_splits; p.tiles_per_split = pl.tiles_per_split;
+  p.paged = (a->kv_layout == TRISPEC_KV_PAGED); p.max_blocks_per_seq = a->max_blocks_per_seq;
+  p.num_blocks = a->num_blocks;
+  p.scale_log2 = a->scale * kLog2e;
+  p.block_table = a->block_table; p.ctx_len = a->ctx_len; p.seq_index = a->seq_index; p.mask = a->mask;
+  p.part_o = static_cast<float*>(a->workspace);
+  p.part_ml = p.part_o + pl.items * AT_BM * AT_D;
+  p.dev_status = a->dev_status;
+  verify_attn_split_kernel<<<static_cast<unsigned>(pl.items), AT_THREADS, AT_SMEM_BYTES, st>>>(tm_q, tm_k, tm_v, tm_kt,
+                                                                                                tm_vt, p);
+  count_launch();
+  TRISPEC_CUDA_OK(cudaGetLastError());
+
+  AttnMergeParams m;
+  m.T = a->T; m.Hq = a->Hq; m.Hkv = a->Hkv; m.G = pl.G; m.NPT = pl.NPT; m.n_mt = pl.n_mt;
+  m.n_splits = pl.n_splits; m.tiles_per_split = pl.tiles_per_split; m.n_seq = pl.n_seq;
+  m.ctx_len = a->ctx_len; m.seq_index = a->seq_index;
+  m.part_o = p.part_o; m.part_ml = p.part_ml;
+  m.o = static_cast<uint16_t*>(a->o); m.lse = a->lse;
+  const long long rows = static_cast<long long>(pl.n_seq) * a->T * a->Hq;
+  verify_attn_merge_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, st>>>(m);
+  count_launch();
+  TRISPEC_CUDA_OK(cudaGetLastError());
+  return TRISPEC_OK;
+}

@@ -152,3 +152,60 @@ def test_lmhead_tiny_vocab_and_argument_errors(H):
     with pytest.raises(ts.TrispecError) as e:
         ts.trispec_lmhead_stats(a)            # workspace too small
     assert e.value.code == 3 and ts.launch_count() == n0
+
+
+# ------------------------------------------------------------------------------ attention
+ATTN_CASES = [
+    # (name, overrides, ctx_len override)
+    ("tiny_chain", dict(), None),                                              # config 1 at full size
+    ("proxy_tree", dict(B=3, L=1000), None),                                   # ragged last tile
+    ("proxy_tree", dict(B=1, L=4096), None),                                   # several KV splits
+    ("target_escalated", dict(B=4, n_active=2, L=700), None),                  # G = 8: 4 M tiles, subset
+    ("llama_tree", dict(B=2, L=520), None),                                    # G = 4, T = 49
+    ("long_paged", dict(B=5, L=2100, L_min=70), None),                         # paged, ragged
+    ("long_paged", dict(B=4, L=300, L_min=1), [0, 1, 64, 65]),                 # empty / one-key contexts
+    ("proxy_tree", dict(B=2, L=64, Hq=8, Hkv=8), [64, 0]),                     # G = 1 (MHA)
+]
+
+
+@pytest.mark.parametrize("name,over,ctx", ATTN_CASES)
+def test_attention_against_oracle(H, name, over, ctx):
+    cfg = gen.small_variant(gen.CONFIGS[name], **over)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    if ctx is not None:
+        inp["ctx_len"] = np.array(ctx, dtype=np.int32)
+    dev = H.to_device(inp)
+    mask_dev, _ = H.run_tree_mask(dev["parent"])
+    o, lse = H.run_attn(dev, cfg, mask_dev)
+    seqs = list(range(cfg.B)) if inp["seq_index"] is None else [int(s) for s in inp["seq_index"]]
+    ref_mask, _ = orc.build_tree_mask(inp["parent"])
+    ref_o, ref_lse = orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], ref_mask, inp["k_cache"],
+                                     inp["v_cache"], inp["ctx_len"], 1.0 / math.sqrt(cfg.D),
+                                     block_table=inp["block_table"], block_size=cfg.block_size, seqs=seqs)
+    for b in range(cfg.B):
+        if b in seqs:
+            err = np.abs(o[b] - ref_o[b]).max()
+            assert err <= 2e-2, (b, err)                      # bf16 in, fp32 accumulate, bf16 out
+            assert np.abs(lse[b] - ref_lse[b]).max() <= 1e-3 * max(1.0, np.abs(ref_lse[b]).max())
+        else:
+            assert np.isnan(o[b]).all()                       # untouched
+
+
+def test_attention_argument_errors(H):
+    import torch
+    from paper_2601_23180_b200 import binding as ts
+    cfg = gen.small_variant(gen.CONFIGS["tiny_chain"], L=64)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    dev = H.to_device(inp)
+    mask_dev, _ = H.run_tree_mask(dev["parent"])
+    o = torch.zeros((cfg.B, cfg.T, cfg.Hq, cfg.D), dtype=torch.bfloat16, device="cuda")
+    a = ts.attn_args(dev["q"], dev["k_tree"], dev["v_tree"], mask_dev, dev["k_cache"], dev["v_cache"],
+                     dev["ctx_len"], 0.1, o)
+    n0 = ts.launch_count()
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_verify_attn(a)                              # no workspace
+    assert e.value.code == 1
+    a.D = 64
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_verify_attn(a)                              # unsupported head dim
+    assert e.value.code == 2 and ts.launch_count() == n0
