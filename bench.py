@@ -1,0 +1,332 @@
+#!/usr/bin/env python
+"""Benchmark of the TriSpec verify pass on B200.
+
+One "step" is one whole verify pass (tree mask -> tree-masked GQA attention -> LM-head softmax
+statistics -> acceptance scan) over one batch of seeded synthetic input, launched through the
+fused C-ABI call. The metric is verified draft tokens per second per verify pass.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints one JSON line (rank 0). With N > 1 (torchrun) every rank runs its own batch of the same
+shape (independent sequences, no data-path collective): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified_draft_tokens_per_s"
+UNIT = "draft tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_gemm_kernel launch on the bench
+# workload, from the ncu capture summarised in profiles/ (None until captured).
+LMHEAD_GEMM_DRAM_TRAFFIC = {"proxy_tree": None}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on a bounded sample of the workload
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(cfg, inp, n_attn_rows: int, n_lm_rows: int):
+    """Times the oracle on a sample of one verify pass and scales to the whole pass.
+    Returns (draft tokens/s, description, threads)."""
+    import numpy as np
+    from oracle import trispec_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    seqs = list(range(cfg.B)) if inp.get("seq_index") is None else [int(s) for s in inp["seq_index"]]
+    T = cfg.T
+    t0 = time.perf_counter()
+    mask, _ = orc.build_tree_mask(inp["parent"])
+    t_mask = time.perf_counter() - t0
+    # attention rows of one (sequence, KV head) group, so that the context is converted once
+    G = cfg.Hq // cfg.Hkv
+    samples = [(seqs[0], i % T, (i // T) % G) for i in range(n_attn_rows)]
+    t0 = time.perf_counter()
+    orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], mask, inp["k_cache"], inp["v_cache"], inp["ctx_len"],
+                    1.0 / math.sqrt(cfg.D), block_table=inp.get("block_table"), block_size=cfg.block_size,
+                    samples=samples)
+    t_attn = time.perf_counter() - t0
+    total_attn_rows = len(seqs) * T * cfg.Hq
+    # LM-head rows: the fp64 copy of W is made once per pass, then one matrix-vector product per row
+    t0 = time.perf_counter()
+    W64 = orc.bf16_to_f64(inp["W"])
+    t_w = time.perf_counter() - t0
+    sub = {k: inp[k][seqs[0]:seqs[0] + 1, :n_lm_rows] for k in ("h",)}
+    par = np.arange(-1, n_lm_rows - 1, dtype=np.int32)[None]
+    tok = inp["tok"][seqs[0]:seqs[0] + 1, :n_lm_rows]
+    t0 = time.perf_counter()
+    st = orc.lmhead_stats(sub["h"], inp["W"], par, tok, cfg.logit_scale, W64=W64)
+    t_lm = time.perf_counter() - t0
+    del W64
+    t0 = time.perf_counter()
+    p1 = np.tile(st["p_top1"][:, :1], (cfg.B, T))
+    orc.accept_scan(p1, p1 * 0.1, np.zeros((cfg.B, T), dtype=np.int64), inp["parent"], inp["tok"], cfg.lam, cfg.mode)
+    t_scan = time.perf_counter() - t0
+    t_pass = (t_mask + t_attn * total_attn_rows / n_attn_rows + t_w + t_lm * (len(seqs) * T) / n_lm_rows + t_scan)
+    desc = (f"{n_attn_rows} of {total_attn_rows} attention rows and {n_lm_rows} of {len(seqs) * T} LM-head rows "
+            f"(+ full mask, scan, one fp64 copy of W), scaled to one pass; measured {t_mask + t_attn + t_w + t_lm + t_scan:.1f} s")
+    return len(seqs) * cfg.k / t_pass, desc, threads
+
+
+def oracle_timed(cfg, inp, budget_s: float):
+    """Probe the oracle's per-row cost, then time a sample sized for about `budget_s` seconds
+    (the whole pass if it fits)."""
+    n_seq = cfg.B if cfg.n_active is None else cfg.n_active
+    tot_a, tot_l = n_seq * cfg.T * cfg.Hq, n_seq * cfg.T
+    v, _, _ = oracle_sample(cfg, inp, n_attn_rows=min(32, tot_a), n_lm_rows=min(2, tot_l))
+    est_full = n_seq * cfg.k / v
+    f = min(1.0, budget_s / est_full)
+    G = cfg.Hq // cfg.Hkv
+    na = max(1, min(int(f * tot_a), cfg.T * G))      # rows of one (sequence, KV head) group at most
+    nl = max(1, min(int(f * tot_l), cfg.T))
+    return oracle_sample(cfg, inp, n_attn_rows=na, n_lm_rows=nl)
+
+
+def run_reference(args, cfg, rank):
+    if rank != 0:
+        return
+    from paper_2601_23180_b200 import inputs as gen
+    inp = gen.make_inputs(cfg)
+    vals = []
+    for step in range(args.warmup + args.steps):
+        v, desc, threads = oracle_timed(cfg, inp, budget_s=4.0)
+        if step >= args.warmup:
+            vals.append(v)
+    value = len(vals) / sum(1.0 / v for v in vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg_tokens(cfg) / value,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "draft_tokens": cfg.k, "context": cfg.L, "Hq": cfg.Hq,
+                   "Hkv": cfg.Hkv, "hidden": cfg.d, "vocab": cfg.V},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def cfg_tokens(cfg):
+    n = cfg.B if cfg.n_active is None else cfg.n_active
+    return n * cfg.k
+
+
+# ---------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="proxy_tree")
+    ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "trispec" else args.warmup
+
+    from paper_2601_23180_b200 import inputs as gen
+    cfg = gen.CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verify pass has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2601_23180_b200 import build as tbuild
+    if rank == 0:
+        tbuild.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2601_23180_b200 import binding as ts
+    from paper_2601_23180_b200 import runner
+
+    # every rank verifies its own batch of the same shape (seed offset by rank)
+    import dataclasses
+    rcfg = dataclasses.replace(cfg, seed=cfg.seed + rank)
+    inp = gen.make_inputs(rcfg)
+    pas = runner.VerifyPass(rcfg, inp)
+    pas.prepare_host(inp)
+    stream = torch.cuda.current_stream()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        pas.run()
+    sync_all()
+    assert int(pas.status.item()) == 0, "a device-side wait timed out"
+
+    # ---- device-resident timing: K passes, CUDA events on the launching stream
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    n0 = ts.launch_count()
+    sync_all()
+    for s, e in ev:
+        s.record(stream)
+        pas.run()
+        e.record(stream)
+    sync_all()
+    launches = ts.launch_count() - n0
+    total_ms = sum(s.elapsed_time(e) for s, e in ev)
+
+    # ---- per-entry-point breakdown (same K passes, events between the entry points)
+    names = ["tree_mask", "attention", "lmhead", "scan"]
+    calls = [lambda: ts.trispec_build_tree_mask(pas.tree_args), lambda: ts.trispec_verify_attn(pas.attn_args),
+             lambda: ts.trispec_lmhead_stats(pas.lm_args), lambda: ts.trispec_accept_scan(pas.scan_args)]
+    acc = [0.0] * 4
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+    for _ in range(args.steps):
+        evs[0].record(stream)
+        for i, c in enumerate(calls):
+            c()
+            evs[i + 1].record(stream)
+        torch.cuda.synchronize()
+        for i in range(4):
+            acc[i] += evs[i].elapsed_time(evs[i + 1])
+    part_ms = {n: a / args.steps for n, a in zip(names, acc)}
+
+    # ---- end to end through the host-buffer entry point: H2D inputs + pass + D2H results per step
+    for _ in range(3):
+        pas.run_host()
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        pas.run_host()
+        torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    clocks = sampler.stop() if rank == 0 else None
+
+    t = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    tokens = cfg_tokens(cfg) * world
+    ms_per_step = total_ms / args.steps
+    value = tokens / (ms_per_step * 1e-3)
+    peaks = _peaks()
+    n_seq = cfg.B if cfg.n_active is None else cfg.n_active
+    M = n_seq * cfg.T
+    lm_flops = 2.0 * M * cfg.d * cfg.V
+    lm_tflops = lm_flops / (part_ms["lmhead"] * 1e-3) / 1e12
+    Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
+    attn_bytes = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 2 * 2 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
+    attn_gbs = attn_bytes / (part_ms["attention"] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "active_sequences": n_seq, "draft_tokens": cfg.k,
+                   "tree_nodes": cfg.T, "context": cfg.L, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "head_dim": cfg.D,
+                   "hidden": cfg.d, "vocab": cfg.V, "kv": "paged" if cfg.paged else "contiguous",
+                   "l2": "inputs larger than L2 (LM-head weights + KV cache are streamed every pass)",
+                   "parallelism": "independent replicas, one batch per GPU"},
+        "e2e": {"value": tokens / (e2e_ms * 1e-3 / args.steps), "unit": UNIT,
+                "h2d_bytes_per_step": pas.h2d_bytes, "d2h_bytes_per_step": pas.d2h_bytes},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "roofline": {"kernel": "lmhead_gemm_kernel", "bound": "tensor", "achieved": lm_tflops,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": lm_tflops / peaks["bf16_tflops"],
+                     "peak_source": f"{peaks['source']} burst bf16", "traffic": LMHEAD_GEMM_DRAM_TRAFFIC.get(cfg.name),
+                     "flops_per_launch": lm_flops, "ms_per_launch": part_ms["lmhead"]},
+        "kernels_ms": part_ms,
+        "attention_roofline": {"bound": "hbm", "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": attn_gbs / peaks["hbm_gbs"], "bytes_per_launch": attn_bytes},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        v, desc, threads = oracle_timed(cfg, inp, budget_s=20.0)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -176,6 +176,27 @@ int trispec_accept_scan(const trispec_scan_args* a, void* stream);
 int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                    const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * The same pass for callers whose per-round data lives in HOST memory (one verification
+ * round of Algorithm 1 as a decode loop sees it: the draft tree and its activations arrive
+ * from the host, the routing decision goes back to it). The KV cache and the LM-head weights
+ * stay resident on the device. In order, on `stream`: copies the per-round inputs from the
+ * host pointers of `io` into the device buffers named by the argument structs
+ * (tree->parent, lm->tok, attn->q, attn->k_tree, attn->v_tree, lm->h), runs trispec_verify,
+ * then copies accept_len, escalate, bonus_tok, last_node and path back to the host pointers.
+ * Host pointers should be page-locked for the copies to be asynchronous; the results are
+ * valid once `stream` has been synchronised. NULL host input pointers skip that copy.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  const int32_t *parent, *tok;              /* host [B][T] */
+  const void *q, *k_tree, *v_tree, *h;      /* host bf16, same layouts as the device tensors */
+  int32_t *accept_len, *bonus_tok, *last_node, *path;  /* host outputs [B], [B], [B], [B][T] */
+  uint8_t* escalate;                         /* host output [B] */
+} trispec_host_io;
+int trispec_verify_host(const trispec_host_io* io, const trispec_tree_args* tree,
+                        const trispec_attn_args* attn, const trispec_lmhead_args* lm,
+                        const trispec_scan_args* scan, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -60,6 +60,11 @@ class ScanArgs(C.Structure):
                 ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
 
 
+class HostIO(C.Structure):
+    _fields_ = [(n, _vp) for n in ("parent", "tok", "q", "k_tree", "v_tree", "h", "accept_len", "bonus_tok",
+                                   "last_node", "path", "escalate")]
+
+
 _lib.trispec_status_string.restype = C.c_char_p
 _lib.trispec_status_string.argtypes = [_i]
 _lib.trispec_launch_count.restype = C.c_longlong
@@ -74,7 +79,10 @@ _lib.trispec_accept_scan.argtypes = [C.POINTER(ScanArgs), _vp]
 _lib.trispec_verify.argtypes = [C.POINTER(TreeArgs), C.POINTER(AttnArgs), C.POINTER(LmheadArgs),
                                 C.POINTER(ScanArgs), _vp]
 
-EXPORTS = ["trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
+_lib.trispec_verify_host.argtypes = [C.POINTER(HostIO), C.POINTER(TreeArgs), C.POINTER(AttnArgs),
+                                     C.POINTER(LmheadArgs), C.POINTER(ScanArgs), _vp]
+
+EXPORTS = ["trispec_verify_host", "trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
            "trispec_verify_attn_workspace", "trispec_verify_attn", "trispec_lmhead_stats_workspace",
            "trispec_lmhead_stats", "trispec_accept_scan", "trispec_verify"]
 
@@ -229,3 +237,18 @@ def trispec_accept_scan(args: ScanArgs, stream=None):
 def trispec_verify(tree: TreeArgs, attn: Optional[AttnArgs], lm: LmheadArgs, scan: ScanArgs, stream=None):
     _check(_lib.trispec_verify(C.byref(tree), None if attn is None else C.byref(attn), C.byref(lm),
                                C.byref(scan), _stream(stream)))
+
+
+def host_io(**host_tensors) -> HostIO:
+    """HostIO from (pinned) CPU tensors; names as in the C struct, missing ones stay NULL."""
+    io = HostIO()
+    for name, _ in HostIO._fields_:
+        t = host_tensors.get(name)
+        setattr(io, name, None if t is None else _p(t))
+    return io
+
+
+def trispec_verify_host(io: HostIO, tree: TreeArgs, attn: Optional[AttnArgs], lm: LmheadArgs, scan: ScanArgs,
+                        stream=None):
+    _check(_lib.trispec_verify_host(C.byref(io), C.byref(tree), None if attn is None else C.byref(attn),
+                                    C.byref(lm), C.byref(scan), _stream(stream)))
