@@ -184,8 +184,8 @@ def cfg_tokens(cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="proxy_tree")
     ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

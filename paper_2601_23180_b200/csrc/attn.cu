@@ -87,17 +87,21 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   uint8_t* sP = sKV + AT_STAGES * AT_KV_STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + AT_P_BYTES);
   uint64_t* q_bar = bars;            // 1
-  uint64_t* full_bar = bars + 1;     // [2]
-  uint64_t* empty_bar = bars + 3;    // [2]
-  uint64_t* s_bar = bars + 5;        // [2]
-  uint64_t* o_bar = bars + 7;        // 1
-  uint64_t* p_bar = bars + 8;        // 1, 128 arrivals
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+  uint64_t* k_full = bars + 1;       // [2]  K tile landed
+  uint64_t* k_empty = bars + 3;      // [2]  S = Q K^T has consumed it
+  uint64_t* v_full = bars + 5;       // [2]  V tile landed
+  uint64_t* v_empty = bars + 7;      // [2]  O += P V has consumed it
+  uint64_t* s_bar = bars + 9;        // [2]  S buffer ready in TMEM
+  uint64_t* o_bar = bars + 11;       // 1    O += P V complete (P buffer free, O stable)
+  uint64_t* p_bar = bars + 12;       // 1    P written by the 128 softmax threads
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     mbar_init(q_bar, 1);
-    for (int i = 0; i < AT_STAGES; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
+    for (int i = 0; i < AT_STAGES; ++i) {
+      mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
+    }
     mbar_init(s_bar, 1); mbar_init(s_bar + 1, 1); mbar_init(o_bar, 1); mbar_init(p_bar, 128);
     fence_mbar_init();
   }
@@ -111,97 +115,106 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 4) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kt); prefetch_tmap(&tm_vt);
-      const int rows = p.NPT * p.G;
-      mbar_expect_tx(q_bar, static_cast<uint32_t>(rows) * AT_D * 2);
-      tma_load_4d(sQ, &tm_q, q_bar, 0, g * p.G, mtile * p.NPT, b);
-      tma_load_4d(sQ + AT_BM * 128, &tm_q, q_bar, 64, g * p.G, mtile * p.NPT, b);
-    }
-    int stage = 0;
-    uint32_t phase = 0;
-    int blk_cache = 0;
-    for (int i = 0; i < n_tiles; ++i) {
-      const bool tree = has_tree && (i == n_tiles - 1);
-      const int t = t_begin + i;
-      int blk = 0;
-      if (p.paged && !tree) {
-        // block ids are fetched 32 at a time by the whole warp
-        if ((i & 31) == 0) {
-          const int tt = t + lane;
-          int v = 0;
-          if (tt < t_end) v = __ldg(p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq + tt);
-          if (v < 0 || v >= p.num_blocks) {
-            if (tt < t_end && p.dev_status) atomicExch(p.dev_status, 6);   // bad block id: clamped
-            v = 0;
-          }
-          blk_cache = v;
-        }
-        blk = __shfl_sync(0xffffffffu, blk_cache, i & 31);
+    // ------------------------------------------------------------------ TMA producers
+    // lane 0 streams K (and loads Q once), lane 1 streams V; the two rings are independent:
+    // a K slot is free as soon as S = Q K^T has read it, a V slot only after O += P V.
+    if (lane < 2) {
+      const bool is_v = (lane == 1);
+      if (!is_v) {
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_kt);
+        const int rows = p.NPT * p.G;
+        mbar_expect_tx(q_bar, static_cast<uint32_t>(rows) * AT_D * 2);
+        tma_load_4d(sQ, &tm_q, q_bar, 0, g * p.G, mtile * p.NPT, b);
+        tma_load_4d(sQ + AT_BM * 128, &tm_q, q_bar, 64, g * p.G, mtile * p.NPT, b);
+      } else {
+        prefetch_tmap(&tm_v); prefetch_tmap(&tm_vt);
       }
-      if (lane == 0) {
-        mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
-        uint8_t* sk = sKV + stage * AT_KV_STAGE_BYTES;
-        uint8_t* sv = sk + 2 * AT_BOX_BYTES;
-        mbar_expect_tx(full_bar + stage, AT_KV_STAGE_BYTES);
+      const CUtensorMap* tm_ctx = is_v ? &tm_v : &tm_k;
+      const CUtensorMap* tm_tree = is_v ? &tm_vt : &tm_kt;
+      uint64_t* full = is_v ? v_full : k_full;
+      uint64_t* empty = is_v ? v_empty : k_empty;
+      const int32_t* table = p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq;
+      auto block_id = [&](int t) -> int {
+        int v = __ldg(table + t);
+        if (v < 0 || v >= p.num_blocks) {
+          if (p.dev_status) atomicExch(p.dev_status, 6);   // bad block id: clamped, flagged
+          v = 0;
+        }
+        return v;
+      };
+      int blk_next = (p.paged && t_begin < t_end) ? block_id(t_begin) : 0;
+      for (int i = 0; i < n_tiles; ++i) {
+        const bool tree = has_tree && (i == n_tiles - 1);
+        const int t = t_begin + i;
+        const int stage = i & 1;
+        const int blk = blk_next;
+        if (p.paged && t + 1 < t_end) blk_next = block_id(t + 1);   // fetched one tile ahead
+        mbar_wait(empty + stage, ((i >> 1) & 1u) ^ 1u, p.dev_status);
+        uint8_t* dst = sKV + stage * AT_KV_STAGE_BYTES + (is_v ? 2 * AT_BOX_BYTES : 0);
+        mbar_expect_tx(full + stage, 2 * AT_BOX_BYTES);
         if (tree) {
-          tma_load_4d(sk, &tm_kt, full_bar + stage, 0, g, 0, b);
-          tma_load_4d(sk + AT_BOX_BYTES, &tm_kt, full_bar + stage, 64, g, 0, b);
-          tma_load_4d(sv, &tm_vt, full_bar + stage, 0, g, 0, b);
-          tma_load_4d(sv + AT_BOX_BYTES, &tm_vt, full_bar + stage, 64, g, 0, b);
+          tma_load_4d(dst, tm_tree, full + stage, 0, g, 0, b);
+          tma_load_4d(dst + AT_BOX_BYTES, tm_tree, full + stage, 64, g, 0, b);
         } else {
           const int c2 = p.paged ? 0 : t * AT_BN;
           const int c3 = p.paged ? blk : b;
-          tma_load_4d(sk, &tm_k, full_bar + stage, 0, g, c2, c3);
-          tma_load_4d(sk + AT_BOX_BYTES, &tm_k, full_bar + stage, 64, g, c2, c3);
-          tma_load_4d(sv, &tm_v, full_bar + stage, 0, g, c2, c3);
-          tma_load_4d(sv + AT_BOX_BYTES, &tm_v, full_bar + stage, 64, g, c2, c3);
+          tma_load_4d(dst, tm_ctx, full + stage, 0, g, c2, c3);
+          tma_load_4d(dst + AT_BOX_BYTES, tm_ctx, full + stage, 64, g, c2, c3);
         }
       }
-      if (++stage == AT_STAGES) { stage = 0; phase ^= 1u; }
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
+    // Polls for whichever of "S of the next tile" / "P V of the oldest pending tile" can go,
+    // so that neither waits behind the other's data.
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(AT_BM, AT_BN, false, false);
       const uint32_t idesc_o = idesc_bf16(AT_BM, AT_D, false, true);
       const uint32_t sQ_u = base_u32, sKV_u = base_u32 + AT_Q_BYTES, sP_u = sKV_u + AT_STAGES * AT_KV_STAGE_BYTES;
-      auto issue_pv = [&](int i) {
-        const int stage = i & 1;
-        const uint32_t sv = sKV_u + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
-#pragma unroll
-        for (int kk = 0; kk < AT_BN / 16; ++kk) {
-          const uint64_t ad = smem_desc_sw128(sP_u + kk * 32, 1024, 16);
-          // V: MN-major, 64-dim blocks 8 KB apart (LBO), 8-key groups 1 KB apart (SBO)
-          const uint64_t bd = smem_desc_sw128(sv + kk * 2048, 1024, AT_BOX_BYTES);
-          tc_mma_ss(tmem_base + 128, ad, bd, idesc_o, (i | kk) != 0);
-        }
-        tc_commit(empty_bar + stage);
-        tc_commit(o_bar);
-      };
       mbar_wait(q_bar, 0, p.dev_status);
-      for (int i = 0; i < n_tiles; ++i) {
-        const int stage = i & 1, buf = i & 1;
-        mbar_wait(full_bar + stage, (i >> 1) & 1u, p.dev_status);
-        tc_fence_after();
-        const uint32_t sk = sKV_u + stage * AT_KV_STAGE_BYTES;
-#pragma unroll
-        for (int kk = 0; kk < AT_D / 16; ++kk) {
-          const uint64_t ad = smem_desc_sw128(sQ_u + (kk >> 2) * (AT_BM * 128) + (kk & 3) * 32, 1024, 16);
-          const uint64_t bd = smem_desc_sw128(sk + (kk >> 2) * AT_BOX_BYTES + (kk & 3) * 32, 1024, 16);
-          tc_mma_ss(tmem_base + buf * AT_BN, ad, bd, idesc_s, kk != 0);
-        }
-        tc_commit(s_bar + buf);
-        if (i > 0) {
-          mbar_wait(p_bar, (i - 1) & 1u, p.dev_status);   // P(i-1) is in shared memory
+      int next_s = 0, next_pv = 0;
+      uint32_t idle = 0;
+      while (next_pv < n_tiles) {
+        bool progressed = false;
+        // S(next_s): its TMEM buffer is free once P(next_s - 2) has been written
+        if (next_s < n_tiles && next_s < next_pv + 2 && mbar_test(k_full + (next_s & 1), (next_s >> 1) & 1u)) {
+          const int stage = next_s & 1, buf = next_s & 1;
           tc_fence_after();
-          issue_pv(i - 1);
+          const uint32_t sk = sKV_u + stage * AT_KV_STAGE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < AT_D / 16; ++kk) {
+            const uint64_t ad = smem_desc_sw128(sQ_u + (kk >> 2) * (AT_BM * 128) + (kk & 3) * 32, 1024, 16);
+            const uint64_t bd = smem_desc_sw128(sk + (kk >> 2) * AT_BOX_BYTES + (kk & 3) * 32, 1024, 16);
+            tc_mma_ss(tmem_base + buf * AT_BN, ad, bd, idesc_s, kk != 0);
+          }
+          tc_commit(s_bar + buf);
+          tc_commit(k_empty + stage);
+          ++next_s;
+          progressed = true;
+        }
+        if (next_pv < next_s && mbar_test(p_bar, next_pv & 1u) && mbar_test(v_full + (next_pv & 1), (next_pv >> 1) & 1u)) {
+          const int stage = next_pv & 1;
+          tc_fence_after();
+          const uint32_t sv = sKV_u + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < AT_BN / 16; ++kk) {
+            const uint64_t ad = smem_desc_sw128(sP_u + kk * 32, 1024, 16);
+            // V: MN-major, 64-dim blocks 8 KB apart (LBO), 8-key groups 1 KB apart (SBO)
+            const uint64_t bd = smem_desc_sw128(sv + kk * 2048, 1024, AT_BOX_BYTES);
+            tc_mma_ss(tmem_base + 128, ad, bd, idesc_o, (next_pv | kk) != 0);
+          }
+          tc_commit(v_empty + stage);
+          tc_commit(o_bar);
+          ++next_pv;
+          progressed = true;
+        }
+        if (progressed) {
+          idle = 0;
+        } else if (++idle > kWaitPolls) {   // bounded: give up, flag, and let the kernel end
+          if (p.dev_status) atomicExch(p.dev_status, 5);
+          break;
         }
       }
-      mbar_wait(p_bar, (n_tiles - 1) & 1u, p.dev_status);
-      tc_fence_after();
-      issue_pv(n_tiles - 1);
     }
   } else {
     // ------------------------------------------------------------------ softmax (warps 0-3)
@@ -282,6 +295,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       l += lsum;
       if (nvalid < AT_BN) {
         // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
+        mbar_wait(v_full + stage, (i >> 1) & 1u, p.dev_status);
         uint8_t* sv = sKV + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
         for (int e = threadIdx.x; e < (AT_BN - nvalid) * 16; e += 128) {
           const int r = nvalid + (e >> 4), c16 = e & 15;

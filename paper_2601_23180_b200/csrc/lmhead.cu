@@ -224,7 +224,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
 }
 
 // ---------------------------------------------------------------------------------------
-// Merge of the per-range partials + drafted-token logits. One block per active sequence.
+// Merge of the per-range partials + drafted-token logits.
 // ---------------------------------------------------------------------------------------
 struct LmFinalizeParams {
   int T, d, V, n_mt, n_ranges;
@@ -236,42 +236,68 @@ struct LmFinalizeParams {
   trispec_stats out;
 };
 
-constexpr int LM_FIN_THREADS = 256;
+constexpr int LM_FIN_THREADS = 256;   // 8 warps = 8 rows per block
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
+// larger value first, lower index on ties; index -1 marks "no entry"
+__device__ __forceinline__ bool lm_better(float va, int ia, float vb, int ib) {
+  return ia >= 0 && (ib < 0 || va > vb || (va == vb && ia < ib));
+}
+__device__ __forceinline__ void lm_top2_insert(float v, int i, float& v1, int& i1, float& v2, int& i2) {
+  if (i < 0) return;
+  if (lm_better(v, i, v1, i1)) { v2 = v1; i2 = i1; v1 = v; i1 = i; }
+  else if (lm_better(v, i, v2, i2)) { v2 = v; i2 = i; }
+}
+
+// log-sum-exp of one row from its per-range partials, computed by a whole warp
+__device__ __forceinline__ void lm_row_lse(const LmPartial* part, size_t stride, size_t prow, int n_ranges, float c,
+                                           int lane, float& M, float& S) {
+  float m = -INFINITY;
+  for (int r = lane; r < n_ranges; r += 32) m = fmaxf(m, part[r * stride + prow].m);
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float sacc = 0.f;
+  for (int r = lane; r < n_ranges; r += 32) {
+    const LmPartial q = part[r * stride + prow];
+    sacc += q.s * ex2f((q.m - m) * c);
+  }
+  for (int o = 16; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
+  M = m; S = sacc;
+}
+
+// One warp per (active sequence, node): merges the row's partial statistics and, for a child
+// node, computes the logit of its drafted token in its parent's row (a d-long dot product).
 __global__ void __launch_bounds__(LM_FIN_THREADS)
-lmhead_finalize_kernel(const LmFinalizeParams p) {
-  __shared__ float lse_s[64];
-  const int a = blockIdx.x;
-  const int seq = p.seq_index ? __ldg(p.seq_index + a) : a;
+lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
+  const int lane = threadIdx.x & 31;
+  const long long w = static_cast<long long>(blockIdx.x) * (LM_FIN_THREADS / 32) + (threadIdx.x >> 5);
   const int T = p.T;
+  if (w >= static_cast<long long>(n_seq) * T) return;
+  const int a = static_cast<int>(w / T), node = static_cast<int>(w % T);
+  const int seq = p.seq_index ? __ldg(p.seq_index + a) : a;
   const long long row0 = static_cast<long long>(seq) * T;
-  const int tid = threadIdx.x;
-  if (tid < T) {
-    const size_t prow = static_cast<size_t>(a) * 64 + tid;
-    const size_t stride = static_cast<size_t>(p.n_mt) * LM_BM;
-    float M = -INFINITY;
-    for (int r = 0; r < p.n_ranges; ++r) M = fmaxf(M, p.partial[r * stride + prow].m);
-    float S = 0.f, v1 = -INFINITY, v2 = -INFINITY;
-    int i1 = -1, i2 = -1;
-    // larger value first, lower index on ties
-    auto better = [](float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia >= 0 && (ib < 0 || ia < ib)); };
-    for (int r = 0; r < p.n_ranges; ++r) {
-      const LmPartial q = p.partial[r * stride + prow];
-      S += q.s * ex2f((q.m - M) * p.c);
-      const float cv[2] = {q.v1, q.v2};
-      const int ci[2] = {q.i1, q.i2};
-#pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        if (ci[k] < 0) continue;
-        if (better(cv[k], ci[k], v1, i1)) { v2 = v1; i2 = i1; v1 = cv[k]; i1 = ci[k]; }
-        else if (better(cv[k], ci[k], v2, i2)) { v2 = cv[k]; i2 = ci[k]; }
-      }
-    }
-    const float lse = M * p.scale + logf(S);
-    const long long o = row0 + tid;
+  const size_t stride = static_cast<size_t>(p.n_mt) * LM_BM;
+  const size_t prow = static_cast<size_t>(a) * 64 + node;
+
+  float M, S;
+  lm_row_lse(p.partial, stride, prow, p.n_ranges, p.c, lane, M, S);
+  float v1 = -INFINITY, v2 = -INFINITY;
+  int i1 = -1, i2 = -1;
+  for (int r = lane; r < p.n_ranges; r += 32) {
+    const LmPartial q = p.partial[r * stride + prow];
+    lm_top2_insert(q.v1, q.i1, v1, i1, v2, i2);
+    lm_top2_insert(q.v2, q.i2, v1, i1, v2, i2);
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov1 = __shfl_xor_sync(0xffffffffu, v1, o), ov2 = __shfl_xor_sync(0xffffffffu, v2, o);
+    const int oi1 = __shfl_xor_sync(0xffffffffu, i1, o), oi2 = __shfl_xor_sync(0xffffffffu, i2, o);
+    lm_top2_insert(ov1, oi1, v1, i1, v2, i2);
+    lm_top2_insert(ov2, oi2, v1, i1, v2, i2);
+  }
+  const float lse = M * p.scale + logf(S);
+  const long long o = row0 + node;
+  if (lane == 0) {
     p.out.max[o] = M * p.scale;
     p.out.lse[o] = lse;
     p.out.top1_val[o] = v1 * p.scale;
@@ -280,20 +306,15 @@ lmhead_finalize_kernel(const LmFinalizeParams p) {
     p.out.top2_idx[o] = i2;
     p.out.p_top1[o] = expf(v1 * p.scale - lse);
     p.out.p_top2[o] = expf(v2 * p.scale - lse);
-    lse_s[tid] = lse;
-    if (tid == 0) {
-      p.out.draft_logit[o] = __int_as_float(0x7fc00000);
-      p.out.p_draft[o] = __int_as_float(0x7fc00000);
-    }
   }
-  __syncthreads();
-  // drafted-token logit z[parent(c)][tok[c]]: one warp per child, 16-byte loads
-  const int warp = tid >> 5, lane = tid & 31;
-  for (int cnode = 1 + warp; cnode < T; cnode += LM_FIN_THREADS / 32) {
-    const int par = __ldg(p.parent + row0 + cnode);
-    const int tk = __ldg(p.tok + row0 + cnode);
-    float dl = __int_as_float(0x7fc00000), pd = dl;
-    if (par >= 0 && par < cnode && tk >= 0 && tk < p.V) {
+  // drafted-token logit z[parent(node)][tok[node]]
+  float dl = __int_as_float(0x7fc00000), pd = dl;
+  if (node >= 1) {
+    const int par = __ldg(p.parent + row0 + node);
+    const int tk = __ldg(p.tok + row0 + node);
+    if (par >= 0 && par < node && tk >= 0 && tk < p.V) {
+      float Mp, Sp;
+      lm_row_lse(p.partial, stride, static_cast<size_t>(a) * 64 + par, p.n_ranges, p.c, lane, Mp, Sp);
       const uint4* hv = reinterpret_cast<const uint4*>(p.h + (row0 + par) * p.d);
       const uint4* wv = reinterpret_cast<const uint4*>(p.W + static_cast<long long>(tk) * p.d);
       float acc = 0.f;
@@ -304,14 +325,14 @@ lmhead_finalize_kernel(const LmFinalizeParams p) {
         acc = fmaf(bf16_lo(x.z), bf16_lo(y.z), acc); acc = fmaf(bf16_hi(x.z), bf16_hi(y.z), acc);
         acc = fmaf(bf16_lo(x.w), bf16_lo(y.w), acc); acc = fmaf(bf16_hi(x.w), bf16_hi(y.w), acc);
       }
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      for (int o2 = 16; o2 > 0; o2 >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o2);
       dl = acc * p.scale;
-      pd = expf(dl - lse_s[par]);
+      pd = expf(dl - (Mp * p.scale + logf(Sp)));
     }
-    if (lane == 0) {
-      p.out.draft_logit[row0 + cnode] = dl;
-      p.out.p_draft[row0 + cnode] = pd;
-    }
+  }
+  if (lane == 0) {
+    p.out.draft_logit[o] = dl;
+    p.out.p_draft[o] = pd;
   }
 }
 
@@ -394,7 +415,7 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   f.W = static_cast<const uint16_t*>(a->W);
   f.parent = a->parent; f.tok = a->tok;
   f.out = a->out;
-  lmhead_finalize_kernel<<<n_seq, LM_FIN_THREADS, 0, st>>>(f);
+  lmhead_finalize_kernel<<<(n_seq * a->T + 7) / 8, LM_FIN_THREADS, 0, st>>>(f, n_seq);
   count_launch();
   TRISPEC_CUDA_OK(cudaGetLastError());
   return TRISPEC_OK;
