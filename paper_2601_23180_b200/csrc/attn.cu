@@ -105,7 +105,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     mbar_init(s_bar, 1); mbar_init(s_bar + 1, 1); mbar_init(o_bar, 1); mbar_init(p_bar, 128);
     fence_mbar_init();
   }
-  if (warp == 4) {
+  if (warp == 5) {
     tmem_alloc(tmem_slot, AT_TMEM_COLS);
     tmem_relinquish();
   }
@@ -115,26 +115,20 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 4) {
-    // ------------------------------------------------------------------ TMA producers
-    // lane 0 streams K (and loads Q once), lane 1 streams V; the two rings are independent:
-    // a K slot is free as soon as S = Q K^T has read it, a V slot only after O += P V.
-    if (lane < 2) {
-      const bool is_v = (lane == 1);
-      if (!is_v) {
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_kt);
+    // ------------------------------------------------------------------ TMA loader
+    // One thread streams K and V with non-blocking tests of the two rings: a K slot is free
+    // as soon as S = Q K^T has read it, a V slot only after O += P V.
+    if (lane == 0) {
+      prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_kt); prefetch_tmap(&tm_v); prefetch_tmap(&tm_vt);
+      {
         const int rows = p.NPT * p.G;
         mbar_expect_tx(q_bar, static_cast<uint32_t>(rows) * AT_D * 2);
         tma_load_4d(sQ, &tm_q, q_bar, 0, g * p.G, mtile * p.NPT, b);
         tma_load_4d(sQ + AT_BM * 128, &tm_q, q_bar, 64, g * p.G, mtile * p.NPT, b);
-      } else {
-        prefetch_tmap(&tm_v); prefetch_tmap(&tm_vt);
       }
-      const CUtensorMap* tm_ctx = is_v ? &tm_v : &tm_k;
-      const CUtensorMap* tm_tree = is_v ? &tm_vt : &tm_kt;
-      uint64_t* full = is_v ? v_full : k_full;
-      uint64_t* empty = is_v ? v_empty : k_empty;
       const int32_t* table = p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq;
-      auto block_id = [&](int t) -> int {
+      auto block_id = [&](int t) -> int {      // fetched two tiles before it is used
+        if (!p.paged || t >= t_end) return 0;
         int v = __ldg(table + t);
         if (v < 0 || v >= p.num_blocks) {
           if (p.dev_status) atomicExch(p.dev_status, 6);   // bad block id: clamped, flagged
@@ -142,31 +136,57 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
         return v;
       };
-      int blk_next = (p.paged && t_begin < t_end) ? block_id(t_begin) : 0;
-      for (int i = 0; i < n_tiles; ++i) {
+      auto load_tile = [&](int i, bool is_v, int blk) {
         const bool tree = has_tree && (i == n_tiles - 1);
-        const int t = t_begin + i;
         const int stage = i & 1;
-        const int blk = blk_next;
-        if (p.paged && t + 1 < t_end) blk_next = block_id(t + 1);   // fetched one tile ahead
-        mbar_wait(empty + stage, ((i >> 1) & 1u) ^ 1u, p.dev_status);
+        uint64_t* full = (is_v ? v_full : k_full) + stage;
         uint8_t* dst = sKV + stage * AT_KV_STAGE_BYTES + (is_v ? 2 * AT_BOX_BYTES : 0);
-        mbar_expect_tx(full + stage, 2 * AT_BOX_BYTES);
+        mbar_expect_tx(full, 2 * AT_BOX_BYTES);
         if (tree) {
-          tma_load_4d(dst, tm_tree, full + stage, 0, g, 0, b);
-          tma_load_4d(dst + AT_BOX_BYTES, tm_tree, full + stage, 64, g, 0, b);
+          const CUtensorMap* tm = is_v ? &tm_vt : &tm_kt;
+          tma_load_4d(dst, tm, full, 0, g, 0, b);
+          tma_load_4d(dst + AT_BOX_BYTES, tm, full, 64, g, 0, b);
         } else {
-          const int c2 = p.paged ? 0 : t * AT_BN;
+          const CUtensorMap* tm = is_v ? &tm_v : &tm_k;
+          const int c2 = p.paged ? 0 : (t_begin + i) * AT_BN;
           const int c3 = p.paged ? blk : b;
-          tma_load_4d(dst, tm_ctx, full + stage, 0, g, c2, c3);
-          tma_load_4d(dst + AT_BOX_BYTES, tm_ctx, full + stage, 64, g, c2, c3);
+          tma_load_4d(dst, tm, full, 0, g, c2, c3);
+          tma_load_4d(dst + AT_BOX_BYTES, tm, full, 64, g, c2, c3);
+        }
+      };
+      int kblk0 = block_id(t_begin), kblk1 = block_id(t_begin + 1);
+      int vblk0 = kblk0, vblk1 = kblk1;
+      int next_k = 0, next_v = 0;
+      uint32_t idle = 0;
+      while (next_v < n_tiles) {
+        bool progressed = false;
+        if (next_k < n_tiles && mbar_test(k_empty + (next_k & 1), ((next_k >> 1) & 1u) ^ 1u)) {
+          load_tile(next_k, false, kblk0);
+          kblk0 = kblk1;
+          kblk1 = block_id(t_begin + next_k + 2);
+          ++next_k;
+          progressed = true;
+        }
+        if (mbar_test(v_empty + (next_v & 1), ((next_v >> 1) & 1u) ^ 1u)) {
+          load_tile(next_v, true, vblk0);
+          vblk0 = vblk1;
+          vblk1 = block_id(t_begin + next_v + 2);
+          ++next_v;
+          progressed = true;
+        }
+        if (progressed) {
+          idle = 0;
+        } else if (++idle > kWaitPolls) {   // bounded: give up, flag, and let the kernel end
+          if (p.dev_status) atomicExch(p.dev_status, 5);
+          break;
         }
       }
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
-    // Polls for whichever of "S of the next tile" / "P V of the oldest pending tile" can go,
-    // so that neither waits behind the other's data.
+    // Polls for whichever of "S of the next tile" (its TMEM buffer is free once P(i-2)
+    // exists) and "P V of the oldest pending tile" (P written, V landed) can go, so that
+    // neither waits behind the other's data.
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(AT_BM, AT_BN, false, false);
       const uint32_t idesc_o = idesc_bf16(AT_BM, AT_D, false, true);
@@ -176,7 +196,6 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       uint32_t idle = 0;
       while (next_pv < n_tiles) {
         bool progressed = false;
-        // S(next_s): its TMEM buffer is free once P(next_s - 2) has been written
         if (next_s < n_tiles && next_s < next_pv + 2 && mbar_test(k_full + (next_s & 1), (next_s >> 1) & 1u)) {
           const int stage = next_s & 1, buf = next_s & 1;
           tc_fence_after();
@@ -192,7 +211,8 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
           ++next_s;
           progressed = true;
         }
-        if (next_pv < next_s && mbar_test(p_bar, next_pv & 1u) && mbar_test(v_full + (next_pv & 1), (next_pv >> 1) & 1u)) {
+        if (next_pv < next_s && mbar_test(p_bar, next_pv & 1u) &&
+            mbar_test(v_full + (next_pv & 1), (next_pv >> 1) & 1u)) {
           const int stage = next_pv & 1;
           tc_fence_after();
           const uint32_t sv = sKV_u + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
@@ -331,7 +351,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 5) {
     tc_fence_after();
     tmem_dealloc(tmem_base, AT_TMEM_COLS);
   }
