@@ -7,13 +7,18 @@
 // row = node_local * G + head_in_group, so one K/V tile serves all of them. An M tile holds
 // NPT = min(128 / G, 64) nodes.
 //
-// Per 64-key tile:  S = Q K^T  (tcgen05.mma M=128, N=64, K=128, both operands K-major)
+// Per 64-key tile:  S = Q K^T  (tcgen05.mma M=128, N=64, K=128; Q is the A operand and lives
+//                   in tensor memory for the whole kernel, K is the K-major B operand)
 //                   online softmax in registers, one TMEM lane (row) per thread, exp2 domain,
 //                   lazy rescaling of O (only when the running max grows by more than 2^8)
 //                   P (bf16) -> shared memory, O += P V (V is the MN-major B operand)
-// S is double-buffered in TMEM so that S(t+1) is computed while the softmax of tile t runs.
-// K/V tiles arrive by TMA (no multicast) through a 2-stage mbarrier ring; two CTAs fit on one
-// SM (shared memory ~111 KB, 256 TMEM columns each) and overlap each other's phases.
+// The kernel is bound by shared-memory bandwidth before anything else (TMA writes, operand
+// reads of the MMAs, P), which is why Q is kept out of shared memory: per tile the MMAs read
+// K, P and V only.
+// Warps 0-3: softmax. Warp 4: one thread streams K and V by TMA (no multicast) through two
+// independent 3-slot rings (a K slot is free once S has read it, a V slot after O += P V).
+// Warp 5: one thread issues the MMAs, polling for whichever of S(i+1) / P V(i) can go.
+// Two CTAs fit on one SM (~112 KB shared memory, 256 TMEM columns each).
 #include <math.h>
 
 #include "host_common.h"
@@ -24,16 +29,16 @@ namespace trispec {
 constexpr int AT_BM = 128;      // rows per M tile
 constexpr int AT_BN = 64;       // keys per tile (= paged block size)
 constexpr int AT_D = 128;
-constexpr int AT_STAGES = 2;
+constexpr int AT_STAGES = 3;
 constexpr int AT_BOX_BYTES = 64 * 64 * 2;               // 64 rows x 64 elements
-constexpr int AT_Q_BYTES = AT_BM * AT_D * 2;            // 32 KB (2 boxes of 128 rows x 64)
 constexpr int AT_KV_STAGE_BYTES = 4 * AT_BOX_BYTES;     // K (2 boxes) + V (2 boxes) = 32 KB
 constexpr int AT_P_BYTES = AT_BM * AT_BN * 2;           // 16 KB
 constexpr int AT_THREADS = 192;
-constexpr int AT_SMEM_USED = AT_Q_BYTES + AT_STAGES * AT_KV_STAGE_BYTES + AT_P_BYTES + 128;
-// two CTAs per SM: 2 x (dynamic + 1 KB reserved) must fit 228 KB, which leaves 896 bytes of alignment slack
-constexpr int AT_SMEM_BYTES = AT_SMEM_USED + 896;
-constexpr int AT_TMEM_COLS = 256;                        // S0 [0,64) S1 [64,128) O [128,256)
+constexpr int AT_SMEM_USED = AT_STAGES * AT_KV_STAGE_BYTES + AT_P_BYTES + 256;
+// two CTAs per SM: 2 x (dynamic + 1 KB reserved) must fit 228 KB, which leaves 768 bytes of alignment slack
+constexpr int AT_SMEM_BYTES = AT_SMEM_USED + 768;
+constexpr int AT_TMEM_COLS = 256;                        // Q [0,64) S [64,128) O [128,256)
+constexpr int AT_TM_Q = 0, AT_TM_S = 64, AT_TM_O = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
@@ -42,6 +47,7 @@ struct AttnParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split;
   int paged, max_blocks_per_seq, num_blocks;
   float scale_log2;
+  const uint16_t* q;
   const int32_t *block_table, *ctx_len, *seq_index;
   const uint64_t* mask;
   float* part_o;    // [items][128][128]
@@ -56,9 +62,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 __global__ void __launch_bounds__(AT_THREADS, 2)
-verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                         const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kt,
-                         const __grid_constant__ CUtensorMap tm_vt, const AttnParams p) {
+verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                         const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt,
+                         const AttnParams p) {
   // ---- which work item
   int idx = blockIdx.x;
   const int mtile = idx % p.n_mt; idx /= p.n_mt;
@@ -82,27 +88,26 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 7);   // shared memory window misaligned
     return;
   }
-  uint8_t* sQ = smem;
-  uint8_t* sKV = smem + AT_Q_BYTES;
+  uint8_t* sKV = smem;
   uint8_t* sP = sKV + AT_STAGES * AT_KV_STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + AT_P_BYTES);
-  uint64_t* q_bar = bars;            // 1
-  uint64_t* k_full = bars + 1;       // [2]  K tile landed
-  uint64_t* k_empty = bars + 3;      // [2]  S = Q K^T has consumed it
-  uint64_t* v_full = bars + 5;       // [2]  V tile landed
-  uint64_t* v_empty = bars + 7;      // [2]  O += P V has consumed it
-  uint64_t* s_bar = bars + 9;        // [2]  S buffer ready in TMEM
-  uint64_t* o_bar = bars + 11;       // 1    O += P V complete (P buffer free, O stable)
-  uint64_t* p_bar = bars + 12;       // 1    P written by the 128 softmax threads
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  uint64_t* k_full = bars;                      // [3]  K tile landed
+  uint64_t* k_empty = bars + AT_STAGES;         // [3]  S = Q K^T has consumed it
+  uint64_t* v_full = bars + 2 * AT_STAGES;      // [3]  V tile landed
+  uint64_t* v_empty = bars + 3 * AT_STAGES;     // [3]  O += P V has consumed it
+  uint64_t* s_bar = bars + 4 * AT_STAGES;       // S ready in TMEM
+  uint64_t* s_free = s_bar + 1;                 // S read into registers by the 128 softmax threads
+  uint64_t* o_bar = s_bar + 2;                  // O += P V complete (P buffer free, O stable)
+  uint64_t* p_bar = s_bar + 3;                  // P written by the 128 softmax threads
+  uint64_t* q_bar = s_bar + 4;                  // Q stored to TMEM by the 128 softmax threads
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_bar + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(q_bar, 1);
     for (int i = 0; i < AT_STAGES; ++i) {
       mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
     }
-    mbar_init(s_bar, 1); mbar_init(s_bar + 1, 1); mbar_init(o_bar, 1); mbar_init(p_bar, 128);
+    mbar_init(s_bar, 1); mbar_init(s_free, 128); mbar_init(o_bar, 1); mbar_init(p_bar, 128); mbar_init(q_bar, 128);
     fence_mbar_init();
   }
   if (warp == 5) {
@@ -116,16 +121,8 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA loader
-    // One thread streams K and V with non-blocking tests of the two rings: a K slot is free
-    // as soon as S = Q K^T has read it, a V slot only after O += P V.
     if (lane == 0) {
-      prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_kt); prefetch_tmap(&tm_v); prefetch_tmap(&tm_vt);
-      {
-        const int rows = p.NPT * p.G;
-        mbar_expect_tx(q_bar, static_cast<uint32_t>(rows) * AT_D * 2);
-        tma_load_4d(sQ, &tm_q, q_bar, 0, g * p.G, mtile * p.NPT, b);
-        tma_load_4d(sQ + AT_BM * 128, &tm_q, q_bar, 64, g * p.G, mtile * p.NPT, b);
-      }
+      prefetch_tmap(&tm_k); prefetch_tmap(&tm_kt); prefetch_tmap(&tm_v); prefetch_tmap(&tm_vt);
       const int32_t* table = p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq;
       auto block_id = [&](int t) -> int {      // fetched two tiles before it is used
         if (!p.paged || t >= t_end) return 0;
@@ -138,7 +135,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       };
       auto load_tile = [&](int i, bool is_v, int blk) {
         const bool tree = has_tree && (i == n_tiles - 1);
-        const int stage = i & 1;
+        const int stage = i % AT_STAGES;
         uint64_t* full = (is_v ? v_full : k_full) + stage;
         uint8_t* dst = sKV + stage * AT_KV_STAGE_BYTES + (is_v ? 2 * AT_BOX_BYTES : 0);
         mbar_expect_tx(full, 2 * AT_BOX_BYTES);
@@ -160,14 +157,14 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       uint32_t idle = 0;
       while (next_v < n_tiles) {
         bool progressed = false;
-        if (next_k < n_tiles && mbar_test(k_empty + (next_k & 1), ((next_k >> 1) & 1u) ^ 1u)) {
+        if (next_k < n_tiles && mbar_test(k_empty + next_k % AT_STAGES, ((next_k / AT_STAGES) & 1u) ^ 1u)) {
           load_tile(next_k, false, kblk0);
           kblk0 = kblk1;
           kblk1 = block_id(t_begin + next_k + 2);
           ++next_k;
           progressed = true;
         }
-        if (mbar_test(v_empty + (next_v & 1), ((next_v >> 1) & 1u) ^ 1u)) {
+        if (mbar_test(v_empty + next_v % AT_STAGES, ((next_v / AT_STAGES) & 1u) ^ 1u)) {
           load_tile(next_v, true, vblk0);
           vblk0 = vblk1;
           vblk1 = block_id(t_begin + next_v + 2);
@@ -176,44 +173,47 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
         if (progressed) {
           idle = 0;
-        } else if (++idle > kWaitPolls) {   // bounded: give up, flag, and let the kernel end
-          if (p.dev_status) atomicExch(p.dev_status, 5);
-          break;
+        } else {
+          __nanosleep(32);                    // leave the issue slots to the softmax warps
+          if (++idle > kWaitPolls) {          // bounded: give up, flag, and let the kernel end
+            if (p.dev_status) atomicExch(p.dev_status, 5);
+            break;
+          }
         }
       }
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
-    // Polls for whichever of "S of the next tile" (its TMEM buffer is free once P(i-2)
-    // exists) and "P V of the oldest pending tile" (P written, V landed) can go, so that
-    // neither waits behind the other's data.
+    // S(i) may be issued once the softmax threads have read S(i-1) out of TMEM and K(i) has
+    // landed; P V(i) once P(i) is in shared memory and V(i) has landed.
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(AT_BM, AT_BN, false, false);
       const uint32_t idesc_o = idesc_bf16(AT_BM, AT_D, false, true);
-      const uint32_t sQ_u = base_u32, sKV_u = base_u32 + AT_Q_BYTES, sP_u = sKV_u + AT_STAGES * AT_KV_STAGE_BYTES;
+      const uint32_t sKV_u = base_u32, sP_u = sKV_u + AT_STAGES * AT_KV_STAGE_BYTES;
       mbar_wait(q_bar, 0, p.dev_status);
+      tc_fence_after();
       int next_s = 0, next_pv = 0;
       uint32_t idle = 0;
       while (next_pv < n_tiles) {
         bool progressed = false;
-        if (next_s < n_tiles && next_s < next_pv + 2 && mbar_test(k_full + (next_s & 1), (next_s >> 1) & 1u)) {
-          const int stage = next_s & 1, buf = next_s & 1;
+        if (next_s < n_tiles && (next_s == 0 || mbar_test(s_free, (next_s - 1) & 1u)) &&
+            mbar_test(k_full + next_s % AT_STAGES, (next_s / AT_STAGES) & 1u)) {
+          const int stage = next_s % AT_STAGES;
           tc_fence_after();
           const uint32_t sk = sKV_u + stage * AT_KV_STAGE_BYTES;
 #pragma unroll
           for (int kk = 0; kk < AT_D / 16; ++kk) {
-            const uint64_t ad = smem_desc_sw128(sQ_u + (kk >> 2) * (AT_BM * 128) + (kk & 3) * 32, 1024, 16);
             const uint64_t bd = smem_desc_sw128(sk + (kk >> 2) * AT_BOX_BYTES + (kk & 3) * 32, 1024, 16);
-            tc_mma_ss(tmem_base + buf * AT_BN, ad, bd, idesc_s, kk != 0);
+            tc_mma_ts(tmem_base + AT_TM_S, tmem_base + AT_TM_Q + kk * 8, bd, idesc_s, kk != 0);
           }
-          tc_commit(s_bar + buf);
+          tc_commit(s_bar);
           tc_commit(k_empty + stage);
           ++next_s;
           progressed = true;
         }
         if (next_pv < next_s && mbar_test(p_bar, next_pv & 1u) &&
-            mbar_test(v_full + (next_pv & 1), (next_pv >> 1) & 1u)) {
-          const int stage = next_pv & 1;
+            mbar_test(v_full + next_pv % AT_STAGES, (next_pv / AT_STAGES) & 1u)) {
+          const int stage = next_pv % AT_STAGES;
           tc_fence_after();
           const uint32_t sv = sKV_u + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
 #pragma unroll
@@ -221,7 +221,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const uint64_t ad = smem_desc_sw128(sP_u + kk * 32, 1024, 16);
             // V: MN-major, 64-dim blocks 8 KB apart (LBO), 8-key groups 1 KB apart (SBO)
             const uint64_t bd = smem_desc_sw128(sv + kk * 2048, 1024, AT_BOX_BYTES);
-            tc_mma_ss(tmem_base + 128, ad, bd, idesc_o, (next_pv | kk) != 0);
+            tc_mma_ss(tmem_base + AT_TM_O, ad, bd, idesc_o, (next_pv | kk) != 0);
           }
           tc_commit(v_empty + stage);
           tc_commit(o_bar);
@@ -230,9 +230,12 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
         if (progressed) {
           idle = 0;
-        } else if (++idle > kWaitPolls) {   // bounded: give up, flag, and let the kernel end
-          if (p.dev_status) atomicExch(p.dev_status, 5);
-          break;
+        } else {
+          __nanosleep(32);                    // leave the issue slots to the softmax warps
+          if (++idle > kWaitPolls) {          // bounded: give up, flag, and let the kernel end
+            if (p.dev_status) atomicExch(p.dev_status, 5);
+            break;
+          }
         }
       }
     }
@@ -243,22 +246,44 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const bool row_valid = (row < p.NPT * p.G) && (node < p.T);
     const uint64_t mrow = row_valid ? __ldg(p.mask + static_cast<long long>(b) * p.T + node) : 0ull;
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    // Q row -> TMEM (A operand of S = Q K^T): lane = row, column c = dims (2c, 2c + 1)
+    {
+      const int hq = g * p.G + row % p.G;
+      const uint4* src = reinterpret_cast<const uint4*>(
+          p.q + ((static_cast<long long>(b) * p.T + (row_valid ? node : 0)) * p.Hq + hq) * AT_D);
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (row_valid) v = __ldg(src + c * 8 + j);
+          r[4 * j] = v.x; r[4 * j + 1] = v.y; r[4 * j + 2] = v.z; r[4 * j + 3] = v.w;
+        }
+        tmem_st32(tmem_base + lane_base + AT_TM_Q + c * 32, r);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(q_bar);
+    }
     float m_ref = -INFINITY, l = 0.f;
 
     for (int i = 0; i < n_tiles; ++i) {
-      const int stage = i & 1, buf = i & 1;
+      const int stage = i % AT_STAGES;
       const bool tree = has_tree && (i == n_tiles - 1);
-      mbar_wait(s_bar + buf, (i >> 1) & 1u, p.dev_status);
+      mbar_wait(s_bar, i & 1u, p.dev_status);
       tc_fence_after();
       uint32_t sr[64];
       {
         uint32_t r0[32], r1[32];
-        tmem_ld32(tmem_base + lane_base + buf * AT_BN, r0);
-        tmem_ld32(tmem_base + lane_base + buf * AT_BN + 32, r1);
+        tmem_ld32(tmem_base + lane_base + AT_TM_S, r0);
+        tmem_ld32(tmem_base + lane_base + AT_TM_S + 32, r1);
         tc_wait_ld();
 #pragma unroll
         for (int j = 0; j < 32; ++j) { sr[j] = r0[j]; sr[32 + j] = r1[j]; }
       }
+      tc_fence_before();
+      mbar_arrive(s_free);                       // S(i + 1) may overwrite the buffer now
       // which keys of this tile does this row see
       uint64_t vis;
       int nvalid = AT_BN;
@@ -290,11 +315,11 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t o[32];
-            tmem_ld32(tmem_base + lane_base + 128 + c * 32, o);
+            tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
             tc_wait_ld();
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * f);
-            tmem_st32(tmem_base + lane_base + 128 + c * 32, o);
+            tmem_st32(tmem_base + lane_base + AT_TM_O + c * 32, o);
           }
           tc_wait_st();
         }
@@ -315,7 +340,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       l += lsum;
       if (nvalid < AT_BN) {
         // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
-        mbar_wait(v_full + stage, (i >> 1) & 1u, p.dev_status);
+        mbar_wait(v_full + stage, (i / AT_STAGES) & 1u, p.dev_status);
         uint8_t* sv = sKV + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
         for (int e = threadIdx.x; e < (AT_BN - nvalid) * 16; e += 128) {
           const int r = nvalid + (e >> 4), c16 = e & 15;
@@ -334,7 +359,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       uint32_t o[32];
-      tmem_ld32(tmem_base + lane_base + 128 + c * 32, o);
+      tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
       tc_wait_ld();
       if (row_valid) {
 #pragma unroll
@@ -474,20 +499,14 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   if (a->workspace_bytes < trispec_verify_attn_workspace(a)) return TRISPEC_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-  const uint64_t D = AT_D, Hq = a->Hq, Hkv = a->Hkv, T = a->T, B = a->B;
-  CUtensorMap tm_q, tm_k, tm_v, tm_kt, tm_vt;
-  {
-    const uint64_t dims[4] = {D, Hq, T, B};
-    const uint64_t str[3] = {D * 2, Hq * D * 2, T * Hq * D * 2};
-    const uint32_t box[4] = {64, static_cast<uint32_t>(pl.G), static_cast<uint32_t>(pl.NPT), 1};
-    if (!encode_tmap_bf16(&tm_q, a->q, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
-  }
+  const uint64_t D = AT_D, Hkv = a->Hkv, T = a->T, B = a->B;
+  CUtensorMap tm_k, tm_v, tm_kt, tm_vt;
   {
     const uint64_t dims[4] = {D, Hkv, T, B};
     const uint64_t str[3] = {D * 2, Hkv * D * 2, T * Hkv * D * 2};
     const uint32_t box[4] = {64, 1, 64, 1};
-    if (!encode_tmap_bf16(&tm_kt, a->k_tree, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
-    if (!encode_tmap_bf16(&tm_vt, a->v_tree, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+    if (!cached_tmap_bf16(&tm_kt, a->k_tree, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+    if (!cached_tmap_bf16(&tm_vt, a->v_tree, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
   }
   if (pl.tiles_max > 0) {
     uint64_t dims[4], str[3];
@@ -499,26 +518,28 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
       str[0] = D * 2; str[1] = Hkv * D * 2; str[2] = static_cast<uint64_t>(AT_BN) * Hkv * D * 2;
     }
     const uint32_t box[4] = {64, 1, 64, 1};
-    if (!encode_tmap_bf16(&tm_k, a->k_cache, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
-    if (!encode_tmap_bf16(&tm_v, a->v_cache, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+    if (!cached_tmap_bf16(&tm_k, a->k_cache, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
+    if (!cached_tmap_bf16(&tm_v, a->v_cache, 4, dims, str, box)) return TRISPEC_ERR_CUDA;
   } else {
     tm_k = tm_kt;   // never dereferenced: every sequence has zero context tiles
     tm_v = tm_vt;
   }
-  TRISPEC_CUDA_OK(cudaFuncSetAttribute(verify_attn_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       AT_SMEM_BYTES));
+  static bool smem_set[64] = {};
+  rc = ensure_smem_limit(reinterpret_cast<const void*>(verify_attn_split_kernel), AT_SMEM_BYTES, smem_set);
+  if (rc != TRISPEC_OK) return rc;
   AttnParams p;
   p.T = a->T; p.Hq = a->Hq; p.Hkv = a->Hkv; p.G = pl.G; p.NPT = pl.NPT; p.n_mt = pl.n_mt;
   p.n_splits = pl.n_splits; p.tiles_per_split = pl.tiles_per_split;
   p.paged = (a->kv_layout == TRISPEC_KV_PAGED); p.max_blocks_per_seq = a->max_blocks_per_seq;
   p.num_blocks = a->num_blocks;
   p.scale_log2 = a->scale * kLog2e;
+  p.q = static_cast<const uint16_t*>(a->q);
   p.block_table = a->block_table; p.ctx_len = a->ctx_len; p.seq_index = a->seq_index; p.mask = a->mask;
   p.part_o = static_cast<float*>(a->workspace);
   p.part_ml = p.part_o + pl.items * AT_BM * AT_D;
   p.dev_status = a->dev_status;
-  verify_attn_split_kernel<<<static_cast<unsigned>(pl.items), AT_THREADS, AT_SMEM_BYTES, st>>>(tm_q, tm_k, tm_v, tm_kt,
-                                                                                                tm_vt, p);
+  verify_attn_split_kernel<<<static_cast<unsigned>(pl.items), AT_THREADS, AT_SMEM_BYTES, st>>>(tm_k, tm_v, tm_kt, tm_vt,
+                                                                                                p);
   count_launch();
   TRISPEC_CUDA_OK(cudaGetLastError());
 

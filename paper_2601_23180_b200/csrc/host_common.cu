@@ -1,3 +1,5 @@
+#include <string.h>
+
 #include <atomic>
 #include <mutex>
 
@@ -41,6 +43,56 @@ bool encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+namespace {
+struct TmapKey {
+  const void* base;
+  int rank;
+  uint64_t dims[4], strides[3];
+  uint32_t box[4];
+  int device;
+};
+struct TmapEntry {
+  TmapKey key;
+  CUtensorMap map;
+  bool valid;
+};
+constexpr int kTmapCache = 32;
+}  // namespace
+
+bool cached_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                      const uint64_t* strides_bytes, const uint32_t* box) {
+  thread_local TmapEntry cache[kTmapCache] = {};
+  thread_local int next = 0;
+  TmapKey k;
+  memset(&k, 0, sizeof(k));
+  k.base = base;
+  k.rank = rank;
+  for (int i = 0; i < rank; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) k.strides[i] = strides_bytes[i];
+  if (cudaGetDevice(&k.device) != cudaSuccess) return false;
+  for (int i = 0; i < kTmapCache; ++i)
+    if (cache[i].valid && memcmp(&cache[i].key, &k, sizeof(k)) == 0) {
+      *out = cache[i].map;
+      return true;
+    }
+  if (!encode_tmap_bf16(out, base, rank, dims, strides_bytes, box)) return false;
+  cache[next].key = k;
+  cache[next].map = *out;
+  cache[next].valid = true;
+  next = (next + 1) % kTmapCache;
+  return true;
+}
+
+int ensure_smem_limit(const void* func, int bytes, bool* done_per_device) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRISPEC_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && done_per_device[dev]) return TRISPEC_OK;
+  if (cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+    return TRISPEC_ERR_CUDA;
+  if (dev >= 0 && dev < 64) done_per_device[dev] = true;
+  return TRISPEC_OK;
 }
 
 int device_sm_count() {

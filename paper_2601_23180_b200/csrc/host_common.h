@@ -18,7 +18,15 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 bool encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
                       const uint64_t* strides_bytes, const uint32_t* box);
 
+// Same, through a small per-thread cache keyed by (base, rank, dims, strides, box): repeated
+// calls with the same buffers (the steady state of a decode loop) skip the driver call.
+bool cached_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims,
+                      const uint64_t* strides_bytes, const uint32_t* box);
+
 int device_sm_count();
+
+// Raises the dynamic shared memory limit of `func` once per device.
+int ensure_smem_limit(const void* func, int bytes, bool* done_per_device /* [64] */);
 
 #define TRISPEC_CUDA_OK(expr)                        \
   do {                                               \

@@ -381,20 +381,17 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
     const uint64_t dims[3] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->T), static_cast<uint64_t>(a->B)};
     const uint64_t strides[2] = {static_cast<uint64_t>(a->d) * 2, static_cast<uint64_t>(a->d) * 2 * a->T};
     const uint32_t box[3] = {LM_BK, 64, 1};
-    if (!encode_tmap_bf16(&tm_h, a->h, 3, dims, strides, box)) return TRISPEC_ERR_CUDA;
+    if (!cached_tmap_bf16(&tm_h, a->h, 3, dims, strides, box)) return TRISPEC_ERR_CUDA;
   }
   {
     const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
     const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
     const uint32_t box[2] = {LM_BK, 64};
-    if (!encode_tmap_bf16(&tm_w, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+    if (!cached_tmap_bf16(&tm_w, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    TRISPEC_CUDA_OK(cudaFuncSetAttribute(lmhead_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         LM_SMEM_BYTES));
-    attr_set = true;
-  }
+  static bool smem_set[64] = {};
+  rc = ensure_smem_limit(reinterpret_cast<const void*>(lmhead_gemm_kernel), LM_SMEM_BYTES, smem_set);
+  if (rc != TRISPEC_OK) return rc;
   LmParams p;
   p.T = a->T; p.d = a->d; p.V = a->V;
   p.n_seq = n_seq; p.n_mt = n_mt; p.n_ranges = n_ranges;
