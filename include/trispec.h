@@ -85,7 +85,10 @@ int trispec_build_tree_mask(const trispec_tree_args* a, void* stream);
  *      NULL = all B (then B_active is ignored).
  *    lse (optional) f32 [B][Hq][T]: log-sum-exp of the scaled scores.
  *    workspace: device scratch of at least trispec_verify_attn_workspace(a) bytes,
- *      256-byte aligned; contents are undefined before and after the call.
+ *      256-byte aligned; contents are undefined before and after the call. The query
+ *      returns 0 (and workspace may be NULL) whenever the context is cut into at most 8
+ *      key/value splits per sequence, which are then merged on chip; only few sequences
+ *      with long contexts need more splits and a workspace.
  *    Pointers of bf16 tensors must be 16-byte aligned.
  * ------------------------------------------------------------------------------------- */
 typedef struct {

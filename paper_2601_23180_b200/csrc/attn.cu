@@ -1,7 +1,12 @@
 // Verification attention (the attention of the parallel verification pass, Eq. 2 / Eq. 5):
 // every draft-tree node attends to the whole committed context plus the tree keys its mask
-// row allows. Split-KV: one CTA handles (sequence, KV head, M tile, KV split) and writes an
-// unnormalised partial (O, m, l); a second kernel merges the splits.
+// row allows. Split-KV: one CTA handles (sequence, KV head, M tile, KV split) and produces an
+// unnormalised partial (O, m, l). With up to 8 splits the CTAs of one (sequence, KV head,
+// M tile) form a thread-block cluster: each leaves its partial in its own shared memory and
+// the cluster merges them through distributed shared memory, every CTA normalising and
+// writing a slice of the rows - no scratch traffic and no second launch. With more splits
+// (few sequences, long contexts) partials go to a caller-provided workspace and a second
+// kernel merges them.
 //
 // GQA packing: the G = Hq / Hkv query heads that share a KV head are stacked on the M axis,
 // row = node_local * G + head_in_group, so one K/V tile serves all of them. An M tile holds
@@ -16,7 +21,8 @@
 // reads of the MMAs, P), which is why Q is kept out of shared memory: per tile the MMAs read
 // K, P and V only.
 // Warps 0-3: softmax. Warp 4: one thread streams K and V by TMA (no multicast) through two
-// independent 3-slot rings (a K slot is free once S has read it, a V slot after O += P V).
+// independent 3-slot rings (a K slot is free once S has read it, a V slot after O += P V); it
+// initialises the ring barriers itself and starts loading before the CTA-wide set-up barrier.
 // Warp 5: one thread issues the MMAs, polling for whichever of S(i+1) / P V(i) can go.
 // Two CTAs fit on one SM (~112 KB shared memory, 256 TMEM columns each).
 #include <math.h>
@@ -42,6 +48,9 @@ constexpr int AT_TM_Q = 0, AT_TM_S = 64, AT_TM_O = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
+constexpr int AT_PART_PITCH = AT_D + 4;                  // floats per row of the in-smem partial (bank spread)
+constexpr int AT_PART_ML_OFF = AT_BM * AT_PART_PITCH * 4; // (m, l) pairs follow the partial O rows
+static_assert(AT_PART_ML_OFF + AT_BM * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
 
 struct AttnParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split;
@@ -50,10 +59,33 @@ struct AttnParams {
   const uint16_t* q;
   const int32_t *block_table, *ctx_len, *seq_index;
   const uint64_t* mask;
-  float* part_o;    // [items][128][128]
+  float* part_o;    // [items][128][128]   (workspace mode only)
   float* part_ml;   // [items][128][2]
+  uint16_t* o;      // bf16 [B][T][Hq][128]  (cluster mode writes the result itself)
+  float* lse;       // [B][Hq][T] or null
   int32_t* dev_status;
 };
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local_saddr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_saddr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -61,33 +93,37 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+template <bool kCluster>
 __global__ void __launch_bounds__(AT_THREADS, 2)
 verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                          const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt,
                          const AttnParams p) {
-  // ---- which work item
+  // ---- which work item: the split index varies fastest, so that in cluster mode the CTAs of
+  // one cluster are the splits of one (sequence, KV head, M tile) and cluster rank == split
   int idx = blockIdx.x;
-  const int mtile = idx % p.n_mt; idx /= p.n_mt;
   const int split = idx % p.n_splits; idx /= p.n_splits;
+  const int mtile = idx % p.n_mt; idx /= p.n_mt;
   const int g = idx % p.Hkv;
   const int a = idx / p.Hkv;
   const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
   const int L = __ldg(p.ctx_len + b);
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
   const int last_split = max(0, (n_ctx_tiles + p.tiles_per_split - 1) / p.tiles_per_split - 1);
-  if (split > last_split) return;            // nothing to do: the merge kernel skips it too
   const int t_begin = split * p.tiles_per_split;
   const int t_end = min(n_ctx_tiles, t_begin + p.tiles_per_split);
   const bool has_tree = (split == last_split);
-  const int n_tiles = (t_end - t_begin) + (has_tree ? 1 : 0);   // >= 1
+  const int n_tiles = (t_end - t_begin) + (has_tree ? 1 : 0);   // >= 1 unless this split is empty
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
-  if (base_u32 - smem_u32(smem_raw) > static_cast<uint32_t>(AT_SMEM_BYTES - AT_SMEM_USED)) {
-    if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 7);   // shared memory window misaligned
-    return;
-  }
+  const bool misaligned = base_u32 - smem_u32(smem_raw) > static_cast<uint32_t>(AT_SMEM_BYTES - AT_SMEM_USED);
+  if (misaligned && threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 7);   // shared window misaligned
+  // a split past the end of this sequence's context has nothing to do; in cluster mode it
+  // still takes part in the merge (with weight zero), so it may not leave early
+  const bool idle_cta = (split > last_split) || misaligned;
+  if (!kCluster && idle_cta) return;           // the merge kernel skips it too
+
   uint8_t* sKV = smem;
   uint8_t* sP = sKV + AT_STAGES * AT_KV_STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + AT_P_BYTES);
@@ -103,21 +139,36 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_bar + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < AT_STAGES; ++i) {
-      mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
+  float* sPartO = reinterpret_cast<float*>(smem);                       // reuses the K/V ring at the end
+  float2* sPartML = reinterpret_cast<float2*>(smem + AT_PART_ML_OFF);
+  uint32_t tmem_base = 0;
+
+  if (!idle_cta) {   // uniform for the whole CTA
+  if (warp == 4) {
+    // the loader owns the ring barriers: it signals the set-up barrier without waiting on it
+    // and starts streaming while the other warps are still allocating TMEM and storing Q
+    if (lane == 0) {
+      for (int i = 0; i < AT_STAGES; ++i) {
+        mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
+      }
+      fence_mbar_init();
     }
-    mbar_init(s_bar, 1); mbar_init(s_free, 128); mbar_init(o_bar, 1); mbar_init(p_bar, 128); mbar_init(q_bar, 128);
-    fence_mbar_init();
+    __syncwarp();
+    asm volatile("bar.arrive 1, 192;" ::: "memory");
+  } else {
+    if (threadIdx.x == 0) {
+      mbar_init(s_bar, 1); mbar_init(s_free, 128); mbar_init(o_bar, 1); mbar_init(p_bar, 128); mbar_init(q_bar, 128);
+      fence_mbar_init();
+    }
+    if (warp == 5) {
+      tmem_alloc(tmem_slot, AT_TMEM_COLS);
+      tmem_relinquish();
+    }
+    tc_fence_before();
+    asm volatile("bar.sync 1, 192;" ::: "memory");
+    tc_fence_after();
+    tmem_base = *tmem_slot;
   }
-  if (warp == 5) {
-    tmem_alloc(tmem_slot, AT_TMEM_COLS);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA loader
@@ -293,14 +344,21 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         nvalid = min(AT_BN, L - (t_begin + i) * AT_BN);
         vis = (nvalid >= 64) ? ~0ull : ((1ull << nvalid) - 1ull);
       }
-      float tmax = -INFINITY;
+      // running maximum on the raw scores (the scale is positive, so it commutes with max);
+      // four chains for instruction-level parallelism
+      float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (!tree && nvalid >= AT_BN) {
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        float v = __uint_as_float(sr[j]) * p.scale_log2;
-        if (!((vis >> j) & 1ull)) v = -INFINITY;
-        sr[j] = __float_as_uint(v);
-        tmax = fmaxf(tmax, v);
+        for (int j = 0; j < 64; ++j) tm[j & 3] = fmaxf(tm[j & 3], __uint_as_float(sr[j]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          const float v = ((vis >> j) & 1ull) ? __uint_as_float(sr[j]) : -INFINITY;
+          sr[j] = __float_as_uint(v);
+          tm[j & 3] = fmaxf(tm[j & 3], v);
+        }
       }
+      const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
       if (i > 0) {
         mbar_wait(o_bar, (i - 1) & 1u, p.dev_status);   // P V of the previous tile is complete
         tc_fence_after();
@@ -324,20 +382,23 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
           tc_wait_st();
         }
       }
-      const float mu = (m_ref == -INFINITY) ? 0.f : m_ref;
-      float lsum = 0.f;
+      const float nmu = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
       uint8_t* prow = sP + row * 128;
 #pragma unroll
       for (int cch = 0; cch < 8; ++cch) {
         float e[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { e[j] = ex2f(__uint_as_float(sr[cch * 8 + j]) - mu); lsum += e[j]; }
+        for (int j = 0; j < 8; ++j) {
+          e[j] = ex2f(fmaf(__uint_as_float(sr[cch * 8 + j]), p.scale_log2, nmu));   // exp2(s * scale - m)
+          ls[j & 3] += e[j];
+        }
         uint4 pk;
         pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]);
         pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
         *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk;
       }
-      l += lsum;
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       if (nvalid < AT_BN) {
         // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
         mbar_wait(v_full + stage, (i / AT_STAGES) & 1u, p.dev_status);
@@ -354,24 +415,42 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     // ---------------------------------------------------------------- epilogue
     mbar_wait(o_bar, (n_tiles - 1) & 1u, p.dev_status);
     tc_fence_after();
-    const size_t item = static_cast<size_t>(blockIdx.x);
-    float* po = p.part_o + (item * AT_BM + row) * AT_D;
+    if (kCluster) {
+      // partial (O, m, l) -> this CTA's shared memory (the K/V ring is idle: every tile has been
+      // consumed by its MMAs); rows are padded to 132 floats so that float4 stores spread over banks
+      float* po = sPartO + row * AT_PART_PITCH;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      uint32_t o[32];
-      tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
-      tc_wait_ld();
-      if (row_valid) {
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
+        tc_wait_ld();
 #pragma unroll
         for (int j = 0; j < 32; j += 4)
           *reinterpret_cast<float4*>(po + c * 32 + j) =
               make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
                           __uint_as_float(o[j + 3]));
       }
-    }
-    if (row_valid) {
-      float2 ml = make_float2(m_ref, l);
-      *reinterpret_cast<float2*>(p.part_ml + (item * AT_BM + row) * 2) = ml;
+      sPartML[row] = make_float2(m_ref, l);
+    } else {
+      const size_t item = static_cast<size_t>(blockIdx.x);
+      float* po = p.part_o + (item * AT_BM + row) * AT_D;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
+        tc_wait_ld();
+        if (row_valid) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<float4*>(po + c * 32 + j) =
+                make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
+                            __uint_as_float(o[j + 3]));
+        }
+      }
+      if (row_valid) {
+        float2 ml = make_float2(m_ref, l);
+        *reinterpret_cast<float2*>(p.part_ml + (item * AT_BM + row) * 2) = ml;
+      }
     }
   }
   tc_fence_before();
@@ -379,6 +458,48 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   if (warp == 5) {
     tc_fence_after();
     tmem_dealloc(tmem_base, AT_TMEM_COLS);
+  }
+  }   // !idle_cta
+
+  if (kCluster) {
+    // ---------------------------------------------------------------- cluster merge
+    // Every CTA of the cluster holds one partial in its shared memory (idle CTAs: weight zero).
+    // CTA `split` normalises rows [split * 128 / n_splits, (split + 1) * 128 / n_splits).
+    if (idle_cta) {
+      for (int r = threadIdx.x; r < AT_BM; r += AT_THREADS) sPartML[r] = make_float2(-INFINITY, 0.f);
+    }
+    cluster_sync_all();
+    const int rows_per_cta = AT_BM / p.n_splits;
+    const uint32_t po_u = smem_u32(sPartO), pml_u = smem_u32(sPartML);
+    for (int rr = warp; rr < rows_per_cta; rr += AT_THREADS / 32) {
+      const int row = split * rows_per_cta + rr;
+      const int node = mtile * p.NPT + row / p.G;
+      if (row >= p.NPT * p.G || node >= p.T) continue;
+      float M = -INFINITY;
+      for (int s = 0; s < p.n_splits; ++s)
+        M = fmaxf(M, ld_cluster_f2(cluster_map(pml_u + row * 8, s)).x);
+      float Lsum = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < p.n_splits; ++s) {
+        const float2 ml = ld_cluster_f2(cluster_map(pml_u + row * 8, s));
+        if (ml.x == -INFINITY) continue;        // empty partial (its O rows hold nothing)
+        const float wgt = ex2f(ml.x - M);
+        Lsum += ml.y * wgt;
+        const float4 v = ld_cluster_f4(cluster_map(po_u + (row * AT_PART_PITCH + lane * 4) * 4, s));
+        acc.x = fmaf(v.x, wgt, acc.x); acc.y = fmaf(v.y, wgt, acc.y);
+        acc.z = fmaf(v.z, wgt, acc.z); acc.w = fmaf(v.w, wgt, acc.w);
+      }
+      const float inv = 1.f / Lsum;
+      const int hq = g * p.G + row % p.G;
+      uint2 out;
+      out.x = pack_bf16(acc.x * inv, acc.y * inv);
+      out.y = pack_bf16(acc.z * inv, acc.w * inv);
+      uint16_t* orow = p.o + ((static_cast<size_t>(b) * p.T + node) * p.Hq + hq) * AT_D;
+      *reinterpret_cast<uint2*>(orow + lane * 4) = out;
+      if (p.lse && lane == 0)
+        p.lse[(static_cast<size_t>(b) * p.Hq + hq) * p.T + node] = (M + log2f(Lsum)) * kLn2;
+    }
+    cluster_sync_all();   // nobody leaves while its shared memory may still be read
   }
 }
 
@@ -409,16 +530,16 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
   const int L = __ldg(p.ctx_len + b);
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
   const int n_valid = max(0, (n_ctx_tiles + p.tiles_per_split - 1) / p.tiles_per_split - 1) + 1;
-  const size_t item0 = ((static_cast<size_t>(a) * p.Hkv + g) * p.n_splits) * p.n_mt + mtile;
+  const size_t item0 = ((static_cast<size_t>(a) * p.Hkv + g) * p.n_mt + mtile) * p.n_splits;
   float M = -INFINITY;
   for (int s = 0; s < n_valid; ++s) {
-    const size_t item = item0 + static_cast<size_t>(s) * p.n_mt;
+    const size_t item = item0 + static_cast<size_t>(s);
     M = fmaxf(M, __ldg(p.part_ml + (item * AT_BM + row) * 2));
   }
   float Lsum = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int s = 0; s < n_valid; ++s) {
-    const size_t item = item0 + static_cast<size_t>(s) * p.n_mt;
+    const size_t item = item0 + static_cast<size_t>(s);
     const float2 ml = __ldg(reinterpret_cast<const float2*>(p.part_ml + (item * AT_BM + row) * 2));
     const float wgt = (ml.x == -INFINITY) ? 0.f : ex2f(ml.x - M);
     Lsum += ml.y * wgt;
@@ -437,6 +558,7 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
 
 struct AttnPlan {
   int n_seq, G, NPT, n_mt, tiles_max, tiles_per_split, n_splits;
+  bool cluster;      // splits merged inside a thread-block cluster (no workspace)
   size_t items;
 };
 
@@ -469,6 +591,14 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   if (c > pl->tiles_max) c = pl->tiles_max > 0 ? pl->tiles_max : 1;
   pl->tiles_per_split = static_cast<int>(c);
   pl->n_splits = pl->tiles_max > 0 ? (pl->tiles_max + pl->tiles_per_split - 1) / pl->tiles_per_split : 1;
+  pl->cluster = pl->n_splits <= 8;
+  if (pl->cluster) {
+    // cluster sizes 1, 2, 4, 8 (the portable limit); rows of the M tile divide evenly among them
+    int s = 1;
+    while (s < pl->n_splits) s <<= 1;
+    pl->n_splits = s;
+    pl->tiles_per_split = pl->tiles_max > 0 ? (pl->tiles_max + s - 1) / s : 1;
+  }
   pl->items = static_cast<size_t>(fixed) * pl->n_splits;
   if (pl->items > 0x7fffffffull) return TRISPEC_ERR_UNSUPPORTED;
   return TRISPEC_OK;
@@ -480,6 +610,7 @@ extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) {
   using namespace trispec;
   AttnPlan pl;
   if (attn_plan(a, &pl) != TRISPEC_OK) return 0;
+  if (pl.cluster) return 0;
   return pl.items * AT_BM * (AT_D + 2) * sizeof(float);
 }
 
@@ -488,8 +619,8 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   AttnPlan pl;
   int rc = attn_plan(a, &pl);
   if (rc != TRISPEC_OK) return rc;
-  if (!a->q || !a->k_tree || !a->v_tree || !a->ctx_len || !a->mask || !a->o || !a->workspace)
-    return TRISPEC_ERR_INVALID_ARG;
+  if (!a->q || !a->k_tree || !a->v_tree || !a->ctx_len || !a->mask || !a->o) return TRISPEC_ERR_INVALID_ARG;
+  if (!pl.cluster && !a->workspace) return TRISPEC_ERR_INVALID_ARG;
   if (pl.tiles_max > 0 && (!a->k_cache || !a->v_cache)) return TRISPEC_ERR_INVALID_ARG;
   if (a->kv_layout == TRISPEC_KV_PAGED && !a->block_table) return TRISPEC_ERR_INVALID_ARG;
   if (!aligned16(a->q) || !aligned16(a->k_tree) || !aligned16(a->v_tree) || !aligned16(a->k_cache) ||
@@ -524,8 +655,10 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
     tm_k = tm_kt;   // never dereferenced: every sequence has zero context tiles
     tm_v = tm_vt;
   }
-  static bool smem_set[64] = {};
-  rc = ensure_smem_limit(reinterpret_cast<const void*>(verify_attn_split_kernel), AT_SMEM_BYTES, smem_set);
+  static bool smem_set_c[64] = {}, smem_set_w[64] = {};
+  rc = pl.cluster
+           ? ensure_smem_limit(reinterpret_cast<const void*>(verify_attn_split_kernel<true>), AT_SMEM_BYTES, smem_set_c)
+           : ensure_smem_limit(reinterpret_cast<const void*>(verify_attn_split_kernel<false>), AT_SMEM_BYTES, smem_set_w);
   if (rc != TRISPEC_OK) return rc;
   AttnParams p;
   p.T = a->T; p.Hq = a->Hq; p.Hkv = a->Hkv; p.G = pl.G; p.NPT = pl.NPT; p.n_mt = pl.n_mt;
@@ -537,9 +670,28 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   p.block_table = a->block_table; p.ctx_len = a->ctx_len; p.seq_index = a->seq_index; p.mask = a->mask;
   p.part_o = static_cast<float*>(a->workspace);
   p.part_ml = p.part_o + pl.items * AT_BM * AT_D;
+  p.o = static_cast<uint16_t*>(a->o);
+  p.lse = a->lse;
   p.dev_status = a->dev_status;
-  verify_attn_split_kernel<<<static_cast<unsigned>(pl.items), AT_THREADS, AT_SMEM_BYTES, st>>>(tm_k, tm_v, tm_kt, tm_vt,
-                                                                                                p);
+  if (pl.cluster) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(pl.items), 1, 1);
+    cfg.blockDim = dim3(AT_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = AT_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(pl.n_splits);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    TRISPEC_CUDA_OK(cudaLaunchKernelEx(&cfg, verify_attn_split_kernel<true>, tm_k, tm_v, tm_kt, tm_vt, p));
+    count_launch();
+    return TRISPEC_OK;
+  }
+  verify_attn_split_kernel<false><<<static_cast<unsigned>(pl.items), AT_THREADS, AT_SMEM_BYTES, st>>>(tm_k, tm_v, tm_kt,
+                                                                                                       tm_vt, p);
   count_launch();
   TRISPEC_CUDA_OK(cudaGetLastError());
 

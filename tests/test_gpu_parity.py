@@ -165,6 +165,8 @@ ATTN_CASES = [
     ("long_paged", dict(B=5, L=2100, L_min=70), None),                         # paged, ragged
     ("long_paged", dict(B=4, L=300, L_min=1), [0, 1, 64, 65]),                 # empty / one-key contexts
     ("proxy_tree", dict(B=2, L=64, Hq=8, Hkv=8), [64, 0]),                     # G = 1 (MHA)
+    ("proxy_tree", dict(B=1, L=9300, Hq=4, Hkv=2), None),                      # > 8 KV splits: workspace merge
+    ("long_paged", dict(B=3, L=5000, L_min=5000, Hq=4, Hkv=2), [5000, 40, 2300]),  # 8-CTA clusters with idle splits
 ]
 
 
@@ -194,17 +196,25 @@ def test_attention_against_oracle(H, name, over, ctx):
 def test_attention_argument_errors(H):
     import torch
     from paper_2601_23180_b200 import binding as ts
-    cfg = gen.small_variant(gen.CONFIGS["tiny_chain"], L=64)
+    # one sequence with a long context is cut into more than 8 KV splits, which are merged
+    # through a caller-provided workspace
+    cfg = gen.small_variant(gen.CONFIGS["tiny_chain"], L=9300, Hq=2, Hkv=2)
     inp = gen.make_inputs(cfg, with_lm_head=False)
     dev = H.to_device(inp)
     mask_dev, _ = H.run_tree_mask(dev["parent"])
     o = torch.zeros((cfg.B, cfg.T, cfg.Hq, cfg.D), dtype=torch.bfloat16, device="cuda")
     a = ts.attn_args(dev["q"], dev["k_tree"], dev["v_tree"], mask_dev, dev["k_cache"], dev["v_cache"],
                      dev["ctx_len"], 0.1, o)
+    assert ts.trispec_verify_attn_workspace(a) > 0
     n0 = ts.launch_count()
     with pytest.raises(ts.TrispecError) as e:
         ts.trispec_verify_attn(a)                              # no workspace
     assert e.value.code == 1
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    a.workspace, a.workspace_bytes = ws.data_ptr(), 256
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_verify_attn(a)                              # workspace too small
+    assert e.value.code == 3 and ts.launch_count() == n0
     a.D = 64
     with pytest.raises(ts.TrispecError) as e:
         ts.trispec_verify_attn(a)                              # unsupported head dim
