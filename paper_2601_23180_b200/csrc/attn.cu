@@ -48,9 +48,10 @@ constexpr int AT_TM_Q = 0, AT_TM_S = 64, AT_TM_O = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
-constexpr int AT_PART_PITCH = AT_D + 4;                  // floats per row of the in-smem partial (bank spread)
-constexpr int AT_PART_ML_OFF = AT_BM * AT_PART_PITCH * 4; // (m, l) pairs follow the partial O rows
-static_assert(AT_PART_ML_OFF + AT_BM * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
+constexpr int AT_PART_PITCH = AT_D * 2 + 16;             // bytes per row of the in-smem partial (bf16, bank spread)
+constexpr int AT_PART_ML_OFF = AT_BM * AT_PART_PITCH;    // (m, l) pairs follow the partial rows
+constexpr int AT_PART_ML2_OFF = AT_PART_ML_OFF + AT_BM * 8;   // gathered (m, l) of every split for this CTA's rows
+static_assert(AT_PART_ML2_OFF + AT_BM * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
 
 struct AttnParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split;
@@ -75,15 +76,15 @@ __device__ __forceinline__ uint32_t cluster_map(uint32_t local_saddr, uint32_t c
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_saddr), "r"(cta_rank));
   return r;
 }
-__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+__device__ __forceinline__ uint4 ld_cluster_u4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
   float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
   return v;
 }
 
@@ -139,7 +140,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_bar + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float* sPartO = reinterpret_cast<float*>(smem);                       // reuses the K/V ring at the end
+  uint8_t* sPartO = smem;                                               // reuses the K/V ring at the end
   float2* sPartML = reinterpret_cast<float2*>(smem + AT_PART_ML_OFF);
   uint32_t tmem_base = 0;
 
@@ -416,19 +417,27 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     mbar_wait(o_bar, (n_tiles - 1) & 1u, p.dev_status);
     tc_fence_after();
     if (kCluster) {
-      // partial (O, m, l) -> this CTA's shared memory (the K/V ring is idle: every tile has been
-      // consumed by its MMAs); rows are padded to 132 floats so that float4 stores spread over banks
-      float* po = sPartO + row * AT_PART_PITCH;
+      // partial (O / l as bf16, m, l) -> this CTA's shared memory (the K/V ring is idle: every
+      // tile has been consumed by its MMAs). The exchange between the CTAs of a cluster goes
+      // over the SM-to-SM network, whose bandwidth is a small fraction of shared memory's, so the
+      // partial travels normalised and in the output precision; m and l stay fp32. Rows are
+      // padded by 16 bytes so that the 16-byte stores of a warp spread over the banks.
+      uint8_t* po = sPartO + row * AT_PART_PITCH;
+      const float invl = (l > 0.f) ? 1.f / l : 0.f;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t o[32];
         tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
         tc_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 32; j += 4)
-          *reinterpret_cast<float4*>(po + c * 32 + j) =
-              make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
-                          __uint_as_float(o[j + 3]));
+        for (int j = 0; j < 32; j += 8) {
+          uint4 pk;
+          pk.x = pack_bf16(__uint_as_float(o[j]) * invl, __uint_as_float(o[j + 1]) * invl);
+          pk.y = pack_bf16(__uint_as_float(o[j + 2]) * invl, __uint_as_float(o[j + 3]) * invl);
+          pk.z = pack_bf16(__uint_as_float(o[j + 4]) * invl, __uint_as_float(o[j + 5]) * invl);
+          pk.w = pack_bf16(__uint_as_float(o[j + 6]) * invl, __uint_as_float(o[j + 7]) * invl);
+          *reinterpret_cast<uint4*>(po + (c * 32 + j) * 2) = pk;
+        }
       }
       sPartML[row] = make_float2(m_ref, l);
     } else {
@@ -469,34 +478,65 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       for (int r = threadIdx.x; r < AT_BM; r += AT_THREADS) sPartML[r] = make_float2(-INFINITY, 0.f);
     }
     cluster_sync_all();
-    const int rows_per_cta = AT_BM / p.n_splits;
+    // Requests over the SM-to-SM network are expensive per instruction, whatever their size,
+    // so they are few and wide: one gather of the (m, l) pairs of all splits for this CTA's
+    // rows, then per pair of rows one 16-byte-per-lane load from every split.
+    const int rpc = AT_BM / p.n_splits;          // rows this CTA normalises: 16 .. 128, even
     const uint32_t po_u = smem_u32(sPartO), pml_u = smem_u32(sPartML);
-    for (int rr = warp; rr < rows_per_cta; rr += AT_THREADS / 32) {
-      const int row = split * rows_per_cta + rr;
+    float2* sML2 = reinterpret_cast<float2*>(smem + AT_PART_ML2_OFF);   // [n_splits][rpc]
+    if (threadIdx.x < AT_BM) {
+      const int s_src = threadIdx.x / rpc, r = threadIdx.x % rpc;
+      sML2[threadIdx.x] = ld_cluster_f2(cluster_map(pml_u + (split * rpc + r) * 8, s_src));
+    }
+    __syncthreads();
+    constexpr int kWarps = AT_THREADS / 32;
+    const int half = lane >> 4, chunk = lane & 15;
+    for (int pr = warp; pr < rpc / 2; pr += kWarps) {
+      const int rl = 2 * pr + half;               // row within this CTA's slice
+      const int row = split * rpc + rl;
       const int node = mtile * p.NPT + row / p.G;
-      if (row >= p.NPT * p.G || node >= p.T) continue;
+      const bool ok = (row < p.NPT * p.G) && (node < p.T);
+      uint4 v[8];
+      float2 ml[8];
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        v[s] = make_uint4(0u, 0u, 0u, 0u);
+        ml[s] = make_float2(-INFINITY, 0.f);
+        if (s < p.n_splits) {
+          ml[s] = sML2[s * rpc + rl];
+          if (ok && ml[s].x != -INFINITY)         // an empty partial's rows hold arbitrary bits
+            v[s] = ld_cluster_u4(cluster_map(po_u + row * AT_PART_PITCH + chunk * 16, s));
+        }
+      }
+      if (!ok) continue;
       float M = -INFINITY;
-      for (int s = 0; s < p.n_splits; ++s)
-        M = fmaxf(M, ld_cluster_f2(cluster_map(pml_u + row * 8, s)).x);
+#pragma unroll
+      for (int s = 0; s < 8; ++s) M = fmaxf(M, ml[s].x);
       float Lsum = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int s = 0; s < p.n_splits; ++s) {
-        const float2 ml = ld_cluster_f2(cluster_map(pml_u + row * 8, s));
-        if (ml.x == -INFINITY) continue;        // empty partial (its O rows hold nothing)
-        const float wgt = ex2f(ml.x - M);
-        Lsum += ml.y * wgt;
-        const float4 v = ld_cluster_f4(cluster_map(po_u + (row * AT_PART_PITCH + lane * 4) * 4, s));
-        acc.x = fmaf(v.x, wgt, acc.x); acc.y = fmaf(v.y, wgt, acc.y);
-        acc.z = fmaf(v.z, wgt, acc.z); acc.w = fmaf(v.w, wgt, acc.w);
+      float acc[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const float wgt = (ml[s].x != -INFINITY) ? ex2f(ml[s].x - M) * ml[s].y : 0.f;
+        Lsum += wgt;
+        const uint32_t w[4] = {v[s].x, v[s].y, v[s].z, v[s].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[2 * j] = fmaf(__uint_as_float(w[j] << 16), wgt, acc[2 * j]);
+          acc[2 * j + 1] = fmaf(__uint_as_float(w[j] & 0xffff0000u), wgt, acc[2 * j + 1]);
+        }
       }
       const float inv = 1.f / Lsum;
       const int hq = g * p.G + row % p.G;
-      uint2 out;
-      out.x = pack_bf16(acc.x * inv, acc.y * inv);
-      out.y = pack_bf16(acc.z * inv, acc.w * inv);
+      uint4 out;
+      out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+      out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+      out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+      out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
       uint16_t* orow = p.o + ((static_cast<size_t>(b) * p.T + node) * p.Hq + hq) * AT_D;
-      *reinterpret_cast<uint2*>(orow + lane * 4) = out;
-      if (p.lse && lane == 0)
+      *reinterpret_cast<uint4*>(orow + chunk * 8) = out;
+      if (p.lse && chunk == 0)
         p.lse[(static_cast<size_t>(b) * p.Hq + hq) * p.T + node] = (M + log2f(Lsum)) * kLn2;
     }
     cluster_sync_all();   // nobody leaves while its shared memory may still be read
