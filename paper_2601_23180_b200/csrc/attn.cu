@@ -67,15 +67,6 @@ struct AttnParams {
   int32_t* dev_status;
 };
 
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t cluster_map(uint32_t local_saddr, uint32_t cta_rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_saddr), "r"(cta_rank));
-  return r;
-}
 __device__ __forceinline__ uint4 ld_cluster_u4(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];"

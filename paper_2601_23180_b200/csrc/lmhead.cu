@@ -6,17 +6,25 @@
 // tiles. A small second kernel merges the per-slice partials and computes the drafted-token
 // probabilities.
 //
-// GEMM kernel layout
-//   M tile  = 128 rows = 2 sequence slots x 64 node slots (T <= 64; missing nodes are
-//             zero-filled by the TMA out-of-bounds rule, missing sequences are not loaded)
-//   N tile  = up to 256 vocabulary entries (one tcgen05.mma N), a multiple of 16
+// GEMM kernel layout (two CTAs on two SMs work as a pair on one 256 x 256 tile)
+//   M tile  = 256 rows = 4 sequence slots x 64 node slots, 128 rows per CTA of the pair
+//             (T <= 64; missing nodes are zero-filled by the TMA out-of-bounds rule)
+//   N tile  = up to 256 vocabulary entries, a multiple of 32; each CTA loads one half of it
 //   K block = 64 bf16 = one 128-byte swizzle row; 4 MMAs of K = 16 per block
+//   Per k-block a CTA stages its own 128 rows of H (16 KB) and half of the W tile (16 KB):
+//   32 KB for 128 x 256 x 64 multiply-adds per SM, against 48 KB when every SM works
+//   alone. The pipeline is bound by how fast W tiles reach shared memory, so this is what
+//   lifts the tensor-core duty cycle.
 //   warps 0-3: epilogue (one TMEM lane = one row per thread), warp 4: TMA producer,
-//   warp 5: MMA issuer and TMEM owner. Accumulators are double-buffered in TMEM
-//   (2 x 256 columns) so that the epilogue of tile i overlaps the MMAs of tile i + 1.
-//   CTA c works on M tile (c % n_mt) and vocabulary range (c / n_mt): CTAs that share a
+//   warp 5: TMEM owner; in the leader CTA (cluster rank 0) one of its threads issues the
+//   MMAs of the pair. Accumulators are double-buffered in TMEM (2 x 256 columns per CTA)
+//   so that the epilogue of tile i overlaps the MMAs of tile i + 1.
+//   Pair c works on M tile (c % n_mt) and vocabulary range (c / n_mt): pairs that share a
 //   vocabulary range are neighbours and stream the same W tiles at the same time, so W is
 //   read from HBM once and re-hit in L2.
+//   Barriers: `full` lives in the leader and counts the bytes of both CTAs' loads; `empty`
+//   and `tmem_full` exist in both CTAs and are signalled by the leader's commits;
+//   `tmem_empty` lives in the leader and collects the epilogue warps of both CTAs.
 #include <math.h>
 
 #include "host_common.h"
@@ -24,18 +32,17 @@
 
 namespace trispec {
 
-constexpr int LM_BM = 128;
+constexpr int LM_BM = 128;                      // rows per CTA
 constexpr int LM_BN = 256;
 constexpr int LM_BK = 64;
-constexpr int LM_STAGES = 4;
-constexpr int LM_A_BYTES = LM_BM * LM_BK * 2;   // 16 KB
-constexpr int LM_B_BYTES = LM_BN * LM_BK * 2;   // 32 KB
+constexpr int LM_STAGES = 6;
+constexpr int LM_A_BYTES = LM_BM * LM_BK * 2;         // 16 KB
+constexpr int LM_B_BYTES = (LM_BN / 2) * LM_BK * 2;   // 16 KB: this CTA's half of the W tile
 constexpr int LM_BOX_BYTES = 64 * LM_BK * 2;    // one TMA box: 64 rows x 64 k
 constexpr int LM_STAGE_BYTES = LM_A_BYTES + LM_B_BYTES;
 constexpr int LM_THREADS = 192;
 constexpr int LM_SMEM_BYTES = LM_STAGES * LM_STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 struct __align__(16) LmPartial {
   float m, s, v1, v2;  // raw (unscaled) running max, sum of 2^((z-m)c), top-1 / top-2 raw logits
@@ -45,27 +52,29 @@ struct __align__(16) LmPartial {
 struct LmParams {
   int T, d, V;
   int n_seq;      // active sequences
-  int n_mt;       // M tiles = ceil(n_seq / 2)
+  int n_mt;       // M tiles of 4 sequence slots = ceil(n_seq / 4)
   int n_ranges;   // vocabulary ranges
   float c;        // logit_scale * log2(e)
   const int32_t* seq_index;
-  LmPartial* partial;  // [n_ranges][n_mt * 128]
+  LmPartial* partial;  // [n_ranges][n_mt * 256]
   int32_t* dev_status;
 };
 
+// Vocabulary range r of n_ranges, cut into tiles of at most 256 columns; all boundaries are
+// multiples of 32 columns so that each CTA of a pair takes a half that is a multiple of 16.
 struct TileIter {
   int u0, units, n_tiles;
   __device__ TileIter(int V, int n_ranges, int r) {
-    const int V16 = (V + 15) >> 4;
-    u0 = static_cast<int>((static_cast<long long>(V16) * r) / n_ranges);
-    const int u1 = static_cast<int>((static_cast<long long>(V16) * (r + 1)) / n_ranges);
+    const int V32 = (V + 31) >> 5;
+    u0 = static_cast<int>((static_cast<long long>(V32) * r) / n_ranges);
+    const int u1 = static_cast<int>((static_cast<long long>(V32) * (r + 1)) / n_ranges);
     units = u1 - u0;
-    n_tiles = (units + 15) >> 4;
+    n_tiles = (units + 7) >> 3;
   }
   __device__ void tile(int t, int& n0, int& nw) const {
     const int a = (units * t) / n_tiles, b = (units * (t + 1)) / n_tiles;
-    n0 = (u0 + a) << 4;
-    nw = (b - a) << 4;
+    n0 = (u0 + a) << 5;
+    nw = (b - a) << 5;
   }
 };
 
@@ -73,66 +82,78 @@ __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                    const LmParams p) {
   extern __shared__ uint8_t smem_raw[];
+  // the dynamic window starts at the same offset in both CTAs of the pair, so the aligned
+  // layouts coincide, as the paired MMA requires
   const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LM_STAGES * LM_STAGE_BYTES);
-  uint64_t* full_bar = bars;                      // [LM_STAGES]
+  uint64_t* full_bar = bars;                      // [LM_STAGES]  (used in the leader)
   uint64_t* empty_bar = bars + LM_STAGES;         // [LM_STAGES]
   uint64_t* tmem_full = bars + 2 * LM_STAGES;     // [2]
-  uint64_t* tmem_empty = bars + 2 * LM_STAGES + 2;  // [2]
+  uint64_t* tmem_empty = bars + 2 * LM_STAGES + 2;  // [2]        (used in the leader)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LM_STAGES + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int mt = blockIdx.x % p.n_mt;
-  const int range = blockIdx.x / p.n_mt;
+  const uint32_t rank = cluster_ctarank();        // 0 = leader
+  const int pair = blockIdx.x >> 1;
+  const int mt = pair % p.n_mt;
+  const int range = pair / p.n_mt;
   const TileIter tiles(p.V, p.n_ranges, range);
   const int n_kb = p.d / LM_BK;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < LM_STAGES; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 8); }
     fence_mbar_init();
   }
   if (warp == 5) {
-    tmem_alloc(tmem_slot, 512);
-    tmem_relinquish();
+    tmem_alloc_pair(tmem_slot, 512);
+    tmem_relinquish_pair();
   }
   if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_h); prefetch_tmap(&tmap_w); }
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();                             // both CTAs' barriers and TMEM are ready
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      const int a0 = 2 * mt, a1 = 2 * mt + 1;
+      // sequence slots of this CTA; a slot past the last active sequence re-reads the M tile's
+      // first sequence (its rows are computed and never looked at), which keeps the byte count
+      // of a stage the same in both CTAs
+      const int a_first = 4 * mt;
+      int a0 = a_first + 2 * static_cast<int>(rank), a1 = a0 + 1;
+      if (a0 >= p.n_seq) a0 = a_first;
+      if (a1 >= p.n_seq) a1 = a_first;
       const int s0 = p.seq_index ? __ldg(p.seq_index + a0) : a0;
-      const bool has1 = a1 < p.n_seq;
-      const int s1 = has1 ? (p.seq_index ? __ldg(p.seq_index + a1) : a1) : 0;
+      const int s1 = p.seq_index ? __ldg(p.seq_index + a1) : a1;
       int stage = 0;
       uint32_t phase = 0;
       for (int t = 0; t < tiles.n_tiles; ++t) {
         int n0, nw;
         tiles.tile(t, n0, nw);
-        const int nbox = (nw + 63) >> 6;
-        const uint32_t tx = static_cast<uint32_t>((has1 ? 2 : 1) + nbox) * LM_BOX_BYTES;
+        const int nh = nw >> 1;                   // rows of W this CTA stages
+        const int nbox = (nh + 63) >> 6;
+        const int w0 = n0 + static_cast<int>(rank) * nh;
+        const uint32_t tx_pair = 2u * static_cast<uint32_t>(2 + nbox) * LM_BOX_BYTES;
         for (int kb = 0; kb < n_kb; ++kb) {
           mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
           uint8_t* sa = smem + stage * LM_STAGE_BYTES;
           uint8_t* sb = sa + LM_A_BYTES;
-          mbar_expect_tx(full_bar + stage, tx);
-          tma_load_3d(sa, &tmap_h, full_bar + stage, kb * LM_BK, 0, s0);
-          if (has1) tma_load_3d(sa + LM_BOX_BYTES, &tmap_h, full_bar + stage, kb * LM_BK, 0, s1);
+          if (rank == 0) mbar_expect_tx(full_bar + stage, tx_pair);
+          const uint32_t fb = cluster_map(smem_u32(full_bar + stage), 0);
+          tma_load_3d_pair(sa, &tmap_h, fb, kb * LM_BK, 0, s0);
+          tma_load_3d_pair(sa + LM_BOX_BYTES, &tmap_h, fb, kb * LM_BK, 0, s1);
           for (int j = 0; j < nbox; ++j)
-            tma_load_2d(sb + j * LM_BOX_BYTES, &tmap_w, full_bar + stage, kb * LM_BK, n0 + 64 * j);
+            tma_load_2d_pair(sb + j * LM_BOX_BYTES, &tmap_w, fb, kb * LM_BK, w0 + 64 * j);
           if (++stage == LM_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA)
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       for (int t = 0; t < tiles.n_tiles; ++t) {
@@ -142,7 +163,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
         mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * LM_BN);
-        const uint32_t idesc = idesc_bf16(LM_BM, nw, false, false);
+        const uint32_t idesc = idesc_bf16(2 * LM_BM, nw, false, false);
         for (int kb = 0; kb < n_kb; ++kb) {
           mbar_wait(full_bar + stage, phase, p.dev_status);
           tc_fence_after();
@@ -153,20 +174,21 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
           for (int k = 0; k < LM_BK / 16; ++k) {
             // advancing 16 elements (32 bytes) along K inside the swizzle row: +2 in the
             // 16-byte-granular start address field
-            tc_mma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
+            tc_mma_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
           }
-          tc_commit(empty_bar + stage);
+          tc_commit_pair(empty_bar + stage, 3);   // the stage is free again in both CTAs
           if (++stage == LM_STAGES) { stage = 0; phase ^= 1u; }
         }
-        tc_commit(tmem_full + buf);
+        tc_commit_pair(tmem_full + buf, 3);       // both CTAs' accumulators are complete
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-3)
-    const int row = warp * 32 + lane;  // TMEM lane == row of the M tile
+    const int row = warp * 32 + lane;  // TMEM lane == row of this CTA's half of the M tile
     float m = -INFINITY, s = 0.f, v1 = -INFINITY, v2 = -INFINITY;
     int i1 = -1, i2 = -1;
     const float c = p.c;
+    const uint32_t tmem_empty_leader = cluster_map(smem_u32(tmem_empty), 0);
     for (int t = 0; t < tiles.n_tiles; ++t) {
       int n0, nw;
       tiles.tile(t, n0, nw);
@@ -208,18 +230,20 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tmem_empty + buf);
+      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + static_cast<uint32_t>(buf) * 8u);
     }
     LmPartial out;
     out.m = m; out.s = s; out.v1 = v1; out.v2 = v2; out.i1 = i1; out.i2 = i2; out.pad0 = 0; out.pad1 = 0;
-    p.partial[static_cast<size_t>(range) * (p.n_mt * LM_BM) + mt * LM_BM + row] = out;
+    p.partial[static_cast<size_t>(range) * (p.n_mt * 2 * LM_BM) + (mt * 2 + rank) * LM_BM + row] = out;
   }
 
+  // nobody leaves, and tensor memory stays allocated, until both CTAs are done: the leader's
+  // MMAs write the peer's tensor memory and its commits arrive on the peer's barriers
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();
   if (warp == 5) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc_pair(tmem_base, 512);
   }
 }
 
@@ -277,7 +301,7 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
   const int a = static_cast<int>(w / T), node = static_cast<int>(w % T);
   const int seq = p.seq_index ? __ldg(p.seq_index + a) : a;
   const long long row0 = static_cast<long long>(seq) * T;
-  const size_t stride = static_cast<size_t>(p.n_mt) * LM_BM;
+  const size_t stride = static_cast<size_t>(p.n_mt) * 2 * LM_BM;
   const size_t prow = static_cast<size_t>(a) * 64 + node;
 
   float M, S;
@@ -341,12 +365,12 @@ static int lm_plan(const trispec_lmhead_args* a, int* n_seq, int* n_mt, int* n_r
   if (a->T > 64 || (a->d % LM_BK) != 0 || a->V < 2) return TRISPEC_ERR_UNSUPPORTED;
   *n_seq = a->seq_index ? a->B_active : a->B;
   if (*n_seq <= 0 || *n_seq > a->B) return TRISPEC_ERR_INVALID_ARG;
-  *n_mt = (*n_seq + 1) / 2;
-  const int sms = device_sm_count();
-  int r = sms / *n_mt;
+  *n_mt = (*n_seq + 3) / 4;
+  const int pairs = device_sm_count() / 2;       // one CTA pair per two SMs
+  int r = pairs / *n_mt;
   if (r < 1) r = 1;
-  const int V16 = (a->V + 15) / 16;
-  if (r > V16) r = V16;
+  const int V32 = (a->V + 31) / 32;
+  if (r > V32) r = V32;
   *n_ranges = r;
   return TRISPEC_OK;
 }
@@ -357,7 +381,7 @@ extern "C" size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a) {
   using namespace trispec;
   int n_seq, n_mt, n_ranges;
   if (lm_plan(a, &n_seq, &n_mt, &n_ranges) != TRISPEC_OK) return 0;
-  return static_cast<size_t>(n_ranges) * n_mt * LM_BM * sizeof(LmPartial);
+  return static_cast<size_t>(n_ranges) * n_mt * 2 * LM_BM * sizeof(LmPartial);
 }
 
 extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) {
@@ -399,9 +423,22 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   p.seq_index = a->seq_index;
   p.partial = static_cast<LmPartial*>(a->workspace);
   p.dev_status = a->dev_status;
-  lmhead_gemm_kernel<<<n_mt * n_ranges, LM_THREADS, LM_SMEM_BYTES, st>>>(tm_h, tm_w, p);
-  count_launch();
-  TRISPEC_CUDA_OK(cudaGetLastError());
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * n_mt * n_ranges), 1, 1);
+    cfg.blockDim = dim3(LM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = LM_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    TRISPEC_CUDA_OK(cudaLaunchKernelEx(&cfg, lmhead_gemm_kernel, tm_h, tm_w, p));
+    count_launch();
+  }
 
   LmFinalizeParams f;
   f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges;
