@@ -54,7 +54,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -241,18 +241,27 @@ def main():
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n0 = ts.launch_count()
     sync_all()
     t_host0 = time.perf_counter()
-    for s, e in ev:
-        s.record(stream)
+    e_start.record(stream)
+    for _ in range(args.steps):
         pas.run()
-        e.record(stream)
+    e_end.record(stream)
     host_us_per_call = (time.perf_counter() - t_host0) / args.steps * 1e6   # launch cost, GPU running behind
     sync_all()
     launches = ts.launch_count() - n0
-    total_ms = sum(s.elapsed_time(e) for s, e in ev)
+    total_ms = e_start.elapsed_time(e_end)      # K passes back to back, one bracket
+    # latency of a single pass (each bracketed by its own events; clocks recover between them)
+    n_lat = min(args.steps, 100)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
+    for s_, e_ in ev:
+        s_.record(stream)
+        pas.run()
+        e_.record(stream)
+    torch.cuda.synchronize()
+    pass_latency_ms = statistics.median(s_.elapsed_time(e_) for s_, e_ in ev)
 
     # ---- per-step breakdown, measured in situ with the launch queue kept full:
     #   lmhead    = K back-to-back calls of trispec_lmhead_stats (W, 0.6 GB, evicts itself from L2)
@@ -337,7 +346,7 @@ def main():
                    "parallelism": "independent replicas, one batch per GPU"},
         "e2e": {"value": tokens / (e2e_ms * 1e-3 / args.steps), "unit": UNIT,
                 "h2d_bytes_per_step": pas.h2d_bytes, "d2h_bytes_per_step": pas.d2h_bytes},
-        "gpu_launches": launches, "host_us_per_call": host_us_per_call,
+        "gpu_launches": launches, "host_us_per_call": host_us_per_call, "pass_latency_ms_median": pass_latency_ms,
         "clocks": clocks,
         "roofline": {"kernel": "lmhead_gemm_kernel", "bound": "tensor", "achieved": lm_tflops,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": lm_tflops / peaks["bf16_tflops"],

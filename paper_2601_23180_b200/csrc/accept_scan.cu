@@ -11,6 +11,8 @@ constexpr int kScanThreads = 256;  // 8 sequences per block
 
 __global__ void __launch_bounds__(kScanThreads)
 accept_scan_kernel(trispec_scan_args a) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long b = static_cast<long long>(blockIdx.x) * (kScanThreads / 32) + (threadIdx.x >> 5);
   if (b >= a.B) return;
@@ -75,6 +77,8 @@ esc_compact_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restr
                    int32_t* __restrict__ n_escalated) {
   __shared__ int warp_excl[32];
   __shared__ int running;
+  pdl_launch_dependents();
+  pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) running = 0;
   __syncthreads();
@@ -131,13 +135,12 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int per_block = kScanThreads / 32;
   unsigned grid = static_cast<unsigned>((static_cast<long long>(a->B) + per_block - 1) / per_block);
-  accept_scan_kernel<<<grid, kScanThreads, 0, st>>>(*a);
+  TRISPEC_CUDA_OK(launch_dependent(accept_scan_kernel, grid, kScanThreads, 0, st, 1, *a));
   count_launch();
-  TRISPEC_CUDA_OK(cudaGetLastError());
   if (a->esc_index) {
-    esc_compact_kernel<<<1, kCompactThreads, 0, st>>>(a->escalate, a->B, a->esc_index, a->n_escalated);
+    TRISPEC_CUDA_OK(launch_dependent(esc_compact_kernel, 1, kCompactThreads, 0, st, 1,
+                                     static_cast<const uint8_t*>(a->escalate), a->B, a->esc_index, a->n_escalated));
     count_launch();
-    TRISPEC_CUDA_OK(cudaGetLastError());
   }
   return TRISPEC_OK;
 }

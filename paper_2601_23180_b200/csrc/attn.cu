@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2)
 verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                          const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt,
                          const AttnParams p) {
+  pdl_launch_dependents();
   // ---- which work item: the split index varies fastest, so that in cluster mode the CTAs of
   // one cluster are the splits of one (sequence, KV head, M tile) and cluster rank == split
   int idx = blockIdx.x;
@@ -287,7 +288,6 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     const int row = warp * 32 + lane;
     const int node = mtile * p.NPT + row / p.G;
     const bool row_valid = (row < p.NPT * p.G) && (node < p.T);
-    const uint64_t mrow = row_valid ? __ldg(p.mask + static_cast<long long>(b) * p.T + node) : 0ull;
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     // Q row -> TMEM (A operand of S = Q K^T): lane = row, column c = dims (2c, 2c + 1)
     {
@@ -331,7 +331,9 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       uint64_t vis;
       int nvalid = AT_BN;
       if (tree) {
-        vis = mrow;
+        // the mask comes from the kernel before this one on the stream: first dependent read
+        pdl_wait();
+        vis = row_valid ? __ldg(p.mask + static_cast<long long>(b) * p.T + node) : 0ull;
       } else {
         nvalid = min(AT_BN, L - (t_begin + i) * AT_BN);
         vis = (nvalid >= 64) ? ~0ull : ((1ull << nvalid) - 1ull);
@@ -432,6 +434,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       }
       sPartML[row] = make_float2(m_ref, l);
     } else {
+      pdl_wait();                                // before the first global write
       const size_t item = static_cast<size_t>(blockIdx.x);
       float* po = p.part_o + (item * AT_BM + row) * AT_D;
 #pragma unroll
@@ -468,6 +471,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     if (idle_cta) {
       for (int r = threadIdx.x; r < AT_BM; r += AT_THREADS) sPartML[r] = make_float2(-INFINITY, 0.f);
     }
+    pdl_wait();                                  // before the first global write (o, lse)
     cluster_sync_all();
     // Requests over the SM-to-SM network are expensive per instruction, whatever their size,
     // so they are few and wide: one gather of the (m, l) pairs of all splits for this CTA's
@@ -547,6 +551,8 @@ struct AttnMergeParams {
 
 __global__ void __launch_bounds__(256)
 verify_attn_merge_kernel(const AttnMergeParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long w = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   const long long total = static_cast<long long>(p.n_seq) * p.T * p.Hq;
@@ -705,26 +711,15 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   p.lse = a->lse;
   p.dev_status = a->dev_status;
   if (pl.cluster) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(pl.items), 1, 1);
-    cfg.blockDim = dim3(AT_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = AT_SMEM_BYTES;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = static_cast<unsigned>(pl.n_splits);
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    TRISPEC_CUDA_OK(cudaLaunchKernelEx(&cfg, verify_attn_split_kernel<true>, tm_k, tm_v, tm_kt, tm_vt, p));
+    TRISPEC_CUDA_OK(launch_dependent(verify_attn_split_kernel<true>, static_cast<unsigned>(pl.items), AT_THREADS,
+                                     AT_SMEM_BYTES, st, static_cast<unsigned>(pl.n_splits), tm_k, tm_v, tm_kt, tm_vt,
+                                     p));
     count_launch();
     return TRISPEC_OK;
   }
-  verify_attn_split_kernel<false><<<static_cast<unsigned>(pl.items), AT_THREADS, AT_SMEM_BYTES, st>>>(tm_k, tm_v, tm_kt,
-                                                                                                       tm_vt, p);
+  TRISPEC_CUDA_OK(launch_dependent(verify_attn_split_kernel<false>, static_cast<unsigned>(pl.items), AT_THREADS,
+                                   AT_SMEM_BYTES, st, 1, tm_k, tm_v, tm_kt, tm_vt, p));
   count_launch();
-  TRISPEC_CUDA_OK(cudaGetLastError());
 
   AttnMergeParams m;
   m.T = a->T; m.Hq = a->Hq; m.Hkv = a->Hkv; m.G = pl.G; m.NPT = pl.NPT; m.n_mt = pl.n_mt;
@@ -733,8 +728,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   m.part_o = p.part_o; m.part_ml = p.part_ml;
   m.o = static_cast<uint16_t*>(a->o); m.lse = a->lse;
   const long long rows = static_cast<long long>(pl.n_seq) * a->T * a->Hq;
-  verify_attn_merge_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, st>>>(m);
+  TRISPEC_CUDA_OK(launch_dependent(verify_attn_merge_kernel, static_cast<unsigned>((rows + 7) / 8), 256, 0, st, 1, m));
   count_launch();
-  TRISPEC_CUDA_OK(cudaGetLastError());
   return TRISPEC_OK;
 }

@@ -28,6 +28,43 @@ int device_sm_count();
 // Raises the dynamic shared memory limit of `func` once per device.
 int ensure_smem_limit(const void* func, int bytes, bool* done_per_device /* [64] */);
 
+// Every kernel of the verify pass is launched as a programmatic dependent of the kernel before
+// it on the stream: its CTAs may be scheduled as soon as all CTAs of that kernel have called
+// pdl_launch_dependents() (they do so at their start) and resources are free, so launch
+// latency, prologues and tails overlap. A kernel calls pdl_wait() before its first read of
+// anything an earlier kernel writes and before its first global write; the wait returns once
+// all earlier kernels on the stream have completed and their writes are visible. Because
+// every kernel waits before it completes, completion stays in stream order.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                    cudaStream_t st, unsigned cluster_x, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(block, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  unsigned n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 #define TRISPEC_CUDA_OK(expr)                        \
   do {                                               \
     cudaError_t _e = (expr);                         \

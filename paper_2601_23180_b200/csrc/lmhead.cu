@@ -81,6 +81,7 @@ struct TileIter {
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                    const LmParams p) {
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   // the dynamic window starts at the same offset in both CTAs of the pair, so the aligned
   // layouts coincide, as the paired MMA requires
@@ -232,11 +233,13 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + static_cast<uint32_t>(buf) * 8u);
     }
+    pdl_wait();   // the partials of the previous pass may still be read until earlier kernels are done
     LmPartial out;
     out.m = m; out.s = s; out.v1 = v1; out.v2 = v2; out.i1 = i1; out.i2 = i2; out.pad0 = 0; out.pad1 = 0;
     p.partial[static_cast<size_t>(range) * (p.n_mt * 2 * LM_BM) + (mt * 2 + rank) * LM_BM + row] = out;
   }
 
+  pdl_wait();
   // nobody leaves, and tensor memory stays allocated, until both CTAs are done: the leader's
   // MMAs write the peer's tensor memory and its commits arrive on the peer's barriers
   tc_fence_before();
@@ -294,6 +297,8 @@ __device__ __forceinline__ void lm_row_lse(const LmPartial* part, size_t stride,
 // node, computes the logit of its drafted token in its parent's row (a d-long dot product).
 __global__ void __launch_bounds__(LM_FIN_THREADS)
 lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long w = static_cast<long long>(blockIdx.x) * (LM_FIN_THREADS / 32) + (threadIdx.x >> 5);
   const int T = p.T;
@@ -423,22 +428,9 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   p.seq_index = a->seq_index;
   p.partial = static_cast<LmPartial*>(a->workspace);
   p.dev_status = a->dev_status;
-  {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(2 * n_mt * n_ranges), 1, 1);
-    cfg.blockDim = dim3(LM_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = LM_SMEM_BYTES;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    TRISPEC_CUDA_OK(cudaLaunchKernelEx(&cfg, lmhead_gemm_kernel, tm_h, tm_w, p));
-    count_launch();
-  }
+  TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel, static_cast<unsigned>(2 * n_mt * n_ranges), LM_THREADS,
+                                   LM_SMEM_BYTES, st, 2, tm_h, tm_w, p));
+  count_launch();
 
   LmFinalizeParams f;
   f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges;
@@ -449,8 +441,8 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   f.W = static_cast<const uint16_t*>(a->W);
   f.parent = a->parent; f.tok = a->tok;
   f.out = a->out;
-  lmhead_finalize_kernel<<<(n_seq * a->T + 7) / 8, LM_FIN_THREADS, 0, st>>>(f, n_seq);
+  TRISPEC_CUDA_OK(launch_dependent(lmhead_finalize_kernel, static_cast<unsigned>((n_seq * a->T + 7) / 8),
+                                   LM_FIN_THREADS, 0, st, 1, f, n_seq));
   count_launch();
-  TRISPEC_CUDA_OK(cudaGetLastError());
   return TRISPEC_OK;
 }

@@ -10,6 +10,8 @@ constexpr int kMaskThreads = 256;
 __global__ void __launch_bounds__(kMaskThreads)
 tree_mask_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask, int32_t* __restrict__ depth,
                  long long n_nodes, int T) {
+  pdl_launch_dependents();
+  pdl_wait();
   long long idx = static_cast<long long>(blockIdx.x) * kMaskThreads + threadIdx.x;
   if (idx >= n_nodes) return;
   long long seq_base = (idx / T) * T;
@@ -40,9 +42,8 @@ extern "C" int trispec_build_tree_mask(const trispec_tree_args* a, void* stream)
   if (a->T > 64) return TRISPEC_ERR_UNSUPPORTED;
   long long n = static_cast<long long>(a->B) * a->T;
   unsigned grid = static_cast<unsigned>((n + kMaskThreads - 1) / kMaskThreads);
-  tree_mask_kernel<<<grid, kMaskThreads, 0, static_cast<cudaStream_t>(stream)>>>(a->parent, a->mask, a->depth, n,
-                                                                                  a->T);
+  TRISPEC_CUDA_OK(launch_dependent(tree_mask_kernel, grid, kMaskThreads, 0, static_cast<cudaStream_t>(stream), 1,
+                                   a->parent, a->mask, a->depth, n, a->T));
   count_launch();
-  TRISPEC_CUDA_OK(cudaGetLastError());
   return TRISPEC_OK;
 }
