@@ -43,7 +43,8 @@ typedef enum {
   TRISPEC_ERR_UNSUPPORTED = 2,     /* D != 128, T > 64, unsupported group size, ... */
   TRISPEC_ERR_WORKSPACE = 3,       /* workspace_bytes smaller than the *_workspace() query */
   TRISPEC_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed */
-  TRISPEC_ERR_DEVICE_TIMEOUT = 5   /* value written to dev_status by a bounded wait */
+  TRISPEC_ERR_DEVICE_TIMEOUT = 5,  /* value written to dev_status by a bounded wait */
+  TRISPEC_ERR_TOO_LARGE = 8        /* problem needs more than the library's built-in scratch */
 } trispec_status;
 
 #define TRISPEC_MODE_PROXY 0   /* margin rule of Eq. 8-9 applied (proxy verifier) */
@@ -142,6 +143,31 @@ typedef struct {
 } trispec_lmhead_args;
 size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a);
 int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 3b. LM-head statistics for callers that cannot allocate device memory. (The paper has no
+ *     counterpart: this is a packaging variant of entry point 3, same inputs, same results.)
+ *     A decode loop embedded in a serving engine often runs after the engine has handed all
+ *     free device memory to its KV-cache pool; a cudaMalloc there fails or, when it works,
+ *     stalls every stream of the process. Such a caller has nowhere to get the per-call
+ *     workspace of trispec_lmhead_stats from. This entry point takes none: the per-slice
+ *     partial statistics go to a fixed array of TRISPEC_NOALLOC_SCRATCH_BYTES that is part of
+ *     the library image (every GPU that loads the library holds that much until the process
+ *     exits). `workspace` and `workspace_bytes` of the argument struct are ignored; inputs
+ *     and outputs are still the caller's. No device or host memory is allocated or freed.
+ *       - Limit: trispec_lmhead_stats_workspace(a) <= TRISPEC_NOALLOC_SCRATCH_BYTES (1 MiB:
+ *         up to 512 active sequences); beyond that the call returns TRISPEC_ERR_TOO_LARGE
+ *         and launches nothing.
+ *       - The first call on each device looks up the device address of the array (one
+ *         runtime call, with that device current); make that first call outside any stream
+ *         capture. Later calls on the device reuse the address.
+ *       - All calls on a device share the one array, and it keeps whatever the last call left
+ *         in it. Nothing in it needs clearing: a call overwrites every entry it later reads.
+ *         Two calls whose kernels overlap on the GPU (different streams) race on it; calls on
+ *         one stream are ordered and safe.
+ * ------------------------------------------------------------------------------------- */
+#define TRISPEC_NOALLOC_SCRATCH_BYTES (1u << 20)
+int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * 4. Acceptance scan (Eq. 6 greedy form, Eq. 7, Eq. 8, Eq. 9, routing cases (i)/(ii),

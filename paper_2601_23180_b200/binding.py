@@ -75,6 +75,7 @@ _lib.trispec_verify_attn.argtypes = [C.POINTER(AttnArgs), _vp]
 _lib.trispec_lmhead_stats_workspace.restype = _sz
 _lib.trispec_lmhead_stats_workspace.argtypes = [C.POINTER(LmheadArgs)]
 _lib.trispec_lmhead_stats.argtypes = [C.POINTER(LmheadArgs), _vp]
+_lib.trispec_lmhead_stats_noalloc.argtypes = [C.POINTER(LmheadArgs), _vp]
 _lib.trispec_accept_scan.argtypes = [C.POINTER(ScanArgs), _vp]
 _lib.trispec_verify.argtypes = [C.POINTER(TreeArgs), C.POINTER(AttnArgs), C.POINTER(LmheadArgs),
                                 C.POINTER(ScanArgs), _vp]
@@ -84,7 +85,7 @@ _lib.trispec_verify_host.argtypes = [C.POINTER(HostIO), C.POINTER(TreeArgs), C.P
 
 EXPORTS = ["trispec_verify_host", "trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
            "trispec_verify_attn_workspace", "trispec_verify_attn", "trispec_lmhead_stats_workspace",
-           "trispec_lmhead_stats", "trispec_accept_scan", "trispec_verify"]
+           "trispec_lmhead_stats", "trispec_lmhead_stats_noalloc", "trispec_accept_scan", "trispec_verify"]
 
 
 class TrispecError(RuntimeError):
@@ -228,6 +229,15 @@ def trispec_lmhead_stats_workspace(args: LmheadArgs) -> int:
 
 def trispec_lmhead_stats(args: LmheadArgs, stream=None):
     _check(_lib.trispec_lmhead_stats(C.byref(args), _stream(stream)))
+
+
+NOALLOC_SCRATCH_BYTES = 1 << 20
+
+
+def trispec_lmhead_stats_noalloc(args: LmheadArgs, stream=None):
+    """LM-head statistics without a caller workspace (the library's built-in 1 MiB scratch is
+    used; `args.workspace` is ignored). For callers that must not allocate device memory."""
+    _check(_lib.trispec_lmhead_stats_noalloc(C.byref(args), _stream(stream)))
 
 
 def trispec_accept_scan(args: ScanArgs, stream=None):

@@ -117,6 +117,7 @@ extern "C" const char* trispec_status_string(int s) {
     case TRISPEC_ERR_WORKSPACE: return "workspace too small";
     case TRISPEC_ERR_CUDA: return "CUDA call failed";
     case TRISPEC_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case TRISPEC_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }

@@ -27,6 +27,8 @@
 //   `tmem_empty` lives in the leader and collects the epilogue warps of both CTAs.
 #include <math.h>
 
+#include <mutex>
+
 #include "host_common.h"
 #include "sm100.cuh"
 
@@ -445,4 +447,48 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
                                    LM_FIN_THREADS, 0, st, 1, f, n_seq));
   count_launch();
   return TRISPEC_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// No-allocation variant: the partial statistics live in an array that is part of the library
+// image instead of a caller-provided workspace.
+// ---------------------------------------------------------------------------------------
+namespace trispec {
+// Scratch shared by every call on a device. In host code this name is only a handle for the
+// runtime's symbol table, not an address a kernel could use: the device address is looked up
+// once per device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_lm_noalloc_scratch[TRISPEC_NOALLOC_SCRATCH_BYTES];
+
+// Device address of the scratch array on the current device; looked up on the first call per
+// device (with that device current) and remembered.
+static int lm_noalloc_scratch(void** out) {
+  static void* addr[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TRISPEC_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return TRISPEC_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_lm_noalloc_scratch) != cudaSuccess || !ptr) return TRISPEC_ERR_CUDA;
+    addr[dev] = ptr;
+  }
+  *out = addr[dev];
+  return TRISPEC_OK;
+}
+}  // namespace trispec
+
+extern "C" int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream) {
+  using namespace trispec;
+  int n_seq, n_mt, n_ranges;
+  int rc = lm_plan(a, &n_seq, &n_mt, &n_ranges);
+  if (rc != TRISPEC_OK) return rc;
+  if (trispec_lmhead_stats_workspace(a) > TRISPEC_NOALLOC_SCRATCH_BYTES) return TRISPEC_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  rc = lm_noalloc_scratch(&scratch);
+  if (rc != TRISPEC_OK) return rc;
+  trispec_lmhead_args b = *a;     // same call, with the built-in array as its workspace
+  b.workspace = scratch;
+  b.workspace_bytes = TRISPEC_NOALLOC_SCRATCH_BYTES;
+  return trispec_lmhead_stats(&b, stream);
 }
