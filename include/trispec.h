@@ -209,10 +209,14 @@ int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
  * The same pass for callers whose per-round data lives in HOST memory (one verification
  * round of Algorithm 1 as a decode loop sees it: the draft tree and its activations arrive
  * from the host, the routing decision goes back to it). The KV cache and the LM-head weights
- * stay resident on the device. In order, on `stream`: copies the per-round inputs from the
- * host pointers of `io` into the device buffers named by the argument structs
- * (tree->parent, lm->tok, attn->q, attn->k_tree, attn->v_tree, lm->h), runs trispec_verify,
- * then copies accept_len, escalate, bonus_tok, last_node and path back to the host pointers.
+ * stay resident on the device. Copies the per-round inputs from the host pointers of `io`
+ * into the device buffers named by the argument structs (tree->parent, lm->tok, lm->h on
+ * `stream`; attn->q, attn->k_tree, attn->v_tree on a stream of the library's own, ordered
+ * after everything already on `stream`, so that they overlap the LM-head GEMM), runs the
+ * tree mask, the LM-head statistics, the attention and the scan, then copies accept_len,
+ * escalate, bonus_tok, last_node and path back to the host pointers. Seen from `stream` the
+ * call is one ordered unit of work. The first call on a device creates that stream and two
+ * events (host resources, kept until the process exits); no device memory is allocated.
  * Host pointers should be page-locked for the copies to be asynchronous; the results are
  * valid once `stream` has been synchronised. NULL host input pointers skip that copy.
  * ------------------------------------------------------------------------------------- */
