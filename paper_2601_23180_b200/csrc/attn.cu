@@ -54,7 +54,7 @@ constexpr int AT_PART_ML2_OFF = AT_PART_ML_OFF + AT_BM * 8;   // gathered (m, l)
 static_assert(AT_PART_ML2_OFF + AT_BM * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
 
 struct AttnParams {
-  int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split;
+  int T, Hq, Hkv, G, NPT, n_mt, n_splits;
   int paged, max_blocks_per_seq, num_blocks;
   float scale_log2;
   const uint16_t* q;
@@ -101,9 +101,12 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
   const int L = __ldg(p.ctx_len + b);
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
-  const int last_split = max(0, (n_ctx_tiles + p.tiles_per_split - 1) / p.tiles_per_split - 1);
-  const int t_begin = split * p.tiles_per_split;
-  const int t_end = min(n_ctx_tiles, t_begin + p.tiles_per_split);
+  // every sequence spreads its own context tiles evenly over the splits, so that the CTAs that
+  // merge with each other finish together whatever the sequence's length
+  const int tiles_per_split = max(1, (n_ctx_tiles + p.n_splits - 1) / p.n_splits);
+  const int last_split = max(0, (n_ctx_tiles + tiles_per_split - 1) / tiles_per_split - 1);
+  const int t_begin = split * tiles_per_split;
+  const int t_end = min(n_ctx_tiles, t_begin + tiles_per_split);
   const bool has_tree = (split == last_split);
   const int n_tiles = (t_end - t_begin) + (has_tree ? 1 : 0);   // >= 1 unless this split is empty
 
@@ -542,7 +545,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 // Merge of the KV splits: one warp per output row (sequence, node, query head).
 // ---------------------------------------------------------------------------------------
 struct AttnMergeParams {
-  int T, Hq, Hkv, G, NPT, n_mt, n_splits, tiles_per_split, n_seq;
+  int T, Hq, Hkv, G, NPT, n_mt, n_splits, n_seq;
   const int32_t *ctx_len, *seq_index;
   const float *part_o, *part_ml;
   uint16_t* o;   // bf16 [B][T][Hq][128]
@@ -566,7 +569,8 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
   const int row = (node % p.NPT) * p.G + j;
   const int L = __ldg(p.ctx_len + b);
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
-  const int n_valid = max(0, (n_ctx_tiles + p.tiles_per_split - 1) / p.tiles_per_split - 1) + 1;
+  const int tiles_per_split = max(1, (n_ctx_tiles + p.n_splits - 1) / p.n_splits);
+  const int n_valid = max(0, (n_ctx_tiles + tiles_per_split - 1) / tiles_per_split - 1) + 1;
   const size_t item0 = ((static_cast<size_t>(a) * p.Hkv + g) * p.n_mt + mtile) * p.n_splits;
   float M = -INFINITY;
   for (int s = 0; s < n_valid; ++s) {
@@ -594,7 +598,7 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
 }
 
 struct AttnPlan {
-  int n_seq, G, NPT, n_mt, tiles_max, tiles_per_split, n_splits;
+  int n_seq, G, NPT, n_mt, tiles_max, n_splits;
   bool cluster;      // splits merged inside a thread-block cluster (no workspace)
   size_t items;
 };
@@ -622,20 +626,22 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   pl->n_mt = (a->T + pl->NPT - 1) / pl->NPT;
   pl->tiles_max = (Lmax + AT_BN - 1) / AT_BN;
   const long long fixed = static_cast<long long>(pl->n_seq) * a->Hkv * pl->n_mt;
-  const long long target = static_cast<long long>(device_sm_count()) * 2 * 8;   // ~8 waves of 2 CTAs/SM
-  long long c = (static_cast<long long>(pl->tiles_max) * fixed + target - 1) / target;
-  if (c < 16) c = 16;
-  if (c > pl->tiles_max) c = pl->tiles_max > 0 ? pl->tiles_max : 1;
-  pl->tiles_per_split = static_cast<int>(c);
-  pl->n_splits = pl->tiles_max > 0 ? (pl->tiles_max + pl->tiles_per_split - 1) / pl->tiles_per_split : 1;
-  pl->cluster = pl->n_splits <= 8;
-  if (pl->cluster) {
-    // cluster sizes 1, 2, 4, 8 (the portable limit); rows of the M tile divide evenly among them
-    int s = 1;
-    while (s < pl->n_splits) s <<= 1;
-    pl->n_splits = s;
-    pl->tiles_per_split = pl->tiles_max > 0 ? (pl->tiles_max + s - 1) / s : 1;
+  // Number of KV splits: a power of two that minimises waves x (fixed cost + tiles per CTA).
+  // The fixed cost of a CTA (pipeline fill, Q load, merge) is worth about 8 context tiles; more
+  // than 8 splits cannot form a cluster and pay for a second kernel (about 6 tiles).
+  const long long slots = static_cast<long long>(device_sm_count()) * 2;   // two CTAs per SM
+  long long best_cost = -1;
+  int best_s = 1;
+  for (int sp = 1; sp <= 1024; sp <<= 1) {
+    if (sp > 1 && pl->tiles_max / sp < 4) break;
+    const long long ctas = fixed * sp;
+    const long long waves = (ctas + slots - 1) / slots;
+    const long long per_cta = 8 + (pl->tiles_max + sp - 1) / sp;
+    const long long cost = waves * per_cta + (sp > 8 ? 6 : 0);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_s = sp; }
   }
+  pl->n_splits = best_s;
+  pl->cluster = pl->n_splits <= 8;
   pl->items = static_cast<size_t>(fixed) * pl->n_splits;
   if (pl->items > 0x7fffffffull) return TRISPEC_ERR_UNSUPPORTED;
   return TRISPEC_OK;
@@ -699,7 +705,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   if (rc != TRISPEC_OK) return rc;
   AttnParams p;
   p.T = a->T; p.Hq = a->Hq; p.Hkv = a->Hkv; p.G = pl.G; p.NPT = pl.NPT; p.n_mt = pl.n_mt;
-  p.n_splits = pl.n_splits; p.tiles_per_split = pl.tiles_per_split;
+  p.n_splits = pl.n_splits;
   p.paged = (a->kv_layout == TRISPEC_KV_PAGED); p.max_blocks_per_seq = a->max_blocks_per_seq;
   p.num_blocks = a->num_blocks;
   p.scale_log2 = a->scale * kLog2e;
@@ -723,7 +729,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
 
   AttnMergeParams m;
   m.T = a->T; m.Hq = a->Hq; m.Hkv = a->Hkv; m.G = pl.G; m.NPT = pl.NPT; m.n_mt = pl.n_mt;
-  m.n_splits = pl.n_splits; m.tiles_per_split = pl.tiles_per_split; m.n_seq = pl.n_seq;
+  m.n_splits = pl.n_splits; m.n_seq = pl.n_seq;
   m.ctx_len = a->ctx_len; m.seq_index = a->seq_index;
   m.part_o = p.part_o; m.part_ml = p.part_ml;
   m.o = static_cast<uint16_t*>(a->o); m.lse = a->lse;
