@@ -346,7 +346,12 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       if (!tree && nvalid >= AT_BN) {
 #pragma unroll
-        for (int j = 0; j < 64; ++j) tm[j & 3] = fmaxf(tm[j & 3], __uint_as_float(sr[j]));
+        for (int j = 0; j < 64; j += 8) {
+          tm[0] = fmax3(tm[0], __uint_as_float(sr[j]), __uint_as_float(sr[j + 1]));
+          tm[1] = fmax3(tm[1], __uint_as_float(sr[j + 2]), __uint_as_float(sr[j + 3]));
+          tm[2] = fmax3(tm[2], __uint_as_float(sr[j + 4]), __uint_as_float(sr[j + 5]));
+          tm[3] = fmax3(tm[3], __uint_as_float(sr[j + 6]), __uint_as_float(sr[j + 7]));
+        }
       } else {
 #pragma unroll
         for (int j = 0; j < 64; ++j) {
@@ -380,22 +385,27 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         }
       }
       const float nmu = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nmu2 = make_float2(nmu, nmu);
       uint8_t* prow = sP + row * 128;
 #pragma unroll
       for (int cch = 0; cch < 8; ++cch) {
         float e[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          e[j] = ex2f(fmaf(__uint_as_float(sr[cch * 8 + j]), p.scale_log2, nmu));   // exp2(s * scale - m)
-          ls[j & 3] += e[j];
+        for (int j = 0; j < 8; j += 2) {
+          // exp2(s * scale - m) on two scores at a time
+          const float2 t = ffma2(make_float2(__uint_as_float(sr[cch * 8 + j]), __uint_as_float(sr[cch * 8 + j + 1])),
+                                 sc2, nmu2);
+          e[j] = ex2f(t.x);
+          e[j + 1] = ex2f(t.y);
+          ls[(j >> 1) & 1] = fadd2(ls[(j >> 1) & 1], make_float2(e[j], e[j + 1]));
         }
         uint4 pk;
         pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]);
         pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
         *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk;
       }
-      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      l += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
       if (nvalid < AT_BN) {
         // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
         mbar_wait(v_full + stage, (i / AT_STAGES) & 1u, p.dev_status);
@@ -412,7 +422,31 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     // ---------------------------------------------------------------- epilogue
     mbar_wait(o_bar, (n_tiles - 1) & 1u, p.dev_status);
     tc_fence_after();
-    if (kCluster) {
+    if (kCluster && p.n_splits == 1) {
+      // a single split is the whole result: normalise and store it straight from tensor memory
+      pdl_wait();                                // before the first global write
+      const float invl = (l > 0.f) ? 1.f / l : 0.f;
+      const int hq = g * p.G + row % p.G;
+      uint16_t* orow = p.o + ((static_cast<size_t>(b) * p.T + (row_valid ? node : 0)) * p.Hq + hq) * AT_D;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
+        tc_wait_ld();
+        if (row_valid) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(o[j]) * invl, __uint_as_float(o[j + 1]) * invl);
+            pk.y = pack_bf16(__uint_as_float(o[j + 2]) * invl, __uint_as_float(o[j + 3]) * invl);
+            pk.z = pack_bf16(__uint_as_float(o[j + 4]) * invl, __uint_as_float(o[j + 5]) * invl);
+            pk.w = pack_bf16(__uint_as_float(o[j + 6]) * invl, __uint_as_float(o[j + 7]) * invl);
+            *reinterpret_cast<uint4*>(orow + c * 32 + j) = pk;
+          }
+        }
+      }
+      if (row_valid && p.lse) p.lse[(static_cast<size_t>(b) * p.Hq + hq) * p.T + node] = (m_ref + log2f(l)) * kLn2;
+    } else if (kCluster) {
       // partial (O / l as bf16, m, l) -> this CTA's shared memory (the K/V ring is idle: every
       // tile has been consumed by its MMAs). The exchange between the CTAs of a cluster goes
       // over the SM-to-SM network, whose bandwidth is a small fraction of shared memory's, so the
@@ -467,7 +501,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   }
   }   // !idle_cta
 
-  if (kCluster) {
+  if (kCluster && p.n_splits > 1) {
     // ---------------------------------------------------------------- cluster merge
     // Every CTA of the cluster holds one partial in its shared memory (idle CTAs: weight zero).
     // CTA `split` normalises rows [split * 128 / n_splits, (split + 1) * 128 / n_splits).
