@@ -28,9 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "verified_draft_tokens_per_s"
 UNIT = "draft tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_gemm_kernel launch on the bench
-# workload, from the ncu capture summarised in profiles/ (None until captured).
-LMHEAD_GEMM_DRAM_TRAFFIC = {"proxy_tree": None}
+# dram__bytes_read.sum + dram__bytes_write.sum (bytes) of one lmhead_gemm_kernel launch on the bench
+# workload, from the ncu capture summarised in profiles/lmhead_gemm_kernel_proxy_tree.md.
+LMHEAD_GEMM_DRAM_TRAFFIC = {"proxy_tree": 629.1e6}
 
 
 def _peaks():
@@ -109,7 +109,12 @@ def oracle_sample(cfg, inp, n_attn_rows: int, n_lm_rows: int):
     t_mask = time.perf_counter() - t0
     # attention rows of one (sequence, KV head) group, so that the context is converted once
     G = cfg.Hq // cfg.Hkv
-    samples = [(seqs[0], i % T, (i // T) % G) for i in range(n_attn_rows)]
+    # whole (sequence, KV head) groups in order, T * G rows each, until n_attn_rows are taken
+    samples = []
+    for grp in range((n_attn_rows + T * G - 1) // (T * G)):
+        b, kvh = seqs[(grp // cfg.Hkv) % len(seqs)], grp % cfg.Hkv
+        for i in range(min(T * G, n_attn_rows - len(samples))):
+            samples.append((b, i % T, kvh * G + (i // T) % G))
     t0 = time.perf_counter()
     orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], mask, inp["k_cache"], inp["v_cache"], inp["ctx_len"],
                     1.0 / math.sqrt(cfg.D), block_table=inp.get("block_table"), block_size=cfg.block_size,
@@ -120,12 +125,16 @@ def oracle_sample(cfg, inp, n_attn_rows: int, n_lm_rows: int):
     t0 = time.perf_counter()
     W64 = orc.bf16_to_f64(inp["W"])
     t_w = time.perf_counter() - t0
-    sub = {k: inp[k][seqs[0]:seqs[0] + 1, :n_lm_rows] for k in ("h",)}
-    par = np.arange(-1, n_lm_rows - 1, dtype=np.int32)[None]
-    tok = inp["tok"][seqs[0]:seqs[0] + 1, :n_lm_rows]
-    t0 = time.perf_counter()
-    st = orc.lmhead_stats(sub["h"], inp["W"], par, tok, cfg.logit_scale, W64=W64)
-    t_lm = time.perf_counter() - t0
+    t_lm, left = 0.0, n_lm_rows
+    for b in seqs:                                  # whole sequences, then a prefix of the next one
+        n = min(T, left)
+        if n <= 0:
+            break
+        t0 = time.perf_counter()
+        st = orc.lmhead_stats(inp["h"][b:b + 1, :n], inp["W"], inp["parent"][b:b + 1, :n], inp["tok"][b:b + 1, :n],
+                              cfg.logit_scale, W64=W64)
+        t_lm += time.perf_counter() - t0
+        left -= n
     del W64
     t0 = time.perf_counter()
     p1 = np.tile(st["p_top1"][:, :1], (cfg.B, T))
@@ -146,8 +155,8 @@ def oracle_timed(cfg, inp, budget_s: float):
     est_full = n_seq * cfg.k / v
     f = min(1.0, budget_s / est_full)
     G = cfg.Hq // cfg.Hkv
-    na = max(1, min(int(f * tot_a), cfg.T * G))      # rows of one (sequence, KV head) group at most
-    nl = max(1, min(int(f * tot_l), cfg.T))
+    na = max(1, min(int(f * tot_a), tot_a))
+    nl = max(1, min(int(f * tot_l), tot_l))
     return oracle_sample(cfg, inp, n_attn_rows=na, n_lm_rows=nl)
 
 
@@ -189,11 +198,17 @@ def main():
     ap.add_argument("--workload", default="proxy_tree")
     ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override the number of sequences of the workload (reduced copies for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "trispec" else args.warmup
 
     from paper_2601_23180_b200 import inputs as gen
     cfg = gen.CONFIGS[args.workload]
+    if args.batch is not None:
+        import dataclasses as _dc
+        cfg = _dc.replace(cfg, B=args.batch, name=f"{cfg.name}[B={args.batch}]",
+                          n_active=None if cfg.n_active is None else min(cfg.n_active, args.batch))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -331,7 +346,25 @@ def main():
     n_seq = cfg.B if cfg.n_active is None else cfg.n_active
     M = n_seq * cfg.T
     lm_flops = 2.0 * M * cfg.d * cfg.V
+    lm_bytes = 2.0 * cfg.V * cfg.d + 2.0 * M * cfg.d + 40.0 * M
     lm_tflops = lm_flops / (part_ms["lmhead"] * 1e-3) / 1e12
+    lm_gbs = lm_bytes / (part_ms["lmhead"] * 1e-3) / 1e9
+    # the back-to-back loop is a sustained run when it lasts long enough for the power cap to bite
+    sustained = peaks.get("bf16_tflops_sustained") and part_ms["lmhead"] * args.steps >= 200.0
+    tc_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    lm_tensor_bound = lm_flops / (tc_peak * 1e12) >= lm_bytes / (peaks["hbm_gbs"] * 1e9)
+    if lm_tensor_bound:
+        roof = {"kernel": "lmhead_gemm_kernel", "bound": "tensor", "achieved": lm_tflops, "peak": tc_peak,
+                "unit": "TFLOP/s", "frac": lm_tflops / tc_peak,
+                "peak_source": f"{peaks['source']} {'sustained' if sustained else 'burst'} bf16 GEMM",
+                "frac_of_burst_peak": lm_tflops / peaks["bf16_tflops"],
+                "work_per_launch": lm_flops}
+    else:
+        roof = {"kernel": "lmhead_gemm_kernel", "bound": "hbm", "achieved": lm_gbs, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": lm_gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} copy bandwidth",
+                "work_per_launch": lm_bytes}
+    roof.update({"traffic": LMHEAD_GEMM_DRAM_TRAFFIC.get(cfg.name), "ms_per_launch": part_ms["lmhead"],
+                 "timed": "trispec_lmhead_stats back to back (GEMM + finalize kernel; CUDA events on the stream)"})
     Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
     attn_bytes = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 2 * 2 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
     attn_gbs = attn_bytes / (part_ms["attention"] * 1e-3) / 1e9
@@ -348,10 +381,7 @@ def main():
                 "h2d_bytes_per_step": pas.h2d_bytes, "d2h_bytes_per_step": pas.d2h_bytes},
         "gpu_launches": launches, "host_us_per_call": host_us_per_call, "pass_latency_ms_median": pass_latency_ms,
         "clocks": clocks,
-        "roofline": {"kernel": "lmhead_gemm_kernel", "bound": "tensor", "achieved": lm_tflops,
-                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": lm_tflops / peaks["bf16_tflops"],
-                     "peak_source": f"{peaks['source']} burst bf16", "traffic": LMHEAD_GEMM_DRAM_TRAFFIC.get(cfg.name),
-                     "flops_per_launch": lm_flops, "ms_per_launch": part_ms["lmhead"]},
+        "roofline": roof,
         "kernels_ms": part_ms,
         "attention_roofline": {"bound": "hbm", "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": attn_gbs / peaks["hbm_gbs"], "bytes_per_launch": attn_bytes},
