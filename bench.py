@@ -184,6 +184,139 @@ def run_reference(args, cfg, rank):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------
+# One kernel alone, L2 flushed before every launch (--only attention | lmhead | scan)
+# ---------------------------------------------------------------------------------------------
+def _roof(peaks, flops, byts, ms):
+    """Roofline record of one launch: the bound is the larger of the two lower-bound times."""
+    tensor_bound = flops / (peaks["bf16_tflops"] * 1e12) > byts / (peaks["hbm_gbs"] * 1e9)
+    r = ({"bound": "tensor", "achieved": flops / ms / 1e9, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+          "work_per_launch": flops} if tensor_bound else
+         {"bound": "hbm", "achieved": byts / ms / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+          "work_per_launch": byts})
+    r.update({"frac": r["achieved"] / r["peak"], "ms_per_launch": ms, "traffic": None,
+              "hbm_gbs": byts / ms / 1e6, "tflops": flops / ms / 1e9,
+              "peak_source": f"{peaks['source']} (burst: the kernel is timed alone)"})
+    return r
+
+
+def _scan_stress_inputs(cfg, B):
+    """2^20-sequence input of the scan kernels: the workload's tree generator (1024 distinct
+    trees, tiled), statistics synthesised on the device: the top-1 of a node is the token of
+    its first child (so that walks go on) or a random token; about a quarter of the nodes
+    fail the margin test."""
+    import numpy as np
+    import torch
+    from paper_2601_23180_b200 import inputs as gen
+    T = cfg.T
+    trees = np.stack([gen.make_tree(cfg, b) for b in range(1024)])
+    toks = np.stack([gen.make_tokens(cfg, b, trees[b]) for b in range(1024)])
+    parent = torch.from_numpy(trees).cuda().repeat(B // 1024, 1).contiguous()
+    tok = torch.from_numpy(toks.astype(np.int32)).cuda().repeat(B // 1024, 1).contiguous()
+    g = torch.Generator(device="cuda").manual_seed(cfg.seed)
+    first_child = np.full((1024, T), -1, dtype=np.int64)
+    for b in range(1024):
+        for c in range(T - 1, 0, -1):
+            first_child[b, trees[b, c]] = c
+    fc = torch.from_numpy(first_child).cuda().repeat(B // 1024, 1)
+    rnd = torch.randint(0, cfg.V, (B, T), generator=g, device="cuda", dtype=torch.int32)
+    top1 = torch.where(fc >= 0, torch.gather(tok, 1, fc.clamp(min=0)), rnd).to(torch.int32).contiguous()
+    p1 = 0.5 + 0.5 * torch.rand((B, T), generator=g, device="cuda")
+    p1 = torch.where(torch.rand((B, T), generator=g, device="cuda") < 0.15, p1 * 0.5, p1).contiguous()
+    p2 = (0.1 * torch.rand((B, T), generator=g, device="cuda")).contiguous()
+    return parent, tok, {"p_top1": p1, "p_top2": p2, "top1_idx": top1}
+
+
+def run_only(args, cfg):
+    """Times one entry point by itself: every call bracketed by CUDA events on its stream, a
+    buffer larger than L2 zeroed before each call; prints one JSON line with that kernel's
+    roofline. `scan` runs the scan-only stress input (2^20 sequences), where HBM, not launch
+    latency, bounds the integer kernels."""
+    import dataclasses
+    import numpy as np
+    import torch
+    from paper_2601_23180_b200 import binding as ts
+    from paper_2601_23180_b200 import inputs as gen
+    from paper_2601_23180_b200 import runner
+    torch.cuda.set_device(0)
+    peaks = _peaks()
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    n = max(3, min(args.steps, 200))
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for s_, e_ in evs:
+            flush.zero_()
+            s_.record(stream)
+            fn()
+            e_.record(stream)
+        torch.cuda.synchronize()
+        return statistics.median(s_.elapsed_time(e_) for s_, e_ in evs)
+
+    out = {"only": args.only, "metric": METRIC, "unit": UNIT, "n_gpus": 1, "steps": n, "data": "synthetic",
+           "config": {"workload": cfg.name, "l2": "256 MB buffer zeroed before every timed call"}}
+    n_seq = cfg.B if cfg.n_active is None else cfg.n_active
+    if args.only == "scan":
+        B, T = 1 << 20, cfg.T
+        parent, tok, stats = _scan_stress_inputs(cfg, B)
+        so = ts.alloc_scan_out(B, T)
+        sa = ts.scan_args(stats, parent, tok, cfg.lam, gen.MODE_PROXY, so)
+        so_nc = {k: v for k, v in so.items() if k not in ("esc_index", "n_escalated")}
+        sa_nc = ts.scan_args(stats, parent, tok, cfg.lam, gen.MODE_PROXY, so_nc)
+        mask = torch.zeros((B, T), dtype=torch.int64, device="cuda")
+        depth = torch.zeros((B, T), dtype=torch.int32, device="cuda")
+        ta = ts.tree_args(parent, mask, depth)
+        ms_both = timed(lambda: ts.trispec_accept_scan(sa))
+        ms_scan = timed(lambda: ts.trispec_accept_scan(sa_nc))
+        ms_mask = timed(lambda: ts.trispec_build_tree_mask(ta))
+        # per sequence: parent, tok, top1_idx, p_top1, p_top2 (4 B per node, each read once); outputs: path
+        # (4 B per node), accept_len, bonus, last_node, near_thr (4 B each), escalate (1 B); the compaction
+        # adds 1 B read and 4 B written per sequence; the mask kernel reads 4 B and writes 12 B per node
+        scan_bytes, compact_bytes, mask_bytes = B * (T * 24 + 17), B * 5, B * T * 16
+        hb = peaks["hbm_gbs"]
+        out.update({
+            "config": {"workload": f"scan stress: 2^20 sequences of the {cfg.name} tree shape", "T": T,
+                       "mean_accept_len": so["accept_len"].float().mean().item(),
+                       "escalated": int(so["n_escalated"].item()), "l2": out["config"]["l2"]},
+            "value": B * cfg.k / (ms_scan * 1e-3), "ms_per_step": ms_scan, "dtype": "int32",
+            "roofline": {"kernel": "accept_scan_kernel", "bound": "hbm", "achieved": scan_bytes / ms_scan / 1e6,
+                         "peak": hb, "unit": "GB/s", "frac": scan_bytes / ms_scan / 1e6 / hb,
+                         "work_per_launch": scan_bytes, "ms_per_launch": ms_scan, "traffic": None},
+            "scan_with_compaction": {"kernel": "accept_scan_kernel + esc_compact_kernel (one block)", "ms": ms_both,
+                                     "achieved": (scan_bytes + compact_bytes) / ms_both / 1e6, "unit": "GB/s",
+                                     "frac": (scan_bytes + compact_bytes) / ms_both / 1e6 / hb},
+            "tree_mask_roofline": {"kernel": "tree_mask_kernel", "bound": "hbm", "achieved": mask_bytes / ms_mask / 1e6,
+                                   "peak": hb, "unit": "GB/s", "frac": mask_bytes / ms_mask / 1e6 / hb,
+                                   "work_per_launch": mask_bytes, "ms_per_launch": ms_mask}})
+        print(json.dumps(out), flush=True)
+        return
+    if args.only == "attention":
+        inp = gen.make_inputs(cfg, with_lm_head=False)
+        small = dataclasses.replace(cfg, V=4096, d=64)      # the LM head is not run: a token-sized stand-in
+        inp.update({k: v for k, v in gen.make_inputs(small, with_attention=False).items() if k in ("h", "W")})
+        pas = runner.VerifyPass(small, inp)
+        ms = timed(lambda: ts.trispec_verify_attn(pas.attn_args))
+        Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
+        byts = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 4 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
+        flops = 4.0 * cfg.T * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
+        roof = _roof(peaks, flops, byts, ms)
+        roof["kernel"] = "verify_attn_split_kernel"
+    else:
+        inp = gen.make_inputs(cfg, with_attention=False)
+        pas = runner.VerifyPass(cfg, inp, with_attention=False)
+        ms = timed(lambda: ts.trispec_lmhead_stats(pas.lm_args))
+        M = n_seq * cfg.T
+        roof = _roof(peaks, 2.0 * M * cfg.d * cfg.V, 2.0 * cfg.V * cfg.d + 2.0 * M * cfg.d + 40.0 * M, ms)
+        roof["kernel"] = "lmhead_gemm_kernel (+ finalize)"
+        roof["traffic"] = LMHEAD_GEMM_DRAM_TRAFFIC.get(cfg.name)
+    assert int(pas.status.item()) == 0, "a device-side wait timed out"
+    out.update({"value": n_seq * cfg.k / (ms * 1e-3), "ms_per_step": ms, "dtype": "bf16", "roofline": roof})
+    print(json.dumps(out), flush=True)
+
+
 def cfg_tokens(cfg):
     n = cfg.B if cfg.n_active is None else cfg.n_active
     return n * cfg.k
@@ -198,6 +331,8 @@ def main():
     ap.add_argument("--workload", default="proxy_tree")
     ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan"],
+                    help="time one entry point alone (L2 flushed before each call) instead of the pass")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the number of sequences of the workload (reduced copies for profiler captures)")
     args = ap.parse_args()
@@ -215,6 +350,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, cfg, rank)
+        return
+    if args.only is not None:
+        if rank == 0:
+            run_only(args, cfg)
         return
 
     import numpy as np

@@ -1,8 +1,12 @@
 // Acceptance scan: greedy acceptance (Eq. 6), acceptance length tau_a (Eq. 7), margin
 // predicate (Eq. 8), trusted prefix tau_m (Eq. 9) and the routing cases (i)/(ii)
 // (Algorithm 1), evaluated along the path the greedy matches select in the draft tree.
-// One warp per sequence: each lane keeps two tree nodes in registers, the child match is a
-// warp ballot. A second single-block kernel compacts the escalated sequence ids in order.
+// One warp per sequence. Each lane loads nodes `lane` and `lane + 32` of every per-node
+// array once, coalesced (parent, token, top-1 index, the two probabilities); the margin test
+// of all nodes becomes two ballots, and the walk then runs on registers: the current node's
+// top-1 comes from a warp shuffle, the child match is a warp ballot. The accepted path is
+// collected in registers and stored as one row. A second kernel compacts the escalated
+// sequence ids in order.
 #include "host_common.h"
 
 namespace trispec {
@@ -19,35 +23,62 @@ accept_scan_kernel(trispec_scan_args a) {
   const int T = a.T;
   const long long base = b * T;
   int32_t* path = a.path + base;
+  const bool has0 = lane < T, has1 = lane + 32 < T;
 
   if (a.active && a.active[b] == 0) {
-    if (lane < T) path[lane] = -1;
-    if (lane + 32 < T) path[lane + 32] = -1;
+    if (has0) path[lane] = -1;
+    if (has1) path[lane + 32] = -1;
     if (lane == 0) {
       a.accept_len[b] = 0;
       a.escalate[b] = 0;
       a.bonus_tok[b] = -1;
       a.last_node[b] = -1;
       if (a.near_thr) a.near_thr[b] = 0;
+      if (a.esc_index) a.esc_index[b] = -1;
     }
     return;
   }
 
   // nodes `lane` and `lane + 32` of this sequence
-  int par0 = -2, par1 = -2, tok0 = 0, tok1 = 0;
-  if (lane < T) { par0 = __ldg(a.parent + base + lane); tok0 = __ldg(a.tok + base + lane); }
-  if (lane + 32 < T) { par1 = __ldg(a.parent + base + lane + 32); tok1 = __ldg(a.tok + base + lane + 32); }
+  const bool proxy = (a.mode == TRISPEC_MODE_PROXY);
+  int par0 = -2, par1 = -2, tok0 = 0, tok1 = 0, top0 = -1, top1v = -1;
+  bool tr0 = true, tr1 = true, nr0 = false, nr1 = false;   // margin >= lambda / within 1e-3 of it
+  if (has0) {
+    par0 = __ldg(a.parent + base + lane); tok0 = __ldg(a.tok + base + lane);
+    top0 = __ldg(a.in.top1_idx + base + lane);
+    if (proxy) {
+      const float mg = __ldg(a.in.p_top1 + base + lane) - __ldg(a.in.p_top2 + base + lane);
+      tr0 = mg >= a.lambda; nr0 = fabsf(mg - a.lambda) < 1e-3f;
+    }
+  }
+  if (has1) {
+    par1 = __ldg(a.parent + base + lane + 32); tok1 = __ldg(a.tok + base + lane + 32);
+    top1v = __ldg(a.in.top1_idx + base + lane + 32);
+    if (proxy) {
+      const float mg = __ldg(a.in.p_top1 + base + lane + 32) - __ldg(a.in.p_top2 + base + lane + 32);
+      tr1 = mg >= a.lambda; nr1 = fabsf(mg - a.lambda) < 1e-3f;
+    }
+  }
+  // the margin test of every node as one bit (Eq. 8), known to the whole warp
+  const unsigned long long trusted =
+      __ballot_sync(0xffffffffu, tr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, tr1)) << 32);
+  const unsigned long long near_bits =
+      __ballot_sync(0xffffffffu, nr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, nr1)) << 32);
+  // the compaction kernel only writes the leading entries of esc_index
+  if (a.esc_index && lane == 0) a.esc_index[b] = -1;
 
   int cur = a.start_node ? a.start_node[b] : 0;
   if (cur < 0 || cur >= T) cur = 0;
   int n = 0, esc = 0, bonus = -1, near = 0;
+  int path0 = -1, path1 = -1;   // entries `lane` and `lane + 32` of the accepted path
   // each accepted node has a larger index than the previous one: at most T iterations
   for (int it = 0; it < T; ++it) {
-    const int top1 = __ldg(a.in.top1_idx + base + cur);
-    if (a.mode == TRISPEC_MODE_PROXY) {
-      const float margin = __ldg(a.in.p_top1 + base + cur) - __ldg(a.in.p_top2 + base + cur);
-      if (fabsf(margin - a.lambda) < 1e-3f) ++near;
-      if (!(margin >= a.lambda)) { esc = 1; break; }
+    const int src = cur & 31;
+    const int t_lo = __shfl_sync(0xffffffffu, top0, src), t_hi = __shfl_sync(0xffffffffu, top1v, src);
+    const int top1 = (cur < 32) ? t_lo : t_hi;
+    if (proxy) {
+      near += static_cast<int>((near_bits >> cur) & 1ull);
+      if (!((trusted >> cur) & 1ull)) { esc = 1; break; }
     }
     const unsigned m0 = __ballot_sync(0xffffffffu, par0 == cur && tok0 == top1);
     const unsigned m1 = __ballot_sync(0xffffffffu, par1 == cur && tok1 == top1);
@@ -55,12 +86,13 @@ accept_scan_kernel(trispec_scan_args a) {
     if (m0) nxt = __ffs(m0) - 1;
     else if (m1) nxt = 32 + __ffs(m1) - 1;
     if (nxt < 0) { bonus = top1; break; }
-    if (lane == 0) path[n] = nxt;
+    if (lane == n) path0 = nxt;
+    if (lane + 32 == n) path1 = nxt;
     ++n;
     cur = nxt;
   }
-  if (lane >= n && lane < T) path[lane] = -1;
-  if (lane + 32 >= n && lane + 32 < T) path[lane + 32] = -1;
+  if (has0) path[lane] = path0;
+  if (has1) path[lane + 32] = path1;
   if (lane == 0) {
     a.accept_len[b] = n;
     a.escalate[b] = static_cast<uint8_t>(esc);
@@ -70,54 +102,83 @@ accept_scan_kernel(trispec_scan_args a) {
   }
 }
 
-// Ordered compaction of the escalated sequence ids: one block, 16 flags per thread per round.
+// Ordered compaction of the escalated sequence ids by one block. Per round a warp owns 2048
+// consecutive flags: lane l reads the 4-byte words l, l + 32, ... of them (coalesced), the
+// block orders the warp totals with one barrier (double-buffered; the running total is carried
+// in registers), and each word column is scattered with a warp scan, so that a warp writes
+// consecutive entries of esc_index. Entries past the last escalated sequence were set to -1 by
+// the scan kernel. 65536 flags per round.
 constexpr int kCompactThreads = 1024;
+constexpr int kCompactWords = 16;                       // 4-byte words per lane and round
+constexpr int kCompactPerWarp = 32 * kCompactWords * 4;  // flags per warp and round
 __global__ void __launch_bounds__(kCompactThreads)
 esc_compact_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restrict__ esc_index,
                    int32_t* __restrict__ n_escalated) {
-  __shared__ int warp_excl[32];
-  __shared__ int running;
+  __shared__ int warp_total[2][32];
   pdl_launch_dependents();
   pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) running = 0;
-  __syncthreads();
-  for (long long start = 0; start < B; start += static_cast<long long>(kCompactThreads) * 16) {
-    const long long first = start + static_cast<long long>(tid) * 16;
-    unsigned bits = 0;
-    for (int j = 0; j < 16; ++j) {
-      long long s = first + j;
-      if (s < B && escalate[s]) bits |= (1u << j);
-    }
-    const int cnt = __popc(bits);
-    int incl = cnt;  // inclusive prefix inside the warp
-    for (int o = 1; o < 32; o <<= 1) {
-      int v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_excl[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      const int w = warp_excl[lane];
-      int wi = w;
-      for (int o = 1; o < 32; o <<= 1) {
-        int v = __shfl_up_sync(0xffffffffu, wi, o);
-        if (lane >= o) wi += v;
+  const bool word_ok = (reinterpret_cast<uintptr_t>(escalate) & 3u) == 0;
+  int running = 0;      // escalated sequences in earlier rounds (same value in every thread)
+  int round = 0;
+  for (long long start = 0; start < B; start += static_cast<long long>(kCompactThreads / 32) * kCompactPerWarp, ++round) {
+    const long long region = start + static_cast<long long>(warp) * kCompactPerWarp;
+    uint32_t w[kCompactWords];
+    int cnt = 0;
+    if (word_ok && region + kCompactPerWarp <= B) {
+      // whole region in range: sixteen independent coalesced loads in flight
+#pragma unroll
+      for (int j = 0; j < kCompactWords; ++j)
+        w[j] = __ldg(reinterpret_cast<const uint32_t*>(escalate + region) + j * 32 + lane);
+    } else {
+#pragma unroll
+      for (int j = 0; j < kCompactWords; ++j) {
+        const long long first = region + (j * 32 + lane) * 4;
+        uint32_t x = 0;
+        for (int k = 0; k < 4; ++k)
+          if (first + k < B) x |= static_cast<uint32_t>(escalate[first + k]) << (8 * k);
+        w[j] = x;
       }
-      warp_excl[lane] = wi - w;  // exclusive prefix of the warp totals
     }
+#pragma unroll
+    for (int j = 0; j < kCompactWords; ++j) {
+      w[j] = __vcmpne4(w[j], 0u) & 0x01010101u;        // one bit per non-zero flag byte
+      cnt += __popc(w[j]);
+    }
+    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);   // warp total
+    if (lane == 0) warp_total[round & 1][warp] = cnt;
     __syncthreads();
-    const int off = running + warp_excl[warp] + (incl - cnt);
-    int k = 0;
-    for (int j = 0; j < 16; ++j)
-      if (bits & (1u << j)) esc_index[off + (k++)] = static_cast<int32_t>(first + j);
-    __syncthreads();                                   // everyone has read `running`
-    if (tid == kCompactThreads - 1) running = off + cnt;  // last thread: total so far
-    __syncthreads();
+    // every warp scans the 32 warp totals itself
+    const int wt = warp_total[round & 1][lane];
+    int wincl = wt;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, wincl, o);
+      if (lane >= o) wincl += v;
+    }
+    int off = running + __shfl_sync(0xffffffffu, wincl - wt, warp);
+    running += __shfl_sync(0xffffffffu, wincl, 31);
+    if (cnt) {
+#pragma unroll
+      for (int j = 0; j < kCompactWords; ++j) {
+        const int c = __popc(w[j]);
+        int incl = c;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        int dst = off + incl - c;
+        uint32_t x = w[j];
+        while (x) {
+          const int bit = __ffs(x) - 1;
+          x &= x - 1;
+          esc_index[dst++] = static_cast<int32_t>(region + (j * 32 + lane) * 4 + (bit >> 3));
+        }
+        off += __shfl_sync(0xffffffffu, incl, 31);
+      }
+    }
   }
-  const int total = running;
-  for (long long s = static_cast<long long>(total) + tid; s < B; s += kCompactThreads) esc_index[s] = -1;
-  if (tid == 0) *n_escalated = total;
+  // entries past the last escalated sequence already hold -1 (written by the scan kernel)
+  if (tid == 0) *n_escalated = running;
 }
 
 }  // namespace trispec
