@@ -17,6 +17,10 @@ What each function follows:
                    predicate g (Eq. 8), trusted prefix tau_m (Eq. 9) and the routing cases
                    (i)/(ii) of "Adaptive Verification Routing" / Algorithm 1; TARGET mode is
                    the "standard left-to-right acceptance rule" applied after Eq. 10.
+  prune_tree       token pruning of routing case (ii) ("prune these tokens from the draft tree
+                   and pass the remaining branches to the target"; ablation on token pruning).
+  commit_kv        X <- X + Y of Algorithm 1 as the KV cache sees it: the keys/values of the
+                   last committed token and of the accepted draft tokens are appended.
 
 Readings of the paper taken here (the paper states the rule for a chain of k tokens):
   * Tree rule = the chain rule applied along the path the greedy matches select; the margin
@@ -272,3 +276,79 @@ def verify(inp: Dict[str, np.ndarray], scale: float, logit_scale: float, lam: fl
     out["scan"] = accept_scan(st["p_top1"], st["p_top2"], st["top1_idx"], parent, tok, lam,
                               mode=mode, active=active)
     return out
+
+
+# ----------------------------------------------------------------------------------------
+# token pruning (routing case (ii): "prune these tokens from the draft tree and pass the
+# remaining branches to the target"; ablation "Token pruning strategies")
+# ----------------------------------------------------------------------------------------
+def prune_tree(parent: np.ndarray, tok: np.ndarray, root: np.ndarray) -> Dict[str, np.ndarray]:
+    """The branches that remain after the proxy accepted a prefix: the subtree below the last
+    accepted node root[b] (that node becomes node 0 of the new tree: it is the last committed
+    token of the next verifier). Nodes keep their relative order, so parent'[i] < i still holds.
+
+    Outputs, all padded to the input width T: n_keep [B]; node_map [B][T] (new index -> old
+    index, -1 beyond n_keep); parent' and tok' [B][T] (-1 beyond n_keep; parent'[0] = -1).
+    root[b] < 0 (sequence not escalated) gives n_keep 0 and all -1.
+    Reading: "remaining branches" = descendants of the last accepted node; every other branch
+    contradicts the accepted prefix."""
+    parent = np.asarray(parent)
+    B, T = parent.shape
+    out = {"n_keep": np.zeros(B, dtype=np.int32), "node_map": np.full((B, T), -1, dtype=np.int32),
+           "parent": np.full((B, T), -1, dtype=np.int32), "tok": np.full((B, T), -1, dtype=np.int32)}
+    for b in range(B):
+        r = int(root[b])
+        if r < 0:
+            continue
+        new_of = {}
+        for i in range(T):
+            # i is kept iff walking up from i meets r
+            p = i
+            while p >= 0 and p != r:
+                p = int(parent[b, p])
+            if p == r:
+                new_of[i] = len(new_of)
+        for i, j in new_of.items():
+            out["node_map"][b, j] = i
+            out["tok"][b, j] = tok[b, i]
+            out["parent"][b, j] = -1 if i == r else new_of[int(parent[b, i])]
+        out["n_keep"][b] = len(new_of)
+    return out
+
+
+# ----------------------------------------------------------------------------------------
+# KV commit of the accepted path (the step after a verification round in the decode loop:
+# X <- X + Y of Algorithm 1 seen from the KV cache)
+# ----------------------------------------------------------------------------------------
+def commit_kv(k_cache: np.ndarray, v_cache: np.ndarray, ctx_len: np.ndarray, k_tree: np.ndarray,
+              v_tree: np.ndarray, path: np.ndarray, accept_len: np.ndarray,
+              block_table: Optional[np.ndarray] = None, block_size: int = 64,
+              active: Optional[np.ndarray] = None):
+    """Appends to each sequence's cache the keys/values of tree node 0 (the last committed token,
+    whose K/V were not in the cache yet) and of the accept_len[b] accepted nodes path[b][:n], in
+    that order, at positions ctx_len[b], ctx_len[b] + 1, ...; returns (k_cache', v_cache',
+    ctx_len') as new arrays. Layouts as in verify_attn (contiguous [B][L][Hkv][D] or paged pool
+    + block_table). A sequence whose new length would exceed its capacity is left unchanged."""
+    kc, vc = np.array(k_cache, copy=True), np.array(v_cache, copy=True)
+    new_len = np.array(ctx_len, dtype=np.int32, copy=True)
+    B = k_tree.shape[0]
+    for b in range(B):
+        if active is not None and not active[b]:
+            continue
+        n = int(accept_len[b])
+        nodes = [0] + [int(path[b, j]) for j in range(n)]
+        L = int(ctx_len[b])
+        cap = kc.shape[1] if block_table is None else int((np.asarray(block_table[b]) >= 0).sum()) * block_size
+        if L + len(nodes) > cap:
+            continue
+        for j, node in enumerate(nodes):
+            t = L + j
+            if block_table is None:
+                kc[b, t] = k_tree[b, node]
+                vc[b, t] = v_tree[b, node]
+            else:
+                blk = int(block_table[b, t // block_size])
+                kc[blk, t % block_size] = k_tree[b, node]
+                vc[blk, t % block_size] = v_tree[b, node]
+        new_len[b] = L + len(nodes)
+    return kc, vc, new_len

@@ -1,0 +1,207 @@
+"""Pins of the oracle's token pruning and KV commit (CPU only): hand-derived cases, special
+cases that reduce to the identity or to a plain slice, invariants that tie them to the tree mask
+and to the attention oracle, and brute force on small random trees."""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import trispec_oracle as orc
+from paper_2601_23180_b200 import inputs as gen
+
+
+def _cfg(**kw):
+    return gen.small_variant(gen.CONFIGS["proxy_tree"], **kw)
+
+
+# ------------------------------------------------------------------------------ pruning
+def test_prune_hand_case():
+    # routing case (ii): the subtree below the last accepted node remains. Tree (node: parent)
+    # 0:-1 1:0 2:0 3:1 4:1 5:2 6:3 ; accepted up to node 1 -> nodes {1,3,4,6} remain, relabelled 0..3
+    parent = np.array([[-1, 0, 0, 1, 1, 2, 3]], dtype=np.int32)
+    tok = np.array([[10, 11, 12, 13, 14, 15, 16]], dtype=np.int32)
+    r = orc.prune_tree(parent, tok, np.array([1]))
+    assert r["n_keep"][0] == 4
+    assert r["node_map"][0].tolist() == [1, 3, 4, 6, -1, -1, -1]
+    assert r["parent"][0].tolist() == [-1, 0, 0, 1, -1, -1, -1]
+    assert r["tok"][0].tolist() == [11, 13, 14, 16, -1, -1, -1]
+
+
+def test_prune_at_root_is_identity_at_leaf_is_single_node_and_skip():
+    cfg = _cfg(B=3)
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(3)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(3)])
+    T = cfg.T
+    leaf = max(i for i in range(T) if not (parent[1] == i).any())
+    r = orc.prune_tree(parent, tok, np.array([0, leaf, -1]))
+    assert r["n_keep"].tolist() == [T, 1, 0]
+    assert np.array_equal(r["parent"][0], parent[0]) and np.array_equal(r["tok"][0], tok[0])
+    assert np.array_equal(r["node_map"][0], np.arange(T))
+    assert r["node_map"][1, 0] == leaf and r["parent"][1, 0] == -1 and (r["node_map"][1, 1:] == -1).all()
+    assert (r["node_map"][2] == -1).all() and (r["parent"][2] == -1).all()
+
+
+def test_prune_chain_is_a_suffix():
+    T = 9
+    parent = np.arange(-1, T - 1, dtype=np.int32)[None]
+    tok = np.arange(100, 100 + T, dtype=np.int32)[None]
+    for j in range(T):
+        r = orc.prune_tree(parent, tok, np.array([j]))
+        n = T - j
+        assert r["n_keep"][0] == n
+        assert r["tok"][0, :n].tolist() == list(range(100 + j, 100 + T))
+        assert r["parent"][0, :n].tolist() == list(range(-1, n - 1))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_prune_agrees_with_tree_mask_and_subtree_counts(seed):
+    """Independent route: membership through the mask bits (bit r of mask[i]), sizes through a
+    bottom-up child count; the pruned tree's own mask is the old mask with the kept bits packed."""
+    cfg = _cfg(B=4, seed=seed)
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(4)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(4)])
+    T = cfg.T
+    mask, depth = orc.build_tree_mask(parent)
+    g = np.random.default_rng(seed)
+    root = g.integers(0, T, size=4)
+    r = orc.prune_tree(parent, tok, root)
+    for b in range(4):
+        size = np.ones(T, dtype=int)
+        for i in range(T - 1, 0, -1):
+            size[parent[b, i]] += size[i]
+        keep = [i for i in range(T) if (int(mask[b, i]) >> int(root[b])) & 1]
+        assert r["n_keep"][b] == size[root[b]] == len(keep)
+        assert r["node_map"][b, :len(keep)].tolist() == keep
+        # valid tree: parents precede children, one root
+        pp = r["parent"][b, :len(keep)]
+        assert pp[0] == -1 and all(0 <= pp[j] < j for j in range(1, len(keep)))
+        # mask of the pruned tree = packed bits of the old mask restricted to kept nodes
+        new_mask, new_depth = orc.build_tree_mask(pp[None])
+        for j, i in enumerate(keep):
+            packed = 0
+            for jj, ii in enumerate(keep):
+                if (int(mask[b, i]) >> ii) & 1:
+                    packed |= 1 << jj
+            assert int(new_mask[0, j]) == packed
+            assert new_depth[0, j] == depth[b, i] - depth[b, root[b]]
+
+
+def test_prune_then_target_scan_continues_the_proxy_walk():
+    """A TARGET-mode scan of the pruned tree from its node 0 accepts exactly what a TARGET-mode
+    scan of the unpruned tree accepts from start_node = last accepted node (the w/ and w/o token
+    pruning variants verify the same remaining tokens)."""
+    cfg = _cfg(B=6, seed=3)
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(6)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(6)])
+    T = cfg.T
+    g = np.random.default_rng(5)
+    root = g.integers(0, T // 3, size=6).astype(np.int32)
+    # target top-1: first child's token on most nodes, so that walks go on
+    top1 = g.integers(0, cfg.V, size=(6, T))
+    for b in range(6):
+        for i in range(T):
+            kids = np.nonzero(parent[b] == i)[0]
+            if len(kids) and g.random() < 0.8:
+                top1[b, i] = tok[b, kids[0]]
+    full = orc.accept_scan(np.ones((6, T)), np.zeros((6, T)), top1, parent, tok, 0.5, mode=orc.MODE_TARGET,
+                           start_node=root)
+    pr = orc.prune_tree(parent, tok, root)
+    top1_p = np.zeros((6, T), dtype=np.int64)
+    for b in range(6):
+        n = pr["n_keep"][b]
+        top1_p[b, :n] = top1[b, pr["node_map"][b, :n]]
+    pruned = orc.accept_scan(np.ones((6, T)), np.zeros((6, T)), top1_p, pr["parent"], pr["tok"], 0.5,
+                             mode=orc.MODE_TARGET)
+    for b in range(6):
+        n = full["accept_len"][b]
+        assert pruned["accept_len"][b] == n and pruned["bonus_tok"][b] == full["bonus_tok"][b]
+        assert [pr["node_map"][b, j] for j in pruned["path"][b, :n]] == full["path"][b, :n].tolist()
+
+
+# ------------------------------------------------------------------------------ KV commit
+def _kv_case(paged: bool, B=3, L=100, seed=0):
+    name = "long_paged" if paged else "proxy_tree"
+    cfg = gen.small_variant(gen.CONFIGS[name], B=B, L=L + 64, L_min=(L + 64) if paged else None, Hq=4, Hkv=2, seed=seed)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    inp["ctx_len"] = np.array([L, L - 37, 5][:B], dtype=np.int32)
+    return cfg, inp
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_commit_appends_root_and_path_rows_and_touches_nothing_else(paged):
+    cfg, inp = _kv_case(paged)
+    B, T = cfg.B, cfg.T
+    path = np.full((B, T), -1, dtype=np.int32)
+    path[0, :3] = [2, 7, 19]
+    path[1, :1] = [1]
+    acc = np.array([3, 1, 0], dtype=np.int32)
+    kc, vc, nl = orc.commit_kv(inp["k_cache"], inp["v_cache"], inp["ctx_len"], inp["k_tree"], inp["v_tree"], path,
+                               acc, block_table=inp.get("block_table"), block_size=cfg.block_size)
+    assert nl.tolist() == [int(inp["ctx_len"][b]) + int(acc[b]) + 1 for b in range(B)]
+
+    def row(cache, b, t):
+        if not paged:
+            return cache[b, t]
+        return cache[inp["block_table"][b, t // cfg.block_size], t % cfg.block_size]
+    changed = np.zeros(kc.shape[:2], dtype=bool)
+    for b in range(B):
+        L = int(inp["ctx_len"][b])
+        nodes = [0] + path[b, :acc[b]].tolist()
+        for j, node in enumerate(nodes):
+            assert np.array_equal(row(kc, b, L + j), inp["k_tree"][b, node])
+            assert np.array_equal(row(vc, b, L + j), inp["v_tree"][b, node])
+            if paged:
+                changed[inp["block_table"][b, (L + j) // cfg.block_size], (L + j) % cfg.block_size] = True
+            else:
+                changed[b, L + j] = True
+    assert np.array_equal(kc[~changed], inp["k_cache"][~changed])
+    assert np.array_equal(vc[~changed], inp["v_cache"][~changed])
+
+
+def test_commit_paged_equals_contiguous_through_attention():
+    """After a commit, attention of a fresh one-node tree over the longer context must equal
+    attention over [old context + committed rows] assembled by hand (ties commit_kv to verify_attn)."""
+    cfg, inp = _kv_case(False, B=2, L=70, seed=2)
+    B, T = cfg.B, cfg.T
+    inp["ctx_len"] = np.array([70, 33], dtype=np.int32)
+    path = np.full((B, T), -1, dtype=np.int32)
+    path[0, :2] = [1, 5]
+    acc = np.array([2, 0], dtype=np.int32)
+    kc, vc, nl = orc.commit_kv(inp["k_cache"], inp["v_cache"], inp["ctx_len"], inp["k_tree"], inp["v_tree"], path, acc)
+    # by hand: concatenate
+    for b in range(B):
+        L = int(inp["ctx_len"][b])
+        nodes = [0] + path[b, :acc[b]].tolist()
+        hand_k = np.concatenate([inp["k_cache"][b, :L], inp["k_tree"][b, nodes]], axis=0)
+        hand_v = np.concatenate([inp["v_cache"][b, :L], inp["v_tree"][b, nodes]], axis=0)
+        assert np.array_equal(kc[b, :nl[b]], hand_k) and np.array_equal(vc[b, :nl[b]], hand_v)
+    q1 = inp["q"][:, :1]
+    kt1, vt1 = inp["k_tree"][:, :1], inp["v_tree"][:, :1]
+    m1 = np.ones((B, 1), dtype=np.uint64)
+    o_new, _ = orc.verify_attn(q1, kt1, vt1, m1, kc, vc, nl, 0.1)
+    # the same keys presented as [context | tree chain]: a chain tree whose last node is the query
+    for b in range(B):
+        n = int(acc[b]) + 1
+        nodes = [0] + path[b, :acc[b]].tolist()
+        ktc = np.concatenate([inp["k_tree"][b, nodes], kt1[b]], axis=0)[None]
+        vtc = np.concatenate([inp["v_tree"][b, nodes], vt1[b]], axis=0)[None]
+        qc = np.concatenate([inp["q"][b, nodes], q1[b]], axis=0)[None]
+        chain_parent = np.arange(-1, n, dtype=np.int32)[None]
+        mc, _ = orc.build_tree_mask(chain_parent)
+        o_chain, _ = orc.verify_attn(qc, ktc, vtc, mc, inp["k_cache"][b:b + 1], inp["v_cache"][b:b + 1],
+                                     inp["ctx_len"][b:b + 1], 0.1)
+        assert np.allclose(o_new[b, 0], o_chain[0, n], rtol=0, atol=1e-12)
+
+
+def test_commit_respects_capacity_and_active():
+    cfg, inp = _kv_case(False, B=3, L=100)
+    B, T = cfg.B, cfg.T
+    Lcap = inp["k_cache"].shape[1]
+    inp["ctx_len"] = np.array([Lcap - 1, Lcap - 2, 10], dtype=np.int32)
+    path = np.full((B, T), -1, dtype=np.int32)
+    path[:, 0] = 1
+    acc = np.array([1, 1, 1], dtype=np.int32)          # needs 2 rows each
+    kc, vc, nl = orc.commit_kv(inp["k_cache"], inp["v_cache"], inp["ctx_len"], inp["k_tree"], inp["v_tree"], path,
+                               acc, active=np.array([1, 1, 0], dtype=np.uint8))
+    assert nl.tolist() == [Lcap - 1, Lcap, 10]          # 0: no room, 1: fits exactly, 2: inactive
+    assert np.array_equal(kc[0], inp["k_cache"][0]) and np.array_equal(kc[2], inp["k_cache"][2])
