@@ -13,6 +13,10 @@
  *   4. trispec_accept_scan      acceptance length tau_a (Eq. 7), trusted prefix tau_m (Eq. 9)
  *                               and routing: approve or escalate (cases (i)/(ii), Algorithm 1)
  *   trispec_verify              the four in order on one stream.
+ * Around the pass, for the decode loop:
+ *   5. trispec_prune_tree       the branches that remain for the target after the proxy
+ *                               accepted a prefix (routing case (ii), token pruning)
+ *   6. trispec_commit_kv        append the accepted path's keys/values to the KV cache
  *
  * Conventions
  *   - Every data pointer is a DEVICE pointer owned by the caller unless a comment says
@@ -197,6 +201,63 @@ typedef struct {
   uint8_t* escalate;
 } trispec_scan_args;
 int trispec_accept_scan(const trispec_scan_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 5. Token pruning (routing case (ii): the accepted tokens are pruned from the draft tree and
+ *    the remaining branches go to the target; ablation "Token pruning strategies").
+ *    For every sequence with root[b] >= 0 the subtree below node root[b] (the last node the
+ *    proxy accepted, `last_node` of the scan) is compacted into a tree of its own: root[b]
+ *    becomes node 0, the other kept nodes follow in their old order, so parent'[i] < i holds.
+ *      parent, tok [B][T] int32, mask [B][T] uint64 (from trispec_build_tree_mask): inputs.
+ *      root [B] int32: node to keep the subtree of; < 0 = skip the sequence (n_keep 0).
+ *      n_keep [B] int32: size of the subtree.
+ *      node_map [B][T] int32: new index -> old index (the gather list for per-node data of
+ *        the old tree), -1 beyond n_keep.
+ *      parent_out, tok_out [B][T] int32: the pruned tree, -1 beyond n_keep.
+ *      mask_out [B][T] uint64, depth_out [B][T] int32 (either may be NULL): ancestor mask and
+ *        depth of the pruned tree (what trispec_build_tree_mask would give for parent_out);
+ *        entries beyond n_keep are 0 and -1.
+ *    Outputs may not alias inputs.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int B, T;
+  const int32_t *parent, *tok;
+  const uint64_t* mask;
+  const int32_t* root;
+  int32_t *n_keep, *node_map, *parent_out, *tok_out;
+  uint64_t* mask_out;
+  int32_t* depth_out;
+} trispec_prune_args;
+int trispec_prune_tree(const trispec_prune_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 6. KV commit (X <- X + Y of Algorithm 1 as the KV cache sees it). Appends, for every
+ *    active sequence, the keys/values of tree node 0 (the last committed token, not in the
+ *    cache yet) and of the accept_len[b] accepted nodes path[b][0..accept_len[b]) to the
+ *    sequence's cache at positions ctx_len[b], ctx_len[b] + 1, ..., and writes the new length.
+ *      k_tree, v_tree [B][T][Hkv][D] bf16; path [B][T], accept_len [B] (outputs of the scan).
+ *      k_cache, v_cache: the cache to append to, layouts as in trispec_verify_attn
+ *        (contiguous [B][Lmax][Hkv][D], or paged pool + block_table).
+ *      ctx_len [B] int32: current lengths; ctx_len_out [B] int32: lengths after the commit
+ *        (may be the same pointer as ctx_len: updated in place).
+ *      active (optional uint8 [B]): 0 = leave the sequence alone.
+ *    A sequence whose new length would exceed its capacity (Lmax, or 64 x the number of
+ *    non-negative entries at the head of its block_table row) is left unchanged and
+ *    dev_status (optional) receives 9. D = 128 only.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int B, T, Hkv, D;
+  const void *k_tree, *v_tree;
+  int kv_layout;
+  void *k_cache, *v_cache;
+  int Lmax, num_blocks, block_size, max_blocks_per_seq;
+  const int32_t* block_table;
+  const int32_t *ctx_len, *path, *accept_len;
+  const uint8_t* active;
+  int32_t* ctx_len_out;
+  int32_t* dev_status;
+} trispec_commit_args;
+int trispec_commit_kv(const trispec_commit_args* a, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * Fused pass: the four calls above in order on `stream` (one verification round of

@@ -60,6 +60,19 @@ class ScanArgs(C.Structure):
                 ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
 
 
+class PruneArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("parent", _vp), ("tok", _vp), ("mask", _vp), ("root", _vp),
+                ("n_keep", _vp), ("node_map", _vp), ("parent_out", _vp), ("tok_out", _vp),
+                ("mask_out", _vp), ("depth_out", _vp)]
+
+
+class CommitArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("Hkv", _i), ("D", _i), ("k_tree", _vp), ("v_tree", _vp),
+                ("kv_layout", _i), ("k_cache", _vp), ("v_cache", _vp), ("Lmax", _i), ("num_blocks", _i),
+                ("block_size", _i), ("max_blocks_per_seq", _i), ("block_table", _vp), ("ctx_len", _vp),
+                ("path", _vp), ("accept_len", _vp), ("active", _vp), ("ctx_len_out", _vp), ("dev_status", _vp)]
+
+
 class HostIO(C.Structure):
     _fields_ = [(n, _vp) for n in ("parent", "tok", "q", "k_tree", "v_tree", "h", "accept_len", "bonus_tok",
                                    "last_node", "path", "escalate")]
@@ -77,6 +90,8 @@ _lib.trispec_lmhead_stats_workspace.argtypes = [C.POINTER(LmheadArgs)]
 _lib.trispec_lmhead_stats.argtypes = [C.POINTER(LmheadArgs), _vp]
 _lib.trispec_lmhead_stats_noalloc.argtypes = [C.POINTER(LmheadArgs), _vp]
 _lib.trispec_accept_scan.argtypes = [C.POINTER(ScanArgs), _vp]
+_lib.trispec_prune_tree.argtypes = [C.POINTER(PruneArgs), _vp]
+_lib.trispec_commit_kv.argtypes = [C.POINTER(CommitArgs), _vp]
 _lib.trispec_verify.argtypes = [C.POINTER(TreeArgs), C.POINTER(AttnArgs), C.POINTER(LmheadArgs),
                                 C.POINTER(ScanArgs), _vp]
 
@@ -85,7 +100,8 @@ _lib.trispec_verify_host.argtypes = [C.POINTER(HostIO), C.POINTER(TreeArgs), C.P
 
 EXPORTS = ["trispec_verify_host", "trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
            "trispec_verify_attn_workspace", "trispec_verify_attn", "trispec_lmhead_stats_workspace",
-           "trispec_lmhead_stats", "trispec_lmhead_stats_noalloc", "trispec_accept_scan", "trispec_verify"]
+           "trispec_lmhead_stats", "trispec_lmhead_stats_noalloc", "trispec_accept_scan", "trispec_verify",
+           "trispec_prune_tree", "trispec_commit_kv"]
 
 
 class TrispecError(RuntimeError):
@@ -206,6 +222,41 @@ def alloc_scan_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
     }
 
 
+def prune_args(parent, tok, mask, root, out: Dict[str, torch.Tensor]) -> PruneArgs:
+    B, T = parent.shape
+    a = PruneArgs()
+    a.B, a.T = B, T
+    a.parent, a.tok, a.mask, a.root = _p(parent), _p(tok), _p(mask), _p(root)
+    a.n_keep, a.node_map = _p(out["n_keep"]), _p(out["node_map"])
+    a.parent_out, a.tok_out = _p(out["parent"]), _p(out["tok"])
+    a.mask_out, a.depth_out = _p(out.get("mask")), _p(out.get("depth"))
+    return a
+
+
+def alloc_prune_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
+    i32 = dict(dtype=torch.int32, device=device)
+    return {"n_keep": torch.full((B,), -7, **i32), "node_map": torch.full((B, T), -7, **i32),
+            "parent": torch.full((B, T), -7, **i32), "tok": torch.full((B, T), -7, **i32),
+            "mask": torch.full((B, T), -7, dtype=torch.int64, device=device), "depth": torch.full((B, T), -7, **i32)}
+
+
+def commit_args(k_tree, v_tree, k_cache, v_cache, ctx_len, path, accept_len, ctx_len_out, block_table=None,
+                block_size=64, active=None, dev_status=None) -> CommitArgs:
+    B, T, Hkv, D = k_tree.shape
+    a = CommitArgs()
+    a.B, a.T, a.Hkv, a.D = B, T, Hkv, D
+    a.k_tree, a.v_tree, a.k_cache, a.v_cache = _p(k_tree), _p(v_tree), _p(k_cache), _p(v_cache)
+    if block_table is None:
+        a.kv_layout, a.Lmax = KV_CONTIGUOUS, k_cache.shape[1]
+        a.num_blocks, a.block_size, a.max_blocks_per_seq = 0, 0, 0
+    else:
+        a.kv_layout, a.Lmax = KV_PAGED, 0
+        a.num_blocks, a.block_size, a.max_blocks_per_seq = k_cache.shape[0], block_size, block_table.shape[1]
+    a.block_table, a.ctx_len, a.path, a.accept_len = _p(block_table), _p(ctx_len), _p(path), _p(accept_len)
+    a.active, a.ctx_len_out, a.dev_status = _p(active), _p(ctx_len_out), _p(dev_status)
+    return a
+
+
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     return torch.empty(max(256, (nbytes + 255) // 256 * 256), dtype=torch.uint8, device=device)
 
@@ -221,6 +272,14 @@ def trispec_verify_attn_workspace(args: AttnArgs) -> int:
 
 def trispec_verify_attn(args: AttnArgs, stream=None):
     _check(_lib.trispec_verify_attn(C.byref(args), _stream(stream)))
+
+
+def trispec_prune_tree(args: PruneArgs, stream=None):
+    _check(_lib.trispec_prune_tree(C.byref(args), _stream(stream)))
+
+
+def trispec_commit_kv(args: CommitArgs, stream=None):
+    _check(_lib.trispec_commit_kv(C.byref(args), _stream(stream)))
 
 
 def trispec_lmhead_stats_workspace(args: LmheadArgs) -> int:

@@ -1,0 +1,177 @@
+"""GPU parity of token pruning and KV commit against the oracle (bit-exact: integer and byte work),
+through the C ABI, plus a proxy round -> prune -> commit composition on one stream."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import trispec_oracle as orc
+from paper_2601_23180_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+
+def _trees(name, B, seed=0):
+    cfg = gen.small_variant(gen.CONFIGS[name], B=B, seed=seed)
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(B)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(B)])
+    return cfg, parent, tok
+
+
+def _run_prune(parent, tok, root):
+    import torch
+    import tests.gpu_helpers as H
+    from paper_2601_23180_b200 import binding as ts
+    B, T = parent.shape
+    pd, td = H.i32_dev(parent), H.i32_dev(tok)
+    mask, _ = H.run_tree_mask(pd)
+    out = ts.alloc_prune_out(B, T)
+    ts.trispec_prune_tree(ts.prune_args(pd, td, mask, H.i32_dev(root), out))
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+@pytest.mark.parametrize("name,B", [("proxy_tree", 37), ("llama_tree", 9), ("tiny_chain", 5)])
+def test_prune_bit_exact(name, B):
+    cfg, parent, tok = _trees(name, B, seed=3)
+    T = cfg.T
+    g = np.random.default_rng(7)
+    root = g.integers(-1, T, size=B).astype(np.int32)      # -1 = sequence skipped
+    root[0] = 0                                            # identity
+    root[-1] = T - 1                                       # a leaf
+    got = _run_prune(parent, tok, root)
+    ref = orc.prune_tree(parent, tok, root)
+    for k in ("n_keep", "node_map", "parent", "tok"):
+        assert np.array_equal(got[k], ref[k]), k
+    # mask / depth of the pruned tree = what the mask oracle gives for the pruned parents
+    for b in range(B):
+        n = int(ref["n_keep"][b])
+        if n:
+            m, d = orc.build_tree_mask(ref["parent"][b:b + 1, :n])
+            assert np.array_equal(got["mask"][b, :n].view(np.uint64), m[0])
+            assert np.array_equal(got["depth"][b, :n], d[0])
+        assert (got["mask"][b, n:] == 0).all() and (got["depth"][b, n:] == -1).all()
+
+
+def test_prune_large_batch_and_argument_errors():
+    import torch
+    from paper_2601_23180_b200 import binding as ts
+    cfg, parent, tok = _trees("proxy_tree", 64, seed=1)
+    reps = 47                                              # 3008 sequences: many blocks, ragged last block
+    parent, tok = np.tile(parent, (reps, 1)), np.tile(tok, (reps, 1))
+    root = np.random.default_rng(0).integers(-1, cfg.T, size=parent.shape[0]).astype(np.int32)
+    got = _run_prune(parent, tok, root)
+    ref = orc.prune_tree(parent, tok, root)
+    for k in ("n_keep", "node_map", "parent", "tok"):
+        assert np.array_equal(got[k], ref[k]), k
+    a = ts.PruneArgs()
+    a.B, a.T = 4, 65
+    n0 = ts.launch_count()
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_prune_tree(a)
+    assert e.value.code == 2 and ts.launch_count() == n0   # T > 64
+    a.T = 9
+    with pytest.raises(ts.TrispecError) as e:
+        ts.trispec_prune_tree(a)
+    assert e.value.code == 1 and ts.launch_count() == n0   # null pointers
+
+
+def _run_commit(cfg, inp, path, acc, active=None, in_place=False):
+    import torch
+    import tests.gpu_helpers as H
+    from paper_2601_23180_b200 import binding as ts
+    dev = H.to_device(inp)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx_out = dev["ctx_len"] if in_place else torch.full_like(dev["ctx_len"], -7)
+    act = None if active is None else torch.from_numpy(active).cuda()
+    a = ts.commit_args(dev["k_tree"], dev["v_tree"], dev["k_cache"], dev["v_cache"], dev["ctx_len"], H.i32_dev(path),
+                       H.i32_dev(acc), ctx_out, block_table=dev.get("block_table"), block_size=cfg.block_size,
+                       active=act, dev_status=status)
+    ts.trispec_commit_kv(a)
+    torch.cuda.synchronize()
+    bits = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return bits(dev["k_cache"]), bits(dev["v_cache"]), ctx_out.cpu().numpy(), int(status.item())
+
+
+@pytest.mark.parametrize("name,in_place", [("proxy_tree", False), ("long_paged", True), ("target_escalated", False)])
+def test_commit_bit_exact(name, in_place):
+    paged = name == "long_paged"
+    cfg = gen.small_variant(gen.CONFIGS[name], B=6, L=300, L_min=300 if paged else None, n_active=None, seed=4)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    B, T = cfg.B, cfg.T
+    g = np.random.default_rng(11)
+    inp["ctx_len"] = np.array([0, 63, 64, 200, 299 - 7, 128], dtype=np.int32)
+    # accepted paths: descending chains of real tree nodes
+    path = np.full((B, T), -1, dtype=np.int32)
+    acc = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        cur, n = 0, 0
+        while n < [0, 3, 6, 2, 6, 1][b]:
+            kids = np.nonzero(inp["parent"][b] == cur)[0]
+            if not len(kids):
+                break
+            cur = int(g.choice(kids))
+            path[b, n] = cur
+            n += 1
+        acc[b] = n
+    active = np.array([1, 1, 1, 0, 1, 1], dtype=np.uint8)
+    ref_k, ref_v, ref_len = orc.commit_kv(inp["k_cache"], inp["v_cache"], inp["ctx_len"], inp["k_tree"], inp["v_tree"],
+                                          path, acc, block_table=inp.get("block_table"), block_size=cfg.block_size,
+                                          active=active)
+    got_k, got_v, got_len, status = _run_commit(cfg, inp, path, acc, active=active, in_place=in_place)
+    assert status == 0
+    assert np.array_equal(got_len, ref_len)
+    assert np.array_equal(got_k, ref_k) and np.array_equal(got_v, ref_v)
+
+
+def test_commit_without_room_flags_and_leaves_the_sequence_alone():
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=2, L=128, seed=2)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    inp["ctx_len"] = np.array([127, 126], dtype=np.int32)
+    path = np.full((2, cfg.T), -1, dtype=np.int32)
+    path[:, 0] = 1
+    acc = np.array([1, 1], dtype=np.int32)                 # two rows each: only sequence 1 fits
+    ref_k, ref_v, ref_len = orc.commit_kv(inp["k_cache"], inp["v_cache"], inp["ctx_len"], inp["k_tree"], inp["v_tree"],
+                                          path, acc)
+    got_k, got_v, got_len, status = _run_commit(cfg, inp, path, acc)
+    assert status == 9
+    assert got_len.tolist() == ref_len.tolist() == [127, 128]
+    assert np.array_equal(got_k, ref_k) and np.array_equal(got_v, ref_v)
+
+
+def test_round_then_prune_and_commit_on_one_stream():
+    """One proxy round of the decode loop: verify pass -> (escalated sequences) prune at the
+    last accepted node, and commit the accepted path, launched back to back; compared with the
+    oracle run on the GPU's own scan outputs (so only the new steps are under test here)."""
+    import torch
+    import tests.gpu_helpers as H
+    from paper_2601_23180_b200 import binding as ts
+    from paper_2601_23180_b200 import runner
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=6, L=200, V=8000, d=256, rho=0.3,
+                            logit_scale=3.6 / (0.02 * 16.0), seed=5)
+    inp = gen.make_inputs(cfg)
+    inp["ctx_len"] = np.full(cfg.B, 130, dtype=np.int32)   # room for the appended rows
+    pas = runner.VerifyPass(cfg, inp)
+    B, T = cfg.B, cfg.T
+    pout = ts.alloc_prune_out(B, T)
+    # prune where the proxy escalated: root = last_node for escalated sequences, else -1
+    pas.run()
+    esc = pas.scan_out["escalate"].to(torch.bool)
+    root = torch.where(esc, pas.scan_out["last_node"], torch.full_like(pas.scan_out["last_node"], -1))
+    ts.trispec_prune_tree(ts.prune_args(pas.dev["parent"], pas.dev["tok"], pas.mask, root, pout))
+    ctx_out = torch.zeros_like(pas.dev["ctx_len"])
+    ts.trispec_commit_kv(ts.commit_args(pas.dev["k_tree"], pas.dev["v_tree"], pas.dev["k_cache"], pas.dev["v_cache"],
+                                        pas.dev["ctx_len"], pas.scan_out["path"], pas.scan_out["accept_len"], ctx_out,
+                                        dev_status=pas.status))
+    torch.cuda.synchronize()
+    assert int(pas.status.item()) == 0
+    scan = {k: v.cpu().numpy() for k, v in pas.scan_out.items()}
+    ref_p = orc.prune_tree(inp["parent"], inp["tok"], root.cpu().numpy())
+    for k in ("n_keep", "node_map", "parent", "tok"):
+        assert np.array_equal(pout[k].cpu().numpy(), ref_p[k]), k
+    ref_k, ref_v, ref_len = orc.commit_kv(inp["k_cache"], inp["v_cache"], inp["ctx_len"], inp["k_tree"], inp["v_tree"],
+                                          scan["path"], scan["accept_len"])
+    bits = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(ctx_out.cpu().numpy(), ref_len)
+    assert np.array_equal(bits(pas.dev["k_cache"]), ref_k) and np.array_equal(bits(pas.dev["v_cache"]), ref_v)
+    assert scan["escalate"].sum() >= 1 and (scan["accept_len"] > 0).any()
