@@ -308,6 +308,48 @@ def run_only(args, cfg):
                                    "work_per_launch": mask_bytes, "ms_per_launch": ms_mask}})
         print(json.dumps(out), flush=True)
         return
+    if args.only == "prune":
+        # token pruning on the scan stress trees: every sequence pruned at a random node of depth <= 2
+        B, T = 1 << 20, cfg.T
+        parent, tok, _ = _scan_stress_inputs(cfg, B)
+        mask = torch.zeros((B, T), dtype=torch.int64, device="cuda")
+        ts.trispec_build_tree_mask(ts.tree_args(parent, mask, None))
+        g = torch.Generator(device="cuda").manual_seed(cfg.seed)
+        root = torch.randint(0, 8, (B,), generator=g, device="cuda", dtype=torch.int32)
+        po = ts.alloc_prune_out(B, T)
+        pa = ts.prune_args(parent, tok, mask, root, po)
+        byts = B * (T * 40 + 8)       # in: parent, tok (4 B), mask (8 B) per node; out: 24 B per node
+        ms = timed(lambda: ts.trispec_prune_tree(pa), byts)
+        out.update({"config": {"workload": f"prune stress: 2^20 sequences of the {cfg.name} tree shape", "T": T,
+                               "mean_kept_nodes": po["n_keep"].float().mean().item(), "l2": out["config"]["l2"]},
+                    "value": B * cfg.k / (ms * 1e-3), "ms_per_step": ms, "dtype": "int32",
+                    "roofline": {"kernel": "prune_tree_kernel", "bound": "hbm", "achieved": byts / ms / 1e6,
+                                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": byts / ms / 1e6 / peaks["hbm_gbs"],
+                                 "work_per_launch": byts, "ms_per_launch": ms, "traffic": None}})
+        print(json.dumps(out), flush=True)
+        return
+    if args.only == "commit":
+        # KV commit stress: 32768 sequences with the workload's KV heads, 7 rows appended each
+        B, T, Hkv, D = 32768, cfg.T, cfg.Hkv, cfg.D
+        kt = torch.randn((B, T, Hkv, D), device="cuda").to(torch.bfloat16)
+        vt = torch.randn((B, T, Hkv, D), device="cuda").to(torch.bfloat16)
+        Lcap = 8
+        kc = torch.zeros((B, Lcap, Hkv, D), dtype=torch.bfloat16, device="cuda")
+        vc = torch.zeros_like(kc)
+        ctx = torch.zeros(B, dtype=torch.int32, device="cuda")
+        ctx_out = torch.zeros_like(ctx)
+        path = torch.arange(1, T + 1, dtype=torch.int32, device="cuda").clamp(max=T - 1).repeat(B, 1).contiguous()
+        acc = torch.full((B,), 6, dtype=torch.int32, device="cuda")
+        ca = ts.commit_args(kt, vt, kc, vc, ctx, path, acc, ctx_out)
+        byts = B * 7 * Hkv * D * 2 * 2 * 2          # 7 rows of K and V read and written
+        ms = timed(lambda: ts.trispec_commit_kv(ca), byts)
+        out.update({"config": {"workload": f"commit stress: {B} sequences x 7 appended rows, Hkv {Hkv}", "l2": out["config"]["l2"]},
+                    "value": B * 6 / (ms * 1e-3), "ms_per_step": ms, "dtype": "u8",
+                    "roofline": {"kernel": "kv_commit_kernel", "bound": "hbm", "achieved": byts / ms / 1e6,
+                                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": byts / ms / 1e6 / peaks["hbm_gbs"],
+                                 "work_per_launch": byts, "ms_per_launch": ms, "traffic": None}})
+        print(json.dumps(out), flush=True)
+        return
     if args.only == "attention":
         inp = gen.make_inputs(cfg, with_lm_head=False)
         small = dataclasses.replace(cfg, V=4096, d=64)      # the LM head is not run: a token-sized stand-in
@@ -347,7 +389,7 @@ def main():
     ap.add_argument("--workload", default="proxy_tree")
     ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan"],
+    ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan", "prune", "commit"],
                     help="time one entry point alone (L2 flushed before each call) instead of the pass")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the number of sequences of the workload (reduced copies for profiler captures)")

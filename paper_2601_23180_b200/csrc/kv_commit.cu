@@ -1,8 +1,8 @@
 // KV commit of the accepted path (X <- X + Y of Algorithm 1 as the KV cache sees it): the keys
 // and values of tree node 0 (the last committed token) and of the accepted draft nodes are
-// appended to each sequence's cache. One block per (sequence, appended row): a row is
-// Hkv x 128 bf16 for K and the same for V, copied with 16-byte loads and stores. A second,
-// tiny kernel then writes the new lengths (so that they may be updated in place).
+// appended to each sequence's cache. One block per sequence walks its appended rows (a row is
+// Hkv x 128 bf16 for K and the same for V) with 16-byte loads and stores, four per thread in
+// flight. A second, tiny kernel then writes the new lengths (so that they may be updated in place).
 #include "host_common.h"
 
 namespace trispec {
@@ -44,32 +44,48 @@ __global__ void __launch_bounds__(kCommitThreads)
 kv_commit_kernel(const CommitParams p) {
   pdl_launch_dependents();
   pdl_wait();
-  const int b = blockIdx.x / p.T, j = blockIdx.x % p.T;
+  const int b = blockIdx.x;
   const int L = __ldg(p.ctx_len + b);
   const int rows = commit_rows(p, b, L);
   if (rows < 0) {
-    if (j == 0 && threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 9);   // no room: sequence skipped
+    if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 9);   // no room: sequence skipped
     return;
   }
-  if (j >= rows) return;
-  int node = 0;
-  if (j > 0) {
-    node = __ldg(p.path + static_cast<long long>(b) * p.T + (j - 1));
-    if (node < 0 || node >= p.T) return;        // malformed path entry: nothing copied for it
-  }
-  const int t = L + j;
   const int row16 = p.Hkv * 16;                  // 16-byte units per row (Hkv x 128 bf16)
-  const long long src = (static_cast<long long>(b) * p.T + node) * row16;
-  long long dst;
-  if (!p.paged) {
-    dst = (static_cast<long long>(b) * p.Lmax + t) * row16;
-  } else {
-    const int blk = __ldg(p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq + t / 64);
-    dst = (static_cast<long long>(blk) * 64 + (t % 64)) * row16;
-  }
-  for (int i = threadIdx.x; i < 2 * row16; i += kCommitThreads) {
-    if (i < row16) p.k_cache[dst + i] = __ldg(p.k_tree + src + i);
-    else p.v_cache[dst + (i - row16)] = __ldg(p.v_tree + src + (i - row16));
+  const int per_row = 2 * row16;                 // K then V
+  const int total = rows * per_row;
+  // four 16-byte units per thread and round, loads first: keeps 64 bytes per thread in flight
+  for (int i0 = threadIdx.x; i0 < total; i0 += 4 * kCommitThreads) {
+    uint4 val[4];
+    long long dsti[4];
+    bool isv[4], ok[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * kCommitThreads;
+      ok[u] = i < total;
+      dsti[u] = 0; isv[u] = false; val[u] = make_uint4(0, 0, 0, 0);
+      if (!ok[u]) continue;
+      const int j = i / per_row, e = i % per_row;
+      int node = 0;
+      if (j > 0) {
+        node = __ldg(p.path + static_cast<long long>(b) * p.T + (j - 1));
+        if (node < 0 || node >= p.T) { ok[u] = false; continue; }   // malformed path entry: nothing copied
+      }
+      const int t = L + j;
+      isv[u] = e >= row16;
+      const int off = isv[u] ? e - row16 : e;
+      const long long src = (static_cast<long long>(b) * p.T + node) * row16 + off;
+      if (!p.paged) {
+        dsti[u] = (static_cast<long long>(b) * p.Lmax + t) * row16 + off;
+      } else {
+        const int blk = __ldg(p.block_table + static_cast<long long>(b) * p.max_blocks_per_seq + t / 64);
+        dsti[u] = (static_cast<long long>(blk) * 64 + (t % 64)) * row16 + off;
+      }
+      val[u] = __ldg((isv[u] ? p.v_tree : p.k_tree) + src);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (ok[u]) (isv[u] ? p.v_cache : p.k_cache)[dsti[u]] = val[u];
   }
 }
 
@@ -114,7 +130,7 @@ extern "C" int trispec_commit_kv(const trispec_commit_args* a, void* stream) {
   p.block_table = a->block_table; p.ctx_len = a->ctx_len; p.path = a->path; p.accept_len = a->accept_len;
   p.active = a->active; p.ctx_len_out = a->ctx_len_out; p.dev_status = a->dev_status;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  TRISPEC_CUDA_OK(launch_dependent(kv_commit_kernel, static_cast<unsigned>(a->B * a->T), kCommitThreads, 0, st, 1, p));
+  TRISPEC_CUDA_OK(launch_dependent(kv_commit_kernel, static_cast<unsigned>(a->B), kCommitThreads, 0, st, 1, p));
   count_launch();
   TRISPEC_CUDA_OK(launch_dependent(kv_commit_len_kernel, static_cast<unsigned>((a->B + 255) / 256), 256, 0, st, 1, p));
   count_launch();
