@@ -41,6 +41,10 @@ import numpy as np
 
 MODE_PROXY = 0
 MODE_TARGET = 1
+# routing criteria of the "Routing Criteria" study: which proxy feature decides trust at a position
+CRIT_MARGIN = 0    # top_1(p) - top_2(p) >= lambda   (Eq. 8, the default)
+CRIT_TOP1 = 1      # top_1(p) >= lambda
+CRIT_ENTROPY = 2   # H(p) <= lambda
 
 
 def bf16_to_f64(bits: np.ndarray) -> np.ndarray:
@@ -137,7 +141,7 @@ def verify_attn(q: np.ndarray, k_tree: np.ndarray, v_tree: np.ndarray, mask: np.
 # ----------------------------------------------------------------------------------------
 # LM-head softmax statistics (Eq. 5 distributions; top_1/top_2 of Eq. 8)
 # ----------------------------------------------------------------------------------------
-STAT_F = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft")
+STAT_F = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft", "entropy")
 STAT_I = ("top1_idx", "top2_idx")
 
 
@@ -154,7 +158,8 @@ def lmhead_stats(h: np.ndarray, W: np.ndarray, parent: np.ndarray, tok: np.ndarr
     the largest entry among the other indices (top2_val, top2_idx), p_top1, p_top2; and for
     each child node c the logit of its drafted token in its parent's row (draft_logit[b][c])
     and the probability p_draft[b][c] = p_{parent(c)}(tok[c]). Entries of node 0 in
-    draft_logit / p_draft are NaN. h is [B][T][d] bf16 bits, W is [V][d] bf16 bits.
+    draft_logit / p_draft are NaN. entropy = -sum_v p ln p (nats), the feature of the entropy
+    routing criterion of the "Routing Criteria" study. h is [B][T][d] bf16 bits, W is [V][d] bf16 bits.
     All outputs are [B][T]; rows of sequences not in `seqs` are NaN / -1."""
     B, T, d = h.shape
     if W64 is None:
@@ -178,6 +183,9 @@ def lmhead_stats(h: np.ndarray, W: np.ndarray, parent: np.ndarray, tok: np.ndarr
             out["top2_idx"][b, r] = i2
             out["p_top1"][b, r] = np.exp(z[i1] - lse)
             out["p_top2"][b, r] = np.exp(z[i2] - lse)
+            p = np.exp(z - lse)
+            nz = p > 0
+            out["entropy"][b, r] = -(p[nz] * (z[nz] - lse)).sum()     # -sum p ln p, in nats
             for c in range(1, T):
                 if int(parent[b, c]) == r:
                     out["draft_logit"][b, c] = z[int(tok[b, c])]
@@ -192,7 +200,8 @@ def accept_scan(p_top1: np.ndarray, p_top2: np.ndarray, top1_idx: np.ndarray,
                 parent: np.ndarray, tok: np.ndarray, lam: float, mode: int = MODE_PROXY,
                 active: Optional[np.ndarray] = None,
                 start_node: Optional[np.ndarray] = None,
-                near_eps: float = 1e-3) -> Dict[str, np.ndarray]:
+                near_eps: float = 1e-3, criterion: int = CRIT_MARGIN,
+                entropy: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
     """Greedy walk of each draft tree.
 
     At the current node (position i+1 of the chain formulas, i = tokens accepted so far):
@@ -202,10 +211,14 @@ def accept_scan(p_top1: np.ndarray, p_top2: np.ndarray, top1_idx: np.ndarray,
         none -> tau_a = i < tau_m: case (i), approve, bonus = arg-max token of this node;
         found -> accept it and move there.
       TARGET mode: the same without the margin test (never escalates).
+    `criterion` replaces the margin by another proxy feature (the paper's routing-criteria
+    study): CRIT_TOP1 trusts a position iff top_1(p) >= lambda, CRIT_ENTROPY iff the entropy of
+    p is <= lambda (reading: plain Shannon entropy in nats; the paper cites a "composite"
+    entropy criterion without defining it).
 
     Outputs per sequence: accept_len, escalate (0/1), bonus_tok (-1 if escalated), path
     [B][T] (accepted node ids in order, -1 padded), last_node, near_thr (number of visited
-    positions with |margin - lambda| < near_eps; PROXY mode only); plus n_escalated and
+    positions with |feature - lambda| < near_eps; PROXY mode only); plus n_escalated and
     esc_index (ascending sequence ids that escalated, -1 padded). Inactive sequences get
     accept_len 0, escalate 0, bonus -1, last_node -1.
     """
@@ -226,10 +239,18 @@ def accept_scan(p_top1: np.ndarray, p_top2: np.ndarray, top1_idx: np.ndarray,
         n = 0
         while True:
             if mode == MODE_PROXY:
-                margin = float(p_top1[b, cur]) - float(p_top2[b, cur])
-                if abs(margin - lam) < near_eps:
+                if criterion == CRIT_MARGIN:
+                    feature = float(p_top1[b, cur]) - float(p_top2[b, cur])
+                    trusted = feature >= lam
+                elif criterion == CRIT_TOP1:
+                    feature = float(p_top1[b, cur])
+                    trusted = feature >= lam
+                else:
+                    feature = float(entropy[b, cur])
+                    trusted = feature <= lam
+                if abs(feature - lam) < near_eps:
                     res["near_thr"][b] += 1
-                if not (margin >= lam):
+                if not trusted:
                     res["escalate"][b] = 1
                     break
             nxt = -1

@@ -205,3 +205,86 @@ def test_commit_respects_capacity_and_active():
                                acc, active=np.array([1, 1, 0], dtype=np.uint8))
     assert nl.tolist() == [Lcap - 1, Lcap, 10]          # 0: no room, 1: fits exactly, 2: inactive
     assert np.array_equal(kc[0], inp["k_cache"][0]) and np.array_equal(kc[2], inp["k_cache"][2])
+
+
+# ------------------------------------------------------------------------------ entropy, routing criteria
+def _stats_from_logits(z):
+    """Runs lmhead_stats on a [rows][V] logit table by making W the identity-like basis: h = one-hot
+    rows are not needed - instead build h, W with W = I (V x V) and h = the logits (bf16-exact values)."""
+    rows, V = z.shape
+    d = ((V + 63) // 64) * 64
+    W = np.zeros((V, d), dtype=np.float32)
+    W[np.arange(V), np.arange(V)] = 1.0
+    h = np.zeros((1, rows, d), dtype=np.float32)
+    h[0, :, :V] = z
+    to_bits = lambda x: (x.view(np.uint32) >> 16).astype(np.uint16)
+    parent = np.arange(-1, rows - 1, dtype=np.int32)[None]
+    tok = np.zeros((1, rows), dtype=np.int32)
+    return orc.lmhead_stats(to_bits(h), to_bits(W), parent, tok, 1.0)
+
+
+def test_entropy_closed_forms():
+    import math
+    V = 8
+    z = np.zeros((4, V), dtype=np.float32)
+    z[1, 0] = 64.0                      # one-hot in the limit: H -> 0
+    z[2, :2] = 1.0                      # two maxima and six entries lower by 1
+    z[3, 0] = 2.0                       # logits {2, 0 x 7}: p1 = e^2 / (e^2 + 7)
+    st = _stats_from_logits(z)
+    assert abs(st["entropy"][0, 0] - math.log(V)) < 1e-12              # uniform: ln V
+    assert 0 <= st["entropy"][0, 1] < 1e-20
+    a = 2 * math.e / (2 * math.e + 6)
+    h2 = -(a * math.log(a / 2) + (1 - a) * math.log((1 - a) / 6))
+    assert abs(st["entropy"][0, 2] - h2) < 1e-12
+    p1 = math.exp(2) / (math.exp(2) + 7)
+    h3 = -(p1 * math.log(p1) + (1 - p1) * math.log((1 - p1) / 7))
+    assert abs(st["entropy"][0, 3] - h3) < 1e-12
+    assert (st["entropy"][0] <= math.log(V) + 1e-12).all()
+    # H = lse - E_p[z]
+    for r in range(4):
+        p = np.exp(z[r].astype(np.float64) - st["lse"][0, r])
+        assert abs(st["entropy"][0, r] - (st["lse"][0, r] - (p * z[r]).sum())) < 1e-12
+
+
+@pytest.mark.parametrize("crit", [orc.CRIT_TOP1, orc.CRIT_ENTROPY])
+def test_scan_criteria_reduce_to_known_cases(crit):
+    cfg = _cfg(B=5, seed=9)
+    B, T = 5, cfg.T
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(B)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(B)])
+    g = np.random.default_rng(1)
+    top1 = g.integers(0, cfg.V, size=(B, T))
+    for b in range(B):
+        for i in range(T):
+            kids = np.nonzero(parent[b] == i)[0]
+            if len(kids) and g.random() < 0.8:
+                top1[b, i] = tok[b, kids[0]]
+    p1 = g.uniform(0.2, 1.0, size=(B, T))
+    p2 = g.uniform(0.0, 0.2, size=(B, T))
+    ent = g.uniform(0.0, 3.0, size=(B, T))
+    kw = dict(criterion=crit, entropy=ent)
+    target = orc.accept_scan(p1, p2, top1, parent, tok, 0.5, mode=orc.MODE_TARGET)
+    # a threshold nothing fails -> never escalates and equals plain greedy acceptance
+    always = orc.accept_scan(p1, p2, top1, parent, tok, -1.0 if crit == orc.CRIT_TOP1 else 10.0, **kw)
+    assert not always["escalate"].any()
+    for k in ("accept_len", "bonus_tok", "path"):
+        assert np.array_equal(always[k], target[k])
+    # a threshold everything fails -> escalates at the root with nothing accepted
+    never = orc.accept_scan(p1, p2, top1, parent, tok, 2.0 if crit == orc.CRIT_TOP1 else -1.0, **kw)
+    assert never["escalate"].all() and (never["accept_len"] == 0).all() and (never["bonus_tok"] == -1).all()
+    # general threshold: the walk stops at the first visited node whose feature fails
+    lam = 0.6 if crit == orc.CRIT_TOP1 else 1.5
+    r = orc.accept_scan(p1, p2, top1, parent, tok, lam, **kw)
+    for b in range(B):
+        nodes = [0] + target["path"][b, :target["accept_len"][b]].tolist()
+        ok = [(p1[b, n] >= lam) if crit == orc.CRIT_TOP1 else (ent[b, n] <= lam) for n in nodes]
+        if all(ok):
+            assert r["escalate"][b] == 0 and r["accept_len"][b] == target["accept_len"][b]
+        else:
+            j = ok.index(False)
+            assert r["escalate"][b] == 1 and r["accept_len"][b] == j and r["last_node"][b] == nodes[j]
+    # top-1 criterion with p2 = 0 is the margin criterion
+    if crit == orc.CRIT_TOP1:
+        m = orc.accept_scan(p1, np.zeros_like(p2), top1, parent, tok, lam)
+        for k in ("accept_len", "escalate", "bonus_tok", "path"):
+            assert np.array_equal(m[k], r[k])
