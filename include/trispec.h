@@ -54,6 +54,11 @@ typedef enum {
 #define TRISPEC_MODE_PROXY 0   /* margin rule of Eq. 8-9 applied (proxy verifier) */
 #define TRISPEC_MODE_TARGET 1  /* plain left-to-right acceptance (target verifier, after Eq. 10) */
 
+/* routing criteria (Section "Routing Criteria"): a position is trusted iff */
+#define TRISPEC_CRIT_MARGIN 0   /* p_top1 - p_top2 >= lambda (Eq. 8; the paper's default) */
+#define TRISPEC_CRIT_TOP1 1     /* p_top1 >= lambda */
+#define TRISPEC_CRIT_ENTROPY 2  /* entropy <= lambda (plain Shannon entropy in nats) */
+
 #define TRISPEC_KV_CONTIGUOUS 0 /* k_cache, v_cache: [B][Lmax][Hkv][D] */
 #define TRISPEC_KV_PAGED 1      /* pool [num_blocks][block_size][Hkv][D] + block_table */
 
@@ -122,7 +127,8 @@ int trispec_verify_attn(const trispec_attn_args* a, void* stream);
  *    Per row r = b*T + node (all arrays [B*T]):
  *      max, lse = log sum_v exp z; (top1_val, top1_idx) largest entry, (top2_val, top2_idx)
  *      largest entry among the other indices (ties -> lowest index);
- *      p_top1 = exp(top1_val - lse), p_top2 likewise.
+ *      p_top1 = exp(top1_val - lse), p_top2 likewise; entropy = -sum_v p_v ln p_v (the
+ *      feature of the entropy routing criterion, "Routing Criteria" study).
  *    Per CHILD node c >= 1: draft_logit[b*T+c] = z[b*T+parent[c]][tok[c]] and
  *      p_draft = exp(draft_logit - lse[parent row]); entries of node 0 are NaN.
  *    h [B*T][d] bf16, W [V][d] bf16 (row-major, 16-byte aligned, d % 64 == 0).
@@ -131,6 +137,7 @@ typedef struct {
   float *max, *lse, *top1_val, *top2_val, *p_top1, *p_top2;
   int32_t *top1_idx, *top2_idx;
   float *draft_logit, *p_draft;
+  float* entropy;  /* optional (may be NULL): -sum_v p ln p in nats, per row like lse */
 } trispec_stats;
 
 typedef struct {
@@ -184,7 +191,8 @@ int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream);
  *      escalate 0, bonus -1, last_node -1, path -1).
  *    Outputs: accept_len, bonus_tok, last_node, near_thr int32 [B]; escalate uint8 [B];
  *      path int32 [B][T] (accepted node ids in order, -1 padded);
- *      near_thr = visited positions with |margin - lambda| < 1e-3 (PROXY mode);
+ *      near_thr = visited positions with |feature - lambda| < 1e-3 (PROXY mode), the feature
+ *      being the margin, p_top1 or the entropy as `criterion` selects;
  *      n_escalated int32 [1]; esc_index int32 [B] ascending ids of escalated sequences,
  *      -1 padded. near_thr, n_escalated and esc_index may be NULL (n_escalated and esc_index
  *      only together).
@@ -193,8 +201,9 @@ typedef struct {
   int B, T;
   float lambda;
   int mode;
+  int criterion;             /* TRISPEC_CRIT_*: which proxy feature decides trust (0 = margin) */
   const int32_t *parent, *tok;
-  trispec_stats in;          /* only p_top1, p_top2, top1_idx are read */
+  trispec_stats in;          /* read: top1_idx, and p_top1, p_top2 or entropy as the criterion needs */
   const uint8_t* active;
   const int32_t* start_node;
   int32_t *accept_len, *bonus_tok, *path, *last_node, *near_thr, *n_escalated, *esc_index;

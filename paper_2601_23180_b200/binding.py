@@ -44,7 +44,7 @@ class AttnArgs(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [(n, _vp) for n in ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2",
-                                   "top1_idx", "top2_idx", "draft_logit", "p_draft")]
+                                   "top1_idx", "top2_idx", "draft_logit", "p_draft", "entropy")]
 
 
 class LmheadArgs(C.Structure):
@@ -54,7 +54,7 @@ class LmheadArgs(C.Structure):
 
 
 class ScanArgs(C.Structure):
-    _fields_ = [("B", _i), ("T", _i), ("lam", _f), ("mode", _i), ("parent", _vp), ("tok", _vp),
+    _fields_ = [("B", _i), ("T", _i), ("lam", _f), ("mode", _i), ("criterion", _i), ("parent", _vp), ("tok", _vp),
                 ("stats", Stats), ("active", _vp), ("start_node", _vp), ("accept_len", _vp),
                 ("bonus_tok", _vp), ("path", _vp), ("last_node", _vp), ("near_thr", _vp),
                 ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
@@ -135,7 +135,7 @@ def launch_count() -> int:
     return int(_lib.trispec_launch_count())
 
 
-STAT_F32 = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft")
+STAT_F32 = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft", "entropy")
 STAT_I32 = ("top1_idx", "top2_idx")
 
 
@@ -198,11 +198,14 @@ def lmhead_args(h, W, parent, tok, logit_scale, stats, workspace=None, seq_index
     return a
 
 
+CRIT_MARGIN, CRIT_TOP1, CRIT_ENTROPY = 0, 1, 2
+
+
 def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], active=None,
-              start_node=None) -> ScanArgs:
+              start_node=None, criterion=CRIT_MARGIN) -> ScanArgs:
     B, T = parent.shape
     a = ScanArgs()
-    a.B, a.T, a.lam, a.mode = B, T, float(lam), int(mode)
+    a.B, a.T, a.lam, a.mode, a.criterion = B, T, float(lam), int(mode), int(criterion)
     a.parent, a.tok = _p(parent), _p(tok)
     a.stats = _stats_struct(stats)
     a.active, a.start_node = _p(active), _p(start_node)

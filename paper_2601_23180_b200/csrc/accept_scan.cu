@@ -13,6 +13,13 @@ namespace trispec {
 
 constexpr int kScanThreads = 256;  // 8 sequences per block
 
+// the proxy feature the routing criterion looks at (margin of Eq. 8 by default)
+__device__ __forceinline__ float scan_feature(const trispec_scan_args& a, long long idx) {
+  if (a.criterion == TRISPEC_CRIT_TOP1) return __ldg(a.in.p_top1 + idx);
+  if (a.criterion == TRISPEC_CRIT_ENTROPY) return __ldg(a.in.entropy + idx);
+  return __ldg(a.in.p_top1 + idx) - __ldg(a.in.p_top2 + idx);
+}
+
 __global__ void __launch_bounds__(kScanThreads)
 accept_scan_kernel(trispec_scan_args a) {
   pdl_launch_dependents();
@@ -47,16 +54,18 @@ accept_scan_kernel(trispec_scan_args a) {
     par0 = __ldg(a.parent + base + lane); tok0 = __ldg(a.tok + base + lane);
     top0 = __ldg(a.in.top1_idx + base + lane);
     if (proxy) {
-      const float mg = __ldg(a.in.p_top1 + base + lane) - __ldg(a.in.p_top2 + base + lane);
-      tr0 = mg >= a.lambda; nr0 = fabsf(mg - a.lambda) < 1e-3f;
+      const float f = scan_feature(a, base + lane);
+      tr0 = (a.criterion == TRISPEC_CRIT_ENTROPY) ? (f <= a.lambda) : (f >= a.lambda);
+      nr0 = fabsf(f - a.lambda) < 1e-3f;
     }
   }
   if (has1) {
     par1 = __ldg(a.parent + base + lane + 32); tok1 = __ldg(a.tok + base + lane + 32);
     top1v = __ldg(a.in.top1_idx + base + lane + 32);
     if (proxy) {
-      const float mg = __ldg(a.in.p_top1 + base + lane + 32) - __ldg(a.in.p_top2 + base + lane + 32);
-      tr1 = mg >= a.lambda; nr1 = fabsf(mg - a.lambda) < 1e-3f;
+      const float f = scan_feature(a, base + lane + 32);
+      tr1 = (a.criterion == TRISPEC_CRIT_ENTROPY) ? (f <= a.lambda) : (f >= a.lambda);
+      nr1 = fabsf(f - a.lambda) < 1e-3f;
     }
   }
   // the margin test of every node as one bit (Eq. 8), known to the whole warp
@@ -191,7 +200,12 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
       !a->escalate)
     return TRISPEC_ERR_INVALID_ARG;
   if (a->mode != TRISPEC_MODE_PROXY && a->mode != TRISPEC_MODE_TARGET) return TRISPEC_ERR_INVALID_ARG;
-  if (a->mode == TRISPEC_MODE_PROXY && (!a->in.p_top1 || !a->in.p_top2)) return TRISPEC_ERR_INVALID_ARG;
+  if (a->criterion < TRISPEC_CRIT_MARGIN || a->criterion > TRISPEC_CRIT_ENTROPY) return TRISPEC_ERR_INVALID_ARG;
+  if (a->mode == TRISPEC_MODE_PROXY) {
+    if (a->criterion == TRISPEC_CRIT_MARGIN && (!a->in.p_top1 || !a->in.p_top2)) return TRISPEC_ERR_INVALID_ARG;
+    if (a->criterion == TRISPEC_CRIT_TOP1 && !a->in.p_top1) return TRISPEC_ERR_INVALID_ARG;
+    if (a->criterion == TRISPEC_CRIT_ENTROPY && !a->in.entropy) return TRISPEC_ERR_INVALID_ARG;
+  }
   if ((a->n_escalated == nullptr) != (a->esc_index == nullptr)) return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int per_block = kScanThreads / 32;

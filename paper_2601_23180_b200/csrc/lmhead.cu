@@ -48,7 +48,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 struct __align__(16) LmPartial {
   float m, s, v1, v2;  // raw (unscaled) running max, sum of 2^((z-m)c), top-1 / top-2 raw logits
-  int i1, i2, pad0, pad1;
+  int i1, i2;
+  float t;             // sum of 2^((z-m)c) * z over the range (for the entropy: H = lse - E_p[z])
+  int pad;
 };
 
 struct LmParams {
@@ -188,7 +190,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-3)
     const int row = warp * 32 + lane;  // TMEM lane == row of this CTA's half of the M tile
-    float m = -INFINITY, s = 0.f, v1 = -INFINITY, v2 = -INFINITY;
+    float m = -INFINITY, s = 0.f, tz = 0.f, v1 = -INFINITY, v2 = -INFINITY;
     int i1 = -1, i2 = -1;
     const float c = p.c;
     const uint32_t tmem_empty_leader = cluster_map(smem_u32(tmem_empty), 0);
@@ -213,14 +215,22 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
           cmax = fmaxf(cmax, v);
         }
         if (cmax > m) {
-          s *= ex2f((m - cmax) * c);
+          const float f = ex2f((m - cmax) * c);
+          s *= f;
+          tz *= f;
           m = cmax;
         }
         const float mc = m * c;
-        float acc = 0.f;
+        float acc = 0.f, acz = 0.f;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc += ex2f(fmaf(__uint_as_float(r[j]), c, -mc));
+        for (int j = 0; j < 32; ++j) {
+          const float e = ex2f(fmaf(__uint_as_float(r[j]), c, -mc));
+          acc += e;
+          // masked columns hold -inf with e = 0: keep 0 * inf out of the sum
+          acz = fmaf(e, (j < nv) ? __uint_as_float(r[j]) : 0.f, acz);
+        }
         s += acc;
+        tz += acz;
         if (cmax > v2) {
           const int col0 = n0 + c0;
 #pragma unroll
@@ -237,7 +247,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
     }
     pdl_wait();   // the partials of the previous pass may still be read until earlier kernels are done
     LmPartial out;
-    out.m = m; out.s = s; out.v1 = v1; out.v2 = v2; out.i1 = i1; out.i2 = i2; out.pad0 = 0; out.pad1 = 0;
+    out.m = m; out.s = s; out.v1 = v1; out.v2 = v2; out.i1 = i1; out.i2 = i2; out.t = tz; out.pad = 0;
     p.partial[static_cast<size_t>(range) * (p.n_mt * 2 * LM_BM) + (mt * 2 + rank) * LM_BM + row] = out;
   }
 
@@ -282,17 +292,22 @@ __device__ __forceinline__ void lm_top2_insert(float v, int i, float& v1, int& i
 
 // log-sum-exp of one row from its per-range partials, computed by a whole warp
 __device__ __forceinline__ void lm_row_lse(const LmPartial* part, size_t stride, size_t prow, int n_ranges, float c,
-                                           int lane, float& M, float& S) {
+                                           int lane, float& M, float& S, float& TZ) {
   float m = -INFINITY;
   for (int r = lane; r < n_ranges; r += 32) m = fmaxf(m, part[r * stride + prow].m);
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  float sacc = 0.f;
+  float sacc = 0.f, tacc = 0.f;
   for (int r = lane; r < n_ranges; r += 32) {
     const LmPartial q = part[r * stride + prow];
-    sacc += q.s * ex2f((q.m - m) * c);
+    const float f = ex2f((q.m - m) * c);
+    sacc += q.s * f;
+    tacc += q.t * f;
   }
-  for (int o = 16; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
-  M = m; S = sacc;
+  for (int o = 16; o > 0; o >>= 1) {
+    sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
+    tacc += __shfl_xor_sync(0xffffffffu, tacc, o);
+  }
+  M = m; S = sacc; TZ = tacc;
 }
 
 // One warp per (active sequence, node): merges the row's partial statistics and, for a child
@@ -311,8 +326,8 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
   const size_t stride = static_cast<size_t>(p.n_mt) * 2 * LM_BM;
   const size_t prow = static_cast<size_t>(a) * 64 + node;
 
-  float M, S;
-  lm_row_lse(p.partial, stride, prow, p.n_ranges, p.c, lane, M, S);
+  float M, S, TZ;
+  lm_row_lse(p.partial, stride, prow, p.n_ranges, p.c, lane, M, S, TZ);
   float v1 = -INFINITY, v2 = -INFINITY;
   int i1 = -1, i2 = -1;
   for (int r = lane; r < p.n_ranges; r += 32) {
@@ -337,6 +352,8 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
     p.out.top2_idx[o] = i2;
     p.out.p_top1[o] = expf(v1 * p.scale - lse);
     p.out.p_top2[o] = expf(v2 * p.scale - lse);
+    // entropy in nats: H = lse - E_p[z], E_p[z] = scale * sum(e * z_raw) / sum(e); never below 0
+    if (p.out.entropy) p.out.entropy[o] = fmaxf(lse - p.scale * (TZ / S), 0.f);
   }
   // drafted-token logit z[parent(node)][tok[node]]
   float dl = __int_as_float(0x7fc00000), pd = dl;
@@ -344,8 +361,8 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
     const int par = __ldg(p.parent + row0 + node);
     const int tk = __ldg(p.tok + row0 + node);
     if (par >= 0 && par < node && tk >= 0 && tk < p.V) {
-      float Mp, Sp;
-      lm_row_lse(p.partial, stride, static_cast<size_t>(a) * 64 + par, p.n_ranges, p.c, lane, Mp, Sp);
+      float Mp, Sp, Tp;
+      lm_row_lse(p.partial, stride, static_cast<size_t>(a) * 64 + par, p.n_ranges, p.c, lane, Mp, Sp, Tp);
       const uint4* hv = reinterpret_cast<const uint4*>(p.h + (row0 + par) * p.d);
       const uint4* wv = reinterpret_cast<const uint4*>(p.W + static_cast<long long>(tk) * p.d);
       float acc = 0.f;

@@ -56,7 +56,7 @@ def run_lmhead(dev, cfg: gen.VerifyConfig, logit_scale=None):
     return {k: v.cpu().numpy() for k, v in st.items()}
 
 
-def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None):
+def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None, criterion=0):
     from paper_2601_23180_b200 import binding as ts
     B, T = parent.shape
     st = {
@@ -64,10 +64,13 @@ def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None):
         "p_top2": torch.from_numpy(np.asarray(stats_np["p_top2"], dtype=np.float32)).cuda(),
         "top1_idx": i32_dev(stats_np["top1_idx"]),
     }
+    if "entropy" in stats_np:
+        st["entropy"] = torch.from_numpy(np.asarray(stats_np["entropy"], dtype=np.float32)).cuda()
     out = ts.alloc_scan_out(B, T)
     act = None if active is None else torch.from_numpy(np.asarray(active, dtype=np.uint8)).cuda()
     sn = None if start_node is None else i32_dev(start_node)
-    a = ts.scan_args(st, i32_dev(parent), i32_dev(tok), lam, mode, out, active=act, start_node=sn)
+    a = ts.scan_args(st, i32_dev(parent), i32_dev(tok), lam, mode, out, active=act, start_node=sn,
+                     criterion=criterion)
     ts.trispec_accept_scan(a)
     torch.cuda.synchronize()
     return {k: v.cpu().numpy() for k, v in out.items()}
@@ -109,6 +112,10 @@ def check_stats(gpu, ref, seqs, T, near_tie=1e-3):
                 g, e = float(gpu[k][b, r]), float(ref[k][b, r])
                 assert abs(g - e) <= max(1e-3 * e, 1e-9), (k, b, r, g, e)
             assert abs(gpu["top2_val"][b, r] - ref["top2_val"][b, r]) <= 1e-3 * max(1.0, abs(ref["top2_val"][b, r]))
+            if "entropy" in gpu and "entropy" in ref:
+                # H = lse - E_p[z]: the difference of two O(10) fp32 quantities, hence an absolute bound
+                assert abs(gpu["entropy"][b, r] - ref["entropy"][b, r]) <= 1e-3 * max(1.0, ref["entropy"][b, r]), \
+                    ("entropy", b, r, gpu["entropy"][b, r], ref["entropy"][b, r])
             if r >= 1:
                 g, e = float(gpu["p_draft"][b, r]), float(ref["p_draft"][b, r])
                 assert abs(g - e) <= max(1e-3 * e, 1e-9), ("p_draft", b, r, g, e)

@@ -67,6 +67,34 @@ def test_scan_bit_exact_on_oracle_stats(H, name, B, mode):
             assert np.array_equal(got["esc_index"], ref["esc_index"])
 
 
+@pytest.mark.parametrize("crit,lam", [(1, 0.6), (2, 1.5)])
+def test_scan_routing_criteria_bit_exact(H, crit, lam):
+    """Top-1-probability and entropy routing (the routing-criteria study) on fp32 statistics given to
+    both sides: bit-exact except sequences that visit a feature within 1e-3 of the threshold."""
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=41, seed=6)
+    B, T = cfg.B, cfg.T
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(B)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(B)])
+    g = np.random.default_rng(2)
+    top1 = g.integers(0, cfg.V, size=(B, T))
+    for b in range(B):
+        for i in range(T):
+            kids = np.nonzero(parent[b] == i)[0]
+            if len(kids) and g.random() < 0.85:
+                top1[b, i] = tok[b, g.choice(kids)]
+    st = {"p_top1": g.uniform(0.3, 1.0, size=(B, T)).astype(np.float32),
+          "p_top2": g.uniform(0.0, 0.3, size=(B, T)).astype(np.float32),
+          "entropy": g.uniform(0.0, 3.0, size=(B, T)).astype(np.float32), "top1_idx": top1}
+    ref = orc.accept_scan(st["p_top1"].astype(np.float64), st["p_top2"].astype(np.float64), top1, parent, tok, lam,
+                          criterion=crit, entropy=st["entropy"].astype(np.float64))
+    got = H.run_scan(st, parent, tok, lam, gen.MODE_PROXY, criterion=crit)
+    clean = ref["near_thr"] == 0
+    assert clean.sum() >= B - 3 and ref["escalate"].any() and not ref["escalate"].all()
+    for k in ("accept_len", "escalate", "bonus_tok", "last_node", "path"):
+        assert np.array_equal(got[k][clean], ref[k][clean]), k
+    assert np.array_equal(got["near_thr"], ref["near_thr"])
+
+
 def test_scan_start_node_and_large_batch(H):
     cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=3000, V=512, d=64, rho=0.2,
                             logit_scale=3.6 / (0.02 * 8.0))
