@@ -373,3 +373,138 @@ def commit_kv(k_cache: np.ndarray, v_cache: np.ndarray, ctx_len: np.ndarray, k_t
                 vc[blk, t % block_size] = v_tree[b, node]
         new_len[b] = L + len(nodes)
     return kc, vc, new_len
+
+
+# ----------------------------------------------------------------------------------------
+# stochastic acceptance (Eq. 6 at temperature 1) and bonus sampling (Algorithm 1:
+# x_bonus ~ p_{tau_a + 1})
+# ----------------------------------------------------------------------------------------
+def accept_scan_stochastic(p_top1: np.ndarray, p_top2: np.ndarray, p_draft: np.ndarray,
+                           q_draft: np.ndarray, u: np.ndarray, parent: np.ndarray, tok: np.ndarray,
+                           lam: float, mode: int = MODE_PROXY, active: Optional[np.ndarray] = None,
+                           near_eps: float = 1e-3) -> Dict[str, np.ndarray]:
+    """The walk of accept_scan with the Bernoulli acceptance of Eq. 6 in place of the arg-max
+    match: a drafted child c is accepted iff u[c] < min(1, p_draft[c] / q_draft[c]), where
+    p_draft[c] is the verifier's probability of tok[c] at c's parent, q_draft[c] the drafter's,
+    and u[c] a uniform number in [0, 1) supplied by the caller.
+    Readings: the paper states the rule for a chain; on a tree the children of the current node
+    are tried in node order and the first accepted one is taken. When no child is accepted the
+    round ends in case (i) and the bonus token has to be SAMPLED from the current node's
+    distribution (Algorithm 1), which this function cannot do from statistics: it returns
+    bonus_tok = -2 for "sample at last_node". The margin test precedes the children as in
+    accept_scan. Outputs as accept_scan (without the escalation list)."""
+    parent = np.asarray(parent)
+    B, T = parent.shape
+    res = {"accept_len": np.zeros(B, dtype=np.int32), "escalate": np.zeros(B, dtype=np.uint8),
+           "bonus_tok": np.full(B, -1, dtype=np.int32), "path": np.full((B, T), -1, dtype=np.int32),
+           "last_node": np.full(B, -1, dtype=np.int32), "near_thr": np.zeros(B, dtype=np.int32)}
+    for b in range(B):
+        if active is not None and not active[b]:
+            continue
+        cur, n = 0, 0
+        while True:
+            if mode == MODE_PROXY:
+                margin = float(p_top1[b, cur]) - float(p_top2[b, cur])
+                if abs(margin - lam) < near_eps:
+                    res["near_thr"][b] += 1
+                if not (margin >= lam):
+                    res["escalate"][b] = 1
+                    break
+            nxt = -1
+            for c in range(cur + 1, T):
+                if int(parent[b, c]) != cur:
+                    continue
+                ratio = min(1.0, float(p_draft[b, c]) / float(q_draft[b, c])) if q_draft[b, c] > 0 else 1.0
+                if float(u[b, c]) < ratio:
+                    nxt = c
+                    break
+            if nxt < 0:
+                res["bonus_tok"][b] = -2
+                break
+            res["path"][b, n] = nxt
+            n += 1
+            cur = nxt
+        res["accept_len"][b] = n
+        res["last_node"][b] = cur
+    return res
+
+
+_PHILOX_M0, _PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(counter: Sequence[int], key: Sequence[int]) -> Tuple[int, int, int, int]:
+    """Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy
+    as 1, 2, 3", SC'11): a counter-based generator, 128-bit counter and 64-bit key -> four 32-bit
+    words. Written from the published definition."""
+    c0, c1, c2, c3 = (int(x) & 0xFFFFFFFF for x in counter)
+    k0, k1 = (int(x) & 0xFFFFFFFF for x in key)
+    for _ in range(10):
+        p0 = _PHILOX_M0 * c0
+        p1 = _PHILOX_M1 * c2
+        hi0, lo0 = p0 >> 32, p0 & 0xFFFFFFFF
+        hi1, lo1 = p1 >> 32, p1 & 0xFFFFFFFF
+        c0, c1, c2, c3 = (hi1 ^ c1 ^ k0) & 0xFFFFFFFF, lo1, (hi0 ^ c3 ^ k1) & 0xFFFFFFFF, lo0
+        k0 = (k0 + _PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + _PHILOX_W1) & 0xFFFFFFFF
+    return c0, c1, c2, c3
+
+
+def gumbel_noise(seed: int, step: int, b: int, v: int) -> float:
+    """Standard Gumbel variate of vocabulary entry v of sequence b in round `step`:
+    word (v mod 4) of philox4x32_10(counter = (v div 4, b, step low, step high), key = seed) is
+    turned into u = (word + 0.5) / 2^32 in (0, 1), and G = -ln(-ln u)."""
+    w = philox4x32_10((v >> 2, b, step & 0xFFFFFFFF, (step >> 32) & 0xFFFFFFFF),
+                      (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))[v & 3]
+    uu = (w + 0.5) / 4294967296.0
+    return -np.log(-np.log(uu))
+
+
+def gumbel_noise_row(seed: int, step: int, b: int, V: int) -> np.ndarray:
+    """gumbel_noise(seed, step, b, v) for v = 0..V-1, with the same rounds written on numpy
+    arrays (checked against the scalar form in the tests)."""
+    nblk = (V + 3) // 4
+    m32 = np.uint64(0xFFFFFFFF)
+    c0 = np.arange(nblk, dtype=np.uint64)
+    c1 = np.full(nblk, b & 0xFFFFFFFF, dtype=np.uint64)
+    c2 = np.full(nblk, step & 0xFFFFFFFF, dtype=np.uint64)
+    c3 = np.full(nblk, (step >> 32) & 0xFFFFFFFF, dtype=np.uint64)
+    k0, k1 = seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF
+    for _ in range(10):
+        p0 = np.uint64(_PHILOX_M0) * c0
+        p1 = np.uint64(_PHILOX_M1) * c2
+        hi0, lo0 = p0 >> np.uint64(32), p0 & m32
+        hi1, lo1 = p1 >> np.uint64(32), p1 & m32
+        c0, c1, c2, c3 = (hi1 ^ c1 ^ np.uint64(k0)) & m32, lo1, (hi0 ^ c3 ^ np.uint64(k1)) & m32, lo0
+        k0 = (k0 + _PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + _PHILOX_W1) & 0xFFFFFFFF
+    words = np.stack([c0, c1, c2, c3], axis=1).reshape(-1)[:V].astype(np.float64)
+    uu = (words + 0.5) / 4294967296.0
+    return -np.log(-np.log(uu))
+
+
+def sample_bonus(h: np.ndarray, W: np.ndarray, logit_scale: float, node: np.ndarray, seed: int, step: int,
+                 W64: Optional[np.ndarray] = None):
+    """x_bonus ~ softmax(z) at row (b, node[b]) by the Gumbel-max identity: argmax_v (z_v + G_v)
+    with independent standard Gumbel G_v is a sample of softmax(z). node[b] < 0 skips the
+    sequence (-1 returned). Also returns the winning perturbed value and its margin over the
+    runner-up (for the near-tie accounting of the parity tests). h is [B][T][d], W [V][d] bf16 bits."""
+    B = h.shape[0]
+    if W64 is None:
+        W64 = bf16_to_f64(W)
+    V = W64.shape[0]
+    tok = np.full(B, -1, dtype=np.int64)
+    best = np.full(B, np.nan)
+    gap = np.full(B, np.nan)
+    for b in range(B):
+        if int(node[b]) < 0:
+            continue
+        z = row_logits(h[b, int(node[b])], W64, logit_scale)
+        g = gumbel_noise_row(seed, step, b, V)
+        y = z + g
+        i1 = int(np.argmax(y))
+        tok[b], best[b] = i1, y[i1]
+        y2 = y.copy()
+        y2[i1] = -np.inf
+        gap[b] = y[i1] - y2.max()
+    return tok, best, gap

@@ -288,3 +288,75 @@ def test_scan_criteria_reduce_to_known_cases(crit):
         m = orc.accept_scan(p1, np.zeros_like(p2), top1, parent, tok, lam)
         for k in ("accept_len", "escalate", "bonus_tok", "path"):
             assert np.array_equal(m[k], r[k])
+
+
+# ------------------------------------------------------------------------------ stochastic acceptance, sampling
+def test_philox_known_answers_and_vector_form():
+    # known-answer vectors of Philox-4x32-10 (Random123 distribution, kat_vectors)
+    kat = [((0, 0, 0, 0), (0, 0), "6627e8d5 e169c58d bc57ac4c 9b00dbd8"),
+           ((0xffffffff,) * 4, (0xffffffff,) * 2, "408f276d 41c83b0e a20bc7c6 6d5451fd"),
+           ((0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344), (0xa4093822, 0x299f31d0),
+            "d16cfe09 94fdcceb 5001e420 24126ea1")]
+    for c, k, want in kat:
+        assert " ".join("%08x" % x for x in orc.philox4x32_10(c, k)) == want
+    row = orc.gumbel_noise_row(0x1234567890abcdef, 5, 3, 37)
+    for v in (0, 1, 2, 3, 4, 17, 36):
+        assert row[v] == orc.gumbel_noise(0x1234567890abcdef, 5, 3, v)
+    assert np.isfinite(row).all()
+
+
+def test_gumbel_max_samples_the_softmax():
+    """Over many rounds the sampled tokens follow softmax(z) (Gumbel-max identity): 5 tokens,
+    20000 draws, every frequency within 4 standard deviations."""
+    z = np.array([1.0, 0.0, -1.0, 2.0, 0.5])
+    p = np.exp(z) / np.exp(z).sum()
+    n = 20000
+    counts = np.zeros(5)
+    for step in range(n // 8):
+        for b in range(8):
+            counts[np.argmax(z + orc.gumbel_noise_row(99, step, b, 5))] += 1
+    assert np.all(np.abs(counts / n - p) < 4 * np.sqrt(p * (1 - p) / n))
+
+
+def test_stochastic_scan_special_cases_and_acceptance_probability():
+    cfg = _cfg(B=4, seed=12)
+    B, T = 4, cfg.T
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(B)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(B)])
+    g = np.random.default_rng(3)
+    p1, p2 = np.ones((B, T)), np.zeros((B, T))                       # always trusted
+    pd = g.uniform(0.05, 0.9, size=(B, T))
+    u = g.uniform(0, 1, size=(B, T))
+    # q = p: ratio 1, every first child is accepted down to a leaf; bonus has to be sampled
+    r = orc.accept_scan_stochastic(p1, p2, pd, pd, u, parent, tok, 0.5)
+    for b in range(B):
+        cur, want = 0, []
+        while (parent[b] == cur).any():
+            cur = int(np.nonzero(parent[b] == cur)[0][0])
+            want.append(cur)
+        assert r["path"][b, :len(want)].tolist() == want and r["accept_len"][b] == len(want)
+        assert r["bonus_tok"][b] == -2 and r["escalate"][b] == 0
+    # p = 0: nothing is accepted; u = 0 with p > 0: same as q = p
+    r0 = orc.accept_scan_stochastic(p1, p2, np.zeros((B, T)), pd, u, parent, tok, 0.5)
+    assert (r0["accept_len"] == 0).all() and (r0["bonus_tok"] == -2).all()
+    ru = orc.accept_scan_stochastic(p1, p2, pd, 5 * pd, np.zeros((B, T)), parent, tok, 0.5)
+    assert np.array_equal(ru["path"], r["path"])
+    # untrusted root escalates before any Bernoulli test
+    re = orc.accept_scan_stochastic(np.full((B, T), 0.3), p2, pd, pd, u, parent, tok, 0.5)
+    assert re["escalate"].all() and (re["accept_len"] == 0).all() and (re["bonus_tok"] == -1).all()
+    # chain: P(tau_a >= j) = prod_{i<=j} min(1, p_i / q_i) (Eq. 6, Eq. 7), by Monte Carlo
+    Tc = 6
+    cp = np.arange(-1, Tc - 1, dtype=np.int32)[None]
+    ct = np.arange(Tc, dtype=np.int32)[None]
+    ratio = np.array([1.0, 0.9, 0.5, 1.0, 0.8, 0.3])                  # entry 0 unused (root)
+    pdc, qdc = np.minimum(ratio, 1.0)[None] * 0.5, np.full((1, Tc), 0.5)
+    n = 20000
+    lens = np.zeros(Tc, dtype=int)
+    uu = np.random.default_rng(8).uniform(0, 1, size=(n, Tc))
+    for t in range(n):
+        rr = orc.accept_scan_stochastic(np.ones((1, Tc)), np.zeros((1, Tc)), pdc, qdc, uu[t:t + 1], cp, ct, 0.5)
+        lens[rr["accept_len"][0]] += 1
+    surv = np.cumprod(ratio[1:])                                      # P(tau_a >= j), j = 1..5
+    for j in range(1, Tc):
+        pj = surv[j - 1]
+        assert abs(lens[j:].sum() / n - pj) < 4 * np.sqrt(pj * (1 - pj) / n) + 1e-9
