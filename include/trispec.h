@@ -187,6 +187,13 @@ int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream);
  *      the accepted tokens so far are x_{1:tau_m}); else the child whose token equals
  *      top1_idx is accepted and the walk continues; no such child -> approve (case (i)),
  *      bonus_tok = top1_idx of the current node. TARGET mode: no margin test.
+ *    Stochastic acceptance (Eq. 6 at temperature 1), when q_draft and u_accept (f32 [B][T],
+ *      indexed by child node) are given: child c of the current node is accepted iff
+ *      u_accept[c] < min(1, in.p_draft[c] / q_draft[c]) (q_draft = the drafter's probability of
+ *      tok[c], u_accept = the caller's uniform numbers in [0, 1)); the children are tried in
+ *      node order and the first accepted one is taken. When none is accepted the round ends in
+ *      case (i) with bonus_tok = -2: the bonus token has to be sampled at last_node
+ *      (trispec_sample_bonus). The decision is taken in fp32 (IEEE division).
  *    active (optional uint8 [B]): sequences with 0 are skipped (outputs: accept_len 0,
  *      escalate 0, bonus -1, last_node -1, path -1).
  *    Outputs: accept_len, bonus_tok, last_node, near_thr int32 [B]; escalate uint8 [B];
@@ -206,6 +213,7 @@ typedef struct {
   trispec_stats in;          /* read: top1_idx, and p_top1, p_top2 or entropy as the criterion needs */
   const uint8_t* active;
   const int32_t* start_node;
+  const float *q_draft, *u_accept;  /* both NULL: greedy acceptance; both set: Eq. 6 at temperature 1 */
   int32_t *accept_len, *bonus_tok, *path, *last_node, *near_thr, *n_escalated, *esc_index;
   uint8_t* escalate;
 } trispec_scan_args;

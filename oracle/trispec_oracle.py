@@ -414,8 +414,10 @@ def accept_scan_stochastic(p_top1: np.ndarray, p_top2: np.ndarray, p_draft: np.n
             for c in range(cur + 1, T):
                 if int(parent[b, c]) != cur:
                     continue
-                ratio = min(1.0, float(p_draft[b, c]) / float(q_draft[b, c])) if q_draft[b, c] > 0 else 1.0
-                if float(u[b, c]) < ratio:
+                # in the arrays' own precision (fp32 inputs give the fp32 decision the kernel takes)
+                one = p_draft.dtype.type(1)
+                ratio = min(one, p_draft[b, c] / q_draft[b, c]) if q_draft[b, c] > 0 else one
+                if u[b, c] < ratio:
                     nxt = c
                     break
             if nxt < 0:

@@ -55,7 +55,8 @@ class LmheadArgs(C.Structure):
 
 class ScanArgs(C.Structure):
     _fields_ = [("B", _i), ("T", _i), ("lam", _f), ("mode", _i), ("criterion", _i), ("parent", _vp), ("tok", _vp),
-                ("stats", Stats), ("active", _vp), ("start_node", _vp), ("accept_len", _vp),
+                ("stats", Stats), ("active", _vp), ("start_node", _vp), ("q_draft", _vp), ("u_accept", _vp),
+                ("accept_len", _vp),
                 ("bonus_tok", _vp), ("path", _vp), ("last_node", _vp), ("near_thr", _vp),
                 ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
 
@@ -202,13 +203,14 @@ CRIT_MARGIN, CRIT_TOP1, CRIT_ENTROPY = 0, 1, 2
 
 
 def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], active=None,
-              start_node=None, criterion=CRIT_MARGIN) -> ScanArgs:
+              start_node=None, criterion=CRIT_MARGIN, q_draft=None, u_accept=None) -> ScanArgs:
     B, T = parent.shape
     a = ScanArgs()
     a.B, a.T, a.lam, a.mode, a.criterion = B, T, float(lam), int(mode), int(criterion)
     a.parent, a.tok = _p(parent), _p(tok)
     a.stats = _stats_struct(stats)
     a.active, a.start_node = _p(active), _p(start_node)
+    a.q_draft, a.u_accept = _p(q_draft), _p(u_accept)
     for k in ("accept_len", "bonus_tok", "path", "last_node", "near_thr", "n_escalated", "esc_index", "escalate"):
         setattr(a, k, _p(out.get(k)))
     return a

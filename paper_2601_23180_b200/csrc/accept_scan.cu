@@ -73,6 +73,21 @@ accept_scan_kernel(trispec_scan_args a) {
       __ballot_sync(0xffffffffu, tr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, tr1)) << 32);
   const unsigned long long near_bits =
       __ballot_sync(0xffffffffu, nr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, nr1)) << 32);
+  // Bernoulli acceptance of Eq. 6 for every node at once: bit c = child c passes its test
+  const bool stochastic = a.q_draft != nullptr;
+  unsigned long long passes = ~0ull;
+  if (stochastic) {
+    bool ps0 = false, ps1 = false;
+    if (has0 && lane > 0) {
+      const float q = __ldg(a.q_draft + base + lane), pd = __ldg(a.in.p_draft + base + lane);
+      ps0 = __ldg(a.u_accept + base + lane) < ((q > 0.f) ? fminf(1.f, pd / q) : 1.f);
+    }
+    if (has1) {
+      const float q = __ldg(a.q_draft + base + lane + 32), pd = __ldg(a.in.p_draft + base + lane + 32);
+      ps1 = __ldg(a.u_accept + base + lane + 32) < ((q > 0.f) ? fminf(1.f, pd / q) : 1.f);
+    }
+    passes = __ballot_sync(0xffffffffu, ps0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, ps1)) << 32);
+  }
   // the compaction kernel only writes the leading entries of esc_index
   if (a.esc_index && lane == 0) a.esc_index[b] = -1;
 
@@ -89,12 +104,14 @@ accept_scan_kernel(trispec_scan_args a) {
       near += static_cast<int>((near_bits >> cur) & 1ull);
       if (!((trusted >> cur) & 1ull)) { esc = 1; break; }
     }
-    const unsigned m0 = __ballot_sync(0xffffffffu, par0 == cur && tok0 == top1);
-    const unsigned m1 = __ballot_sync(0xffffffffu, par1 == cur && tok1 == top1);
+    // greedy: the child whose token is the arg-max; stochastic: the first child that passed
+    unsigned m0 = __ballot_sync(0xffffffffu, par0 == cur && (stochastic || tok0 == top1));
+    unsigned m1 = __ballot_sync(0xffffffffu, par1 == cur && (stochastic || tok1 == top1));
+    if (stochastic) { m0 &= static_cast<unsigned>(passes); m1 &= static_cast<unsigned>(passes >> 32); }
     int nxt = -1;
     if (m0) nxt = __ffs(m0) - 1;
     else if (m1) nxt = 32 + __ffs(m1) - 1;
-    if (nxt < 0) { bonus = top1; break; }
+    if (nxt < 0) { bonus = stochastic ? -2 : top1; break; }
     if (lane == n) path0 = nxt;
     if (lane + 32 == n) path1 = nxt;
     ++n;
@@ -207,6 +224,8 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
     if (a->criterion == TRISPEC_CRIT_ENTROPY && !a->in.entropy) return TRISPEC_ERR_INVALID_ARG;
   }
   if ((a->n_escalated == nullptr) != (a->esc_index == nullptr)) return TRISPEC_ERR_INVALID_ARG;
+  if ((a->q_draft == nullptr) != (a->u_accept == nullptr)) return TRISPEC_ERR_INVALID_ARG;
+  if (a->q_draft && !a->in.p_draft) return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int per_block = kScanThreads / 32;
   unsigned grid = static_cast<unsigned>((static_cast<long long>(a->B) + per_block - 1) / per_block);

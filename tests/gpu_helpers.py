@@ -56,7 +56,8 @@ def run_lmhead(dev, cfg: gen.VerifyConfig, logit_scale=None):
     return {k: v.cpu().numpy() for k, v in st.items()}
 
 
-def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None, criterion=0):
+def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None, criterion=0, q_draft=None,
+             u_accept=None):
     from paper_2601_23180_b200 import binding as ts
     B, T = parent.shape
     st = {
@@ -64,13 +65,16 @@ def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None, cri
         "p_top2": torch.from_numpy(np.asarray(stats_np["p_top2"], dtype=np.float32)).cuda(),
         "top1_idx": i32_dev(stats_np["top1_idx"]),
     }
+    f32 = lambda x: None if x is None else torch.from_numpy(np.asarray(x, dtype=np.float32)).cuda()
+    if "p_draft" in stats_np:
+        st["p_draft"] = f32(stats_np["p_draft"])
     if "entropy" in stats_np:
         st["entropy"] = torch.from_numpy(np.asarray(stats_np["entropy"], dtype=np.float32)).cuda()
     out = ts.alloc_scan_out(B, T)
     act = None if active is None else torch.from_numpy(np.asarray(active, dtype=np.uint8)).cuda()
     sn = None if start_node is None else i32_dev(start_node)
     a = ts.scan_args(st, i32_dev(parent), i32_dev(tok), lam, mode, out, active=act, start_node=sn,
-                     criterion=criterion)
+                     criterion=criterion, q_draft=f32(q_draft), u_accept=f32(u_accept))
     ts.trispec_accept_scan(a)
     torch.cuda.synchronize()
     return {k: v.cpu().numpy() for k, v in out.items()}

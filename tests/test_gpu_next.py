@@ -175,3 +175,31 @@ def test_round_then_prune_and_commit_on_one_stream():
     assert np.array_equal(ctx_out.cpu().numpy(), ref_len)
     assert np.array_equal(bits(pas.dev["k_cache"]), ref_k) and np.array_equal(bits(pas.dev["v_cache"]), ref_v)
     assert scan["escalate"].sum() >= 1 and (scan["accept_len"] > 0).any()
+
+
+@pytest.mark.parametrize("mode", [gen.MODE_PROXY, gen.MODE_TARGET])
+def test_stochastic_acceptance_bit_exact(mode):
+    """Eq. 6 at temperature 1 on fp32 inputs given to both sides; the oracle takes the Bernoulli
+    decision in fp32 as the kernel does, so every sequence must agree (near-threshold margins excepted)."""
+    import tests.gpu_helpers as H
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=53, seed=8)
+    B, T = cfg.B, cfg.T
+    parent = np.stack([gen.make_tree(cfg, b) for b in range(B)])
+    tok = np.stack([gen.make_tokens(cfg, b, parent[b]) for b in range(B)])
+    g = np.random.default_rng(4)
+    st = {"p_top1": g.uniform(0.4, 1.0, size=(B, T)).astype(np.float32),
+          "p_top2": g.uniform(0.0, 0.2, size=(B, T)).astype(np.float32),
+          "p_draft": g.uniform(0.0, 0.8, size=(B, T)).astype(np.float32),
+          "top1_idx": g.integers(0, cfg.V, size=(B, T))}
+    q = g.uniform(0.05, 0.9, size=(B, T)).astype(np.float32)
+    q[:, 5] = 0.0                                             # drafter probability 0: ratio taken as 1
+    u = g.uniform(0, 1, size=(B, T)).astype(np.float32)
+    ref = orc.accept_scan_stochastic(st["p_top1"], st["p_top2"], st["p_draft"], q, u, parent, tok, 0.5, mode=mode)
+    got = H.run_scan(st, parent, tok, 0.5, mode, q_draft=q, u_accept=u)
+    clean = ref["near_thr"] == 0
+    assert clean.sum() >= B - 2
+    for k in ("accept_len", "escalate", "bonus_tok", "last_node", "path"):
+        assert np.array_equal(got[k][clean], ref[k][clean]), k
+    assert (ref["accept_len"] > 0).any() and (ref["bonus_tok"] == -2).any()
+    if mode == gen.MODE_PROXY:
+        assert ref["escalate"].any()
