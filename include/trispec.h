@@ -17,6 +17,7 @@
  *   5. trispec_prune_tree       the branches that remain for the target after the proxy
  *                               accepted a prefix (routing case (ii), token pruning)
  *   6. trispec_commit_kv        append the accepted path's keys/values to the KV cache
+ *   7. trispec_sample_bonus     draw the bonus token from a node's distribution (temperature 1)
  *
  * Conventions
  *   - Every data pointer is a DEVICE pointer owned by the caller unless a comment says
@@ -275,6 +276,36 @@ typedef struct {
   int32_t* dev_status;
 } trispec_commit_args;
 int trispec_commit_kv(const trispec_commit_args* a, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * 7. Bonus sampling (Algorithm 1: x_bonus ~ p_{tau_a + 1}; needed at temperature 1, where the
+ *    stochastic scan ends case (i) with bonus_tok = -2). For every sequence whose bonus_tok[b]
+ *    equals -2, a token is drawn from softmax(logit_scale * h[b][last_node[b]] . W^T) by the
+ *    Gumbel-max identity: argmax_v (z_v + G_v), G_v independent standard Gumbel variates
+ *    (ties -> lowest index). The noise is counter-based and reproducible: word (v mod 4) of
+ *    Philox-4x32-10 with counter (v div 4, b, step low, step high) and key (seed low, seed high)
+ *    gives u = ((word >> 9) + 0.5) / 2^23 and G = -ln(-ln u). One more pass over W, no logits
+ *    in global memory.
+ *      h [B*T][d], W [V][d] bf16 as in trispec_lmhead_stats; last_node [B] int32.
+ *      bonus_tok [B] int32, in/out: entries equal to -2 are replaced by the sampled token;
+ *        other entries are left alone. sample_value (optional f32 [B]): the winning z_v + G_v.
+ *      seed, step: the caller advances `step` every round.
+ *      workspace: >= trispec_sample_bonus_workspace(a) bytes, 256-byte aligned.
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int B, T, d, V;
+  float logit_scale;
+  const void *h, *W;
+  const int32_t* last_node;
+  int32_t* bonus_tok;
+  float* sample_value;
+  unsigned long long seed, step;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+} trispec_sample_args;
+size_t trispec_sample_bonus_workspace(const trispec_sample_args* a);
+int trispec_sample_bonus(const trispec_sample_args* a, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * Fused pass: the four calls above in order on `stream` (one verification round of

@@ -455,10 +455,11 @@ def philox4x32_10(counter: Sequence[int], key: Sequence[int]) -> Tuple[int, int,
 def gumbel_noise(seed: int, step: int, b: int, v: int) -> float:
     """Standard Gumbel variate of vocabulary entry v of sequence b in round `step`:
     word (v mod 4) of philox4x32_10(counter = (v div 4, b, step low, step high), key = seed) is
-    turned into u = (word + 0.5) / 2^32 in (0, 1), and G = -ln(-ln u)."""
+    turned into u = ((word >> 9) + 0.5) / 2^23, which lies strictly inside (0, 1) and is exact in
+    fp32 as well, and G = -ln(-ln u)."""
     w = philox4x32_10((v >> 2, b, step & 0xFFFFFFFF, (step >> 32) & 0xFFFFFFFF),
                       (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))[v & 3]
-    uu = (w + 0.5) / 4294967296.0
+    uu = ((w >> 9) + 0.5) / 8388608.0
     return -np.log(-np.log(uu))
 
 
@@ -480,8 +481,8 @@ def gumbel_noise_row(seed: int, step: int, b: int, V: int) -> np.ndarray:
         c0, c1, c2, c3 = (hi1 ^ c1 ^ np.uint64(k0)) & m32, lo1, (hi0 ^ c3 ^ np.uint64(k1)) & m32, lo0
         k0 = (k0 + _PHILOX_W0) & 0xFFFFFFFF
         k1 = (k1 + _PHILOX_W1) & 0xFFFFFFFF
-    words = np.stack([c0, c1, c2, c3], axis=1).reshape(-1)[:V].astype(np.float64)
-    uu = (words + 0.5) / 4294967296.0
+    words = (np.stack([c0, c1, c2, c3], axis=1).reshape(-1)[:V] >> np.uint64(9)).astype(np.float64)
+    uu = (words + 0.5) / 8388608.0
     return -np.log(-np.log(uu))
 
 

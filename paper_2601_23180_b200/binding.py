@@ -74,6 +74,12 @@ class CommitArgs(C.Structure):
                 ("path", _vp), ("accept_len", _vp), ("active", _vp), ("ctx_len_out", _vp), ("dev_status", _vp)]
 
 
+class SampleArgs(C.Structure):
+    _fields_ = [("B", _i), ("T", _i), ("d", _i), ("V", _i), ("logit_scale", _f), ("h", _vp), ("W", _vp),
+                ("last_node", _vp), ("bonus_tok", _vp), ("sample_value", _vp), ("seed", C.c_ulonglong),
+                ("step", C.c_ulonglong), ("workspace", _vp), ("workspace_bytes", _sz), ("dev_status", _vp)]
+
+
 class HostIO(C.Structure):
     _fields_ = [(n, _vp) for n in ("parent", "tok", "q", "k_tree", "v_tree", "h", "accept_len", "bonus_tok",
                                    "last_node", "path", "escalate")]
@@ -93,6 +99,9 @@ _lib.trispec_lmhead_stats_noalloc.argtypes = [C.POINTER(LmheadArgs), _vp]
 _lib.trispec_accept_scan.argtypes = [C.POINTER(ScanArgs), _vp]
 _lib.trispec_prune_tree.argtypes = [C.POINTER(PruneArgs), _vp]
 _lib.trispec_commit_kv.argtypes = [C.POINTER(CommitArgs), _vp]
+_lib.trispec_sample_bonus_workspace.restype = _sz
+_lib.trispec_sample_bonus_workspace.argtypes = [C.POINTER(SampleArgs)]
+_lib.trispec_sample_bonus.argtypes = [C.POINTER(SampleArgs), _vp]
 _lib.trispec_verify.argtypes = [C.POINTER(TreeArgs), C.POINTER(AttnArgs), C.POINTER(LmheadArgs),
                                 C.POINTER(ScanArgs), _vp]
 
@@ -102,7 +111,7 @@ _lib.trispec_verify_host.argtypes = [C.POINTER(HostIO), C.POINTER(TreeArgs), C.P
 EXPORTS = ["trispec_verify_host", "trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
            "trispec_verify_attn_workspace", "trispec_verify_attn", "trispec_lmhead_stats_workspace",
            "trispec_lmhead_stats", "trispec_lmhead_stats_noalloc", "trispec_accept_scan", "trispec_verify",
-           "trispec_prune_tree", "trispec_commit_kv"]
+           "trispec_prune_tree", "trispec_commit_kv", "trispec_sample_bonus_workspace", "trispec_sample_bonus"]
 
 
 class TrispecError(RuntimeError):
@@ -281,6 +290,27 @@ def trispec_verify_attn(args: AttnArgs, stream=None):
 
 def trispec_prune_tree(args: PruneArgs, stream=None):
     _check(_lib.trispec_prune_tree(C.byref(args), _stream(stream)))
+
+
+def sample_args(h, W, last_node, bonus_tok, logit_scale, seed, step, sample_value=None, workspace=None,
+                dev_status=None) -> SampleArgs:
+    B, T = last_node.shape[0], h.numel() // (last_node.shape[0] * h.shape[-1])
+    a = SampleArgs()
+    a.B, a.T, a.d, a.V, a.logit_scale = B, T, h.shape[-1], W.shape[0], float(logit_scale)
+    a.h, a.W, a.last_node, a.bonus_tok, a.sample_value = _p(h), _p(W), _p(last_node), _p(bonus_tok), _p(sample_value)
+    a.seed, a.step = int(seed), int(step)
+    a.workspace = _p(workspace)
+    a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a.dev_status = _p(dev_status)
+    return a
+
+
+def trispec_sample_bonus_workspace(args: SampleArgs) -> int:
+    return int(_lib.trispec_sample_bonus_workspace(C.byref(args)))
+
+
+def trispec_sample_bonus(args: SampleArgs, stream=None):
+    _check(_lib.trispec_sample_bonus(C.byref(args), _stream(stream)))
 
 
 def trispec_commit_kv(args: CommitArgs, stream=None):

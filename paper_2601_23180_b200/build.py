@@ -14,7 +14,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtrispec.so")
 STAMP = os.path.join(PKG, "csrc", ".build_stamp")
 SOURCES = ["host_common.cu", "tree_mask.cu", "accept_scan.cu", "lmhead.cu", "attn.cu", "verify.cu", "prune.cu",
-           "kv_commit.cu"]
+           "kv_commit.cu", "sample.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
