@@ -350,6 +350,28 @@ def run_only(args, cfg):
                                  "work_per_launch": byts, "ms_per_launch": ms, "traffic": None}})
         print(json.dumps(out), flush=True)
         return
+    if args.only == "sample":
+        # bonus sampling for every sequence of the workload: one more pass over W
+        inp = gen.make_inputs(cfg, with_attention=False)
+        pas = runner.VerifyPass(cfg, inp, with_attention=False)
+        last = torch.zeros(cfg.B, dtype=torch.int32, device="cuda")
+        bonus = torch.full((cfg.B,), -2, dtype=torch.int32, device="cuda")
+        sa = ts.sample_args(pas.dev["h"], pas.dev["W"], last, bonus, cfg.logit_scale, 1234, 0, dev_status=pas.status)
+        ws = ts.alloc_workspace(ts.trispec_sample_bonus_workspace(sa))
+        sa.workspace, sa.workspace_bytes = ws.data_ptr(), ws.numel()
+
+        def call():
+            bonus.fill_(-2)
+            ts.trispec_sample_bonus(sa)
+        byts = 2.0 * cfg.V * cfg.d + 2.0 * cfg.B * cfg.d
+        ms = timed(call, byts)
+        roof = _roof(peaks, 2.0 * cfg.B * cfg.d * cfg.V, byts, ms)
+        roof["kernel"] = "sample_gemm_kernel (+ gather, finalize, flag reset)"
+        assert int(pas.status.item()) == 0
+        out.update({"value": cfg.B / (ms * 1e-3), "unit": "sampled tokens/s", "ms_per_step": ms, "dtype": "bf16",
+                    "roofline": roof})
+        print(json.dumps(out), flush=True)
+        return
     if args.only == "attention":
         inp = gen.make_inputs(cfg, with_lm_head=False)
         small = dataclasses.replace(cfg, V=4096, d=64)      # the LM head is not run: a token-sized stand-in
@@ -389,7 +411,7 @@ def main():
     ap.add_argument("--workload", default="proxy_tree")
     ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan", "prune", "commit"],
+    ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan", "prune", "commit", "sample"],
                     help="time one entry point alone (L2 flushed before each call) instead of the pass")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the number of sequences of the workload (reduced copies for profiler captures)")
