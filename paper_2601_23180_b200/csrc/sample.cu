@@ -225,6 +225,176 @@ sample_gemm_kernel(const __grid_constant__ CUtensorMap tmap_hc, const __grid_con
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Few sequences (B <= 32): operands swapped. W is the M-side operand (128 vocabulary rows per
+// MMA), the compact rows are the N side (16 or 32 columns), so a pipeline stage is 16 KB of W
+// plus 2-4 KB of Hc and the ring (up to 11 stages) carries almost only W: enough bytes in
+// flight to keep HBM busy, which the 128 x 256 tile above cannot do with its 48 KB stages.
+// TMEM lane = vocabulary entry, column = sequence; each epilogue thread keeps a running best
+// per sequence in registers and the CTA reduces them at the end.
+// ---------------------------------------------------------------------------------------
+constexpr int SW_BM = 128, SW_BK = 64, SW_MAX_STAGES = 12, SW_MAX_SEQ = 32;
+constexpr int SW_A_BYTES = SW_BM * SW_BK * 2;           // 16 KB of W per stage
+
+struct SampleSwapParams {
+  SampleParams base;
+  int N;            // sequence columns: 16 or 32
+  int stages, stage_bytes;
+};
+
+__global__ void __launch_bounds__(SM_THREADS, 1)
+sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_hc,
+                           const SampleSwapParams sp) {
+  pdl_launch_dependents();
+  const SampleParams& p = sp.base;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sp.stages * sp.stage_bytes);
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = bars + SW_MAX_STAGES;
+  uint64_t* tmem_full = bars + 2 * SW_MAX_STAGES;
+  uint64_t* tmem_empty = bars + 2 * SW_MAX_STAGES + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SW_MAX_STAGES + 4);
+  float* red_y = reinterpret_cast<float*>(bars + 2 * SW_MAX_STAGES + 6);    // [4 warps][32 sequences]
+  int* red_i = reinterpret_cast<int*>(red_y + 4 * SW_MAX_SEQ);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int range = blockIdx.x;
+  // vocabulary rows of this CTA: 128-row tiles of an equal share (in units of 16 rows)
+  const int V16 = (p.V + 15) >> 4;
+  const int u0 = static_cast<int>((static_cast<long long>(V16) * range) / p.n_ranges);
+  const int u1 = static_cast<int>((static_cast<long long>(V16) * (range + 1)) / p.n_ranges);
+  const int v_begin = u0 << 4, v_end = min(u1 << 4, p.V);
+  const int n_tiles = (v_end - v_begin + SW_BM - 1) / SW_BM;
+  const int n_kb = p.d / SW_BK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < sp.stages; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 4); }
+    fence_mbar_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, 64);                    // two accumulators of at most 32 columns
+    tmem_relinquish();
+  }
+  if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_hc); prefetch_tmap(&tmap_w); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // the compact rows come from the gather kernel
+
+  if (warp == 4) {
+    if (lane == 0) {   // ---------------------------------------------------------- TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t tx = static_cast<uint32_t>(SW_A_BYTES + sp.N * SW_BK * 2);
+      for (int t = 0; t < n_tiles; ++t) {
+        for (int kb = 0; kb < n_kb; ++kb) {
+          mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
+          uint8_t* sa = smem + stage * sp.stage_bytes;
+          mbar_expect_tx(full_bar + stage, tx);
+          tma_load_2d(sa, &tmap_w, full_bar + stage, kb * SW_BK, v_begin + t * SW_BM);   // rows past V: zero fill
+          tma_load_2d(sa + SW_A_BYTES, &tmap_hc, full_bar + stage, kb * SW_BK, 0);
+          if (++stage == sp.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {   // ---------------------------------------------------------- MMA issuer
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t idesc = idesc_bf16(SW_BM, sp.N, false, false);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int buf = t & 1;
+        mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * 32);
+        for (int kb = 0; kb < n_kb; ++kb) {
+          mbar_wait(full_bar + stage, phase, p.dev_status);
+          tc_fence_after();
+          const uint32_t sa = base_u32 + stage * sp.stage_bytes;
+          const uint64_t adesc = smem_desc_sw128(sa, 1024, 16);
+          const uint64_t bdesc = smem_desc_sw128(sa + SW_A_BYTES, 1024, 16);
+#pragma unroll
+          for (int k = 0; k < SW_BK / 16; ++k) tc_mma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
+          tc_commit(empty_bar + stage);
+          if (++stage == sp.stages) { stage = 0; phase ^= 1u; }
+        }
+        tc_commit(tmem_full + buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3)
+    const int row = warp * 32 + lane;             // TMEM lane = vocabulary entry of the tile
+    unsigned int live_mask = 0;                   // bit b: sequence b wants a sample
+    for (int b = 0; b < p.B; ++b)
+      if (__ldg(p.bonus_tok + b) == -2) live_mask |= 1u << b;
+    float best[SW_MAX_SEQ];
+    int best_idx[SW_MAX_SEQ];
+#pragma unroll
+    for (int b = 0; b < SW_MAX_SEQ; ++b) { best[b] = -INFINITY; best_idx[b] = -1; }
+    const uint2 key = make_uint2(p.seed_lo, p.seed_hi);
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      mbar_wait(tmem_full + buf, (t >> 1) & 1u, p.dev_status);
+      tc_fence_after();
+      uint32_t r[32];
+      tmem_ld32(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(buf * 32), r);
+      tc_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tmem_empty + buf);     // values are in registers: the buffer is free
+      const int v = v_begin + t * SW_BM + row;
+      if (v < v_end) {
+#pragma unroll
+        for (int b = 0; b < SW_MAX_SEQ; ++b) {
+          if ((live_mask >> b) & 1u) {
+            const uint4 w = philox4x32_10(make_uint4(static_cast<unsigned>(v >> 2), static_cast<unsigned>(b),
+                                                     p.step_lo, p.step_hi), key);
+            const unsigned int word = (v & 2) ? ((v & 1) ? w.w : w.z) : ((v & 1) ? w.y : w.x);
+            const float y = fmaf(__uint_as_float(r[b]), p.scale, gumbel_from_word(word));
+            if (y > best[b]) { best[b] = y; best_idx[b] = v; }   // ascending v: ties keep the lowest index
+          }
+        }
+      }
+    }
+    // CTA-wide best per sequence: warp shuffles, then the four warps through shared memory
+#pragma unroll
+    for (int b = 0; b < SW_MAX_SEQ; ++b) {
+      if (!((live_mask >> b) & 1u)) continue;     // uniform across the CTA
+      float y = best[b];
+      int i = best_idx[b];
+      for (int o = 16; o > 0; o >>= 1) {
+        const float oy = __shfl_xor_sync(0xffffffffu, y, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+        if (oi >= 0 && (i < 0 || oy > y || (oy == y && oi < i))) { y = oy; i = oi; }
+      }
+      if (lane == 0) { red_y[warp * SW_MAX_SEQ + b] = y; red_i[warp * SW_MAX_SEQ + b] = i; }
+    }
+    asm volatile("bar.sync 2, 128;" ::: "memory");   // the four epilogue warps
+    if (warp == 0 && lane < p.B && ((live_mask >> lane) & 1u)) {
+      float y = red_y[lane];
+      int i = red_i[lane];
+      for (int w2 = 1; w2 < 4; ++w2) {
+        const float oy = red_y[w2 * SW_MAX_SEQ + lane];
+        const int oi = red_i[w2 * SW_MAX_SEQ + lane];
+        if (oi >= 0 && (i < 0 || oy > y || (oy == y && oi < i))) { y = oy; i = oi; }
+      }
+      SamplePartial out;
+      out.y = y; out.idx = i;
+      p.partial[static_cast<size_t>(range) * (p.n_mt * SM_BM) + lane] = out;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 64);
+  }
+}
+
 __global__ void __launch_bounds__(256)
 sample_finalize_kernel(const SampleParams p) {
   pdl_launch_dependents();
@@ -310,14 +480,44 @@ extern "C" int trispec_sample_bonus(const trispec_sample_args* a, void* stream) 
     const uint32_t box[2] = {SM_BK, 64};
     if (!cached_tmap_bf16(&tm_w, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
   }
-  static bool smem_set[64] = {};
-  rc = ensure_smem_limit(reinterpret_cast<const void*>(sample_gemm_kernel), SM_SMEM_BYTES, smem_set);
-  if (rc != TRISPEC_OK) return rc;
   TRISPEC_CUDA_OK(launch_dependent(sample_gather_kernel, static_cast<unsigned>(n_mt * SM_BM), 256, 0, st, 1, p));
   count_launch();
-  TRISPEC_CUDA_OK(launch_dependent(sample_gemm_kernel, static_cast<unsigned>(n_mt * n_ranges), SM_THREADS, SM_SMEM_BYTES,
-                                   st, 1, tm_hc, tm_w, p));
-  count_launch();
+  if (a->B <= SW_MAX_SEQ) {
+    // few sequences: W on the M side, deep ring of small stages
+    SampleSwapParams sp;
+    sp.base = p;
+    sp.N = a->B <= 16 ? 16 : 32;
+    sp.stage_bytes = SW_A_BYTES + sp.N * SW_BK * 2;
+    sp.stages = (224 * 1024) / sp.stage_bytes;
+    if (sp.stages > SW_MAX_STAGES) sp.stages = SW_MAX_STAGES;
+    const int smem_bytes = sp.stages * sp.stage_bytes + 1024 + 2048;
+    CUtensorMap tm_w128, tm_hcn;
+    {
+      const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
+      const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
+      const uint32_t box[2] = {SW_BK, SW_BM};
+      if (!cached_tmap_bf16(&tm_w128, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+    }
+    {
+      const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(n_mt) * SM_BM};
+      const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
+      const uint32_t box[2] = {SW_BK, static_cast<uint32_t>(sp.N)};
+      if (!cached_tmap_bf16(&tm_hcn, p.hc, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+    }
+    static bool smem_set_sw[64] = {};
+    rc = ensure_smem_limit(reinterpret_cast<const void*>(sample_gemm_swapped_kernel), 227 * 1024, smem_set_sw);
+    if (rc != TRISPEC_OK) return rc;
+    TRISPEC_CUDA_OK(launch_dependent(sample_gemm_swapped_kernel, static_cast<unsigned>(n_ranges), SM_THREADS,
+                                     static_cast<size_t>(smem_bytes), st, 1, tm_w128, tm_hcn, sp));
+    count_launch();
+  } else {
+    static bool smem_set[64] = {};
+    rc = ensure_smem_limit(reinterpret_cast<const void*>(sample_gemm_kernel), SM_SMEM_BYTES, smem_set);
+    if (rc != TRISPEC_OK) return rc;
+    TRISPEC_CUDA_OK(launch_dependent(sample_gemm_kernel, static_cast<unsigned>(n_mt * n_ranges), SM_THREADS,
+                                     SM_SMEM_BYTES, st, 1, tm_hc, tm_w, p));
+    count_launch();
+  }
   TRISPEC_CUDA_OK(launch_dependent(sample_finalize_kernel, static_cast<unsigned>((a->B + 7) / 8), 256, 0, st, 1, p));
   count_launch();
   return TRISPEC_OK;

@@ -222,8 +222,9 @@ def _run_sample(dev, cfg, last_node, bonus_in, seed, step):
     return bonus.cpu().numpy(), val.cpu().numpy()
 
 
-@pytest.mark.parametrize("name,over", [("proxy_tree", dict(B=5, V=20011, d=256)),
-                                       ("llama_tree", dict(B=3, V=128256 // 8, d=512))])
+@pytest.mark.parametrize("name,over", [("proxy_tree", dict(B=5, V=20011, d=256)),        # few sequences: W on the M side
+                                       ("llama_tree", dict(B=19, V=128256 // 8, d=512)),  # 32 sequence columns
+                                       ("proxy_tree", dict(B=40, V=9000, d=128))])        # sequences on the M side
 def test_bonus_sampling_matches_gumbel_max_oracle(name, over):
     """The sampled token is argmax_v (z_v + G_v) with the oracle's counter-based noise. fp32 logits
     can flip the arg-max only where the two best perturbed logits are closer than the LM-head
