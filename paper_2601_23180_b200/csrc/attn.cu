@@ -278,7 +278,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         if (progressed) {
           idle = 0;
         } else {
-          __nanosleep(32);                    // leave the issue slots to the softmax warps
+          // (no sleep here: the sooner an MMA is issued, the sooner its K or V slot is free again)
           if (++idle > kWaitPolls) {          // bounded: give up, flag, and let the kernel end
             if (p.dev_status) atomicExch(p.dev_status, 5);
             break;
