@@ -397,6 +397,30 @@ def run_only(args, cfg):
     print(json.dumps(out), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------
+# Multi-rank host logic (replicas only: sequences are independent, there is no data-path exchange)
+# ---------------------------------------------------------------------------------------------
+def rank_config(cfg, rank: int):
+    """Every rank verifies its own batch of the workload's shape: same config, seed offset by rank."""
+    import dataclasses
+    return dataclasses.replace(cfg, seed=cfg.seed + rank)
+
+
+def max_over_ranks(values, world: int, device="cpu"):
+    """Element-wise maximum of per-rank timings over all ranks (identity for one rank)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_throughput(cfg, world: int, ms_per_step: float) -> float:
+    """Whole-job draft tokens per second: every rank processed one batch per step (weak scaling)."""
+    return cfg_tokens(cfg) * world / (ms_per_step * 1e-3)
+
+
 def cfg_tokens(cfg):
     n = cfg.B if cfg.n_active is None else cfg.n_active
     return n * cfg.k
@@ -453,8 +477,7 @@ def main():
     from paper_2601_23180_b200 import runner
 
     # every rank verifies its own batch of the same shape (seed offset by rank)
-    import dataclasses
-    rcfg = dataclasses.replace(cfg, seed=cfg.seed + rank)
+    rcfg = rank_config(cfg, rank)
     inp = gen.make_inputs(rcfg)
     pas = runner.VerifyPass(rcfg, inp)
     pas.prepare_host(inp)
@@ -549,10 +572,7 @@ def main():
     e2e_s = time.perf_counter() - t0
     clocks = sampler.stop() if rank == 0 else None
 
-    t = torch.tensor([total_ms, e2e_s * 1e3], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_s * 1e3], world, device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -560,7 +580,7 @@ def main():
 
     tokens = cfg_tokens(cfg) * world
     ms_per_step = total_ms / args.steps
-    value = tokens / (ms_per_step * 1e-3)
+    value = aggregate_throughput(cfg, world, ms_per_step)
     peaks = _peaks()
     n_seq = cfg.B if cfg.n_active is None else cfg.n_active
     M = n_seq * cfg.T
