@@ -334,3 +334,32 @@ def test_run_to_run_determinism(H):
     assert np.array_equal(a["o"], b["o"])
     for k in a["stats"]:
         assert np.array_equal(a["stats"][k], b["stats"][k], equal_nan=True)
+
+
+# ------------------------------------------------------------------------------ size limits and degenerate shapes
+EDGE_CASES = [
+    # the largest tree the library takes (T = 64: mask bit 63, both halves of every warp full), a chain of
+    # that length (depth 63), a single node (T = 1: the root alone), 16 query heads per KV head, MHA
+    ("proxy_tree", dict(B=3, k=63, L=200, V=6000, d=128, rho=0.3)),
+    ("tiny_chain", dict(B=2, k=63, max_depth=63, L=130, V=5000, d=128)),
+    ("proxy_tree", dict(B=4, k=0, max_depth=0, L=100, V=4096, d=64)),
+    ("proxy_tree", dict(B=2, k=20, L=300, Hq=16, Hkv=1, V=4000, d=128, rho=0.3)),
+    ("proxy_tree", dict(B=2, k=60, L=70, Hq=4, Hkv=4, V=4000, d=128, rho=0.3)),
+]
+
+
+@pytest.mark.parametrize("name,over", EDGE_CASES)
+def test_fused_pass_at_size_limits(H, name, over):
+    over = dict(over)
+    over.setdefault("logit_scale", 3.6 / (0.02 * math.sqrt(over["d"])))
+    cfg = gen.small_variant(gen.CONFIGS[name], **over)
+    inp = gen.make_inputs(cfg)
+    from paper_2601_23180_b200 import runner
+    import torch
+    pas = runner.VerifyPass(cfg, inp)
+    pas.run()
+    torch.cuda.synchronize()
+    got = pas.results()
+    ref = orc.verify(inp, 1.0 / math.sqrt(cfg.D), cfg.logit_scale, cfg.lam, mode=cfg.mode)
+    _check_pass(H, cfg, inp, got, ref, list(range(cfg.B)))
+    assert got["mask"].view(np.uint64).max() == ref["mask"].max()
