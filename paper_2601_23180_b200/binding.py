@@ -132,6 +132,20 @@ def _p(t: Optional[torch.Tensor]) -> Optional[int]:
     return t.data_ptr()
 
 
+def _hold(a, *objs):
+    """Keeps the tensors whose addresses went into the argument struct alive as long as the struct is:
+    a temporary passed to a builder would otherwise be freed, and its memory handed out again (for
+    instance as the workspace), before the kernels have run."""
+    held = []
+    for o in objs:
+        if isinstance(o, dict):
+            held.extend(v for v in o.values() if v is not None)
+        elif o is not None:
+            held.append(o)
+    a._held = tuple(held)
+    return a
+
+
 def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
     s = torch.cuda.current_stream() if stream is None else stream
     return s.cuda_stream
@@ -165,7 +179,7 @@ def _stats_struct(st: Dict[str, torch.Tensor]) -> Stats:
 # ------------------------------------------------------------------------------ argument builders
 def tree_args(parent: torch.Tensor, mask: torch.Tensor, depth: Optional[torch.Tensor]) -> TreeArgs:
     B, T = parent.shape
-    return TreeArgs(B, T, _p(parent), _p(mask), _p(depth))
+    return _hold(TreeArgs(B, T, _p(parent), _p(mask), _p(depth)), parent, mask, depth)
 
 
 def attn_args(q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, scale, o, workspace=None,
@@ -190,7 +204,8 @@ def attn_args(q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, scale, o, work
     a.workspace = _p(workspace)
     a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     a.dev_status = _p(dev_status)
-    return a
+    return _hold(a, q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, o, workspace, block_table, seq_index, lse,
+                 dev_status)
 
 
 def lmhead_args(h, W, parent, tok, logit_scale, stats, workspace=None, seq_index=None,
@@ -205,7 +220,7 @@ def lmhead_args(h, W, parent, tok, logit_scale, stats, workspace=None, seq_index
     a.workspace = _p(workspace)
     a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     a.dev_status = _p(dev_status)
-    return a
+    return _hold(a, h, W, parent, tok, stats, workspace, seq_index, dev_status)
 
 
 CRIT_MARGIN, CRIT_TOP1, CRIT_ENTROPY = 0, 1, 2
@@ -222,7 +237,7 @@ def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], activ
     a.q_draft, a.u_accept = _p(q_draft), _p(u_accept)
     for k in ("accept_len", "bonus_tok", "path", "last_node", "near_thr", "n_escalated", "esc_index", "escalate"):
         setattr(a, k, _p(out.get(k)))
-    return a
+    return _hold(a, stats, parent, tok, out, active, start_node, q_draft, u_accept)
 
 
 def alloc_scan_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
@@ -244,7 +259,7 @@ def prune_args(parent, tok, mask, root, out: Dict[str, torch.Tensor]) -> PruneAr
     a.n_keep, a.node_map = _p(out["n_keep"]), _p(out["node_map"])
     a.parent_out, a.tok_out = _p(out["parent"]), _p(out["tok"])
     a.mask_out, a.depth_out = _p(out.get("mask")), _p(out.get("depth"))
-    return a
+    return _hold(a, parent, tok, mask, root, out)
 
 
 def alloc_prune_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
@@ -268,7 +283,8 @@ def commit_args(k_tree, v_tree, k_cache, v_cache, ctx_len, path, accept_len, ctx
         a.num_blocks, a.block_size, a.max_blocks_per_seq = k_cache.shape[0], block_size, block_table.shape[1]
     a.block_table, a.ctx_len, a.path, a.accept_len = _p(block_table), _p(ctx_len), _p(path), _p(accept_len)
     a.active, a.ctx_len_out, a.dev_status = _p(active), _p(ctx_len_out), _p(dev_status)
-    return a
+    return _hold(a, k_tree, v_tree, k_cache, v_cache, ctx_len, path, accept_len, ctx_len_out, block_table, active,
+                 dev_status)
 
 
 def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
@@ -302,7 +318,7 @@ def sample_args(h, W, last_node, bonus_tok, logit_scale, seed, step, sample_valu
     a.workspace = _p(workspace)
     a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     a.dev_status = _p(dev_status)
-    return a
+    return _hold(a, h, W, last_node, bonus_tok, sample_value, workspace, dev_status)
 
 
 def trispec_sample_bonus_workspace(args: SampleArgs) -> int:
