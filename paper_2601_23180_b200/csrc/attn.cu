@@ -51,7 +51,8 @@ constexpr float kRescaleThreshold = 8.0f;                // log2 units
 constexpr int AT_PART_PITCH = AT_D * 2 + 16;             // bytes per row of the in-smem partial (bf16, bank spread)
 constexpr int AT_PART_ML_OFF = AT_BM * AT_PART_PITCH;    // (m, l) pairs follow the partial rows
 constexpr int AT_PART_ML2_OFF = AT_PART_ML_OFF + AT_BM * 8;   // gathered (m, l) of every split for this CTA's rows
-static_assert(AT_PART_ML2_OFF + AT_BM * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
+constexpr int AT_PART_ML2_MAX = AT_BM + 2 * 8;                // n_splits x rows per CTA, rows rounded up to even
+static_assert(AT_PART_ML2_OFF + AT_PART_ML2_MAX * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
 
 struct AttnParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits;
@@ -504,7 +505,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   if (kCluster && p.n_splits > 1) {
     // ---------------------------------------------------------------- cluster merge
     // Every CTA of the cluster holds one partial in its shared memory (idle CTAs: weight zero).
-    // CTA `split` normalises rows [split * 128 / n_splits, (split + 1) * 128 / n_splits).
+    // CTA `split` normalises rows [split * rpc, (split + 1) * rpc) of the 128.
     if (idle_cta) {
       for (int r = threadIdx.x; r < AT_BM; r += AT_THREADS) sPartML[r] = make_float2(-INFINITY, 0.f);
     }
@@ -513,12 +514,13 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     // Requests over the SM-to-SM network are expensive per instruction, whatever their size,
     // so they are few and wide: one gather of the (m, l) pairs of all splits for this CTA's
     // rows, then per pair of rows one 16-byte-per-lane load from every split.
-    const int rpc = AT_BM / p.n_splits;          // rows this CTA normalises: 16 .. 128, even
+    // rows this CTA normalises: an even share of the 128 (the last CTA may get fewer)
+    const int rpc = (((AT_BM + p.n_splits - 1) / p.n_splits) + 1) & ~1;
     const uint32_t po_u = smem_u32(sPartO), pml_u = smem_u32(sPartML);
     float2* sML2 = reinterpret_cast<float2*>(smem + AT_PART_ML2_OFF);   // [n_splits][rpc]
-    if (threadIdx.x < AT_BM) {
-      const int s_src = threadIdx.x / rpc, r = threadIdx.x % rpc;
-      sML2[threadIdx.x] = ld_cluster_f2(cluster_map(pml_u + (split * rpc + r) * 8, s_src));
+    for (int t = threadIdx.x; t < p.n_splits * rpc; t += AT_THREADS) {
+      const int s_src = t / rpc, row = split * rpc + t % rpc;
+      if (row < AT_BM) sML2[t] = ld_cluster_f2(cluster_map(pml_u + row * 8, s_src));
     }
     __syncthreads();
     constexpr int kWarps = AT_THREADS / 32;
@@ -527,7 +529,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       const int rl = 2 * pr + half;               // row within this CTA's slice
       const int row = split * rpc + rl;
       const int node = mtile * p.NPT + row / p.G;
-      const bool ok = (row < p.NPT * p.G) && (node < p.T);
+      const bool ok = (row < AT_BM) && (row < p.NPT * p.G) && (node < p.T);
       uint4 v[8];
       float2 ml[8];
 #pragma unroll
@@ -660,19 +662,21 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   pl->n_mt = (a->T + pl->NPT - 1) / pl->NPT;
   pl->tiles_max = (Lmax + AT_BN - 1) / AT_BN;
   const long long fixed = static_cast<long long>(pl->n_seq) * a->Hkv * pl->n_mt;
-  // Number of KV splits: a power of two that minimises waves x (fixed cost + tiles per CTA).
-  // The fixed cost of a CTA (pipeline fill, Q load, merge) is worth about 8 context tiles; more
-  // than 8 splits cannot form a cluster and pay for a second kernel (about 6 tiles).
+  // Number of KV splits (1..8 form a cluster; 16, 32, ... go through the workspace). Measured on the
+  // five workloads: more than about 1.25 waves of CTAs with at least 32 tiles each run best (the fixed
+  // costs of a CTA - pipeline fill, Q load, merge - hide behind other CTAs); when tiles are too few
+  // for that, one wave filled as far as possible; very few (sequence, head) pairs are cut further.
   const long long slots = static_cast<long long>(device_sm_count()) * 2;   // two CTAs per SM
-  long long best_cost = -1;
-  int best_s = 1;
-  for (int sp = 1; sp <= 1024; sp <<= 1) {
-    if (sp > 1 && pl->tiles_max / sp < 4) break;
-    const long long ctas = fixed * sp;
-    const long long waves = (ctas + slots - 1) / slots;
-    const long long per_cta = 8 + (pl->tiles_max + sp - 1) / sp;
-    const long long cost = waves * per_cta + (sp > 8 ? 6 : 0);
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_s = sp; }
+  const int tiles = pl->tiles_max;
+  int best_s = 0;
+  for (int sp = 1; sp <= 8 && !best_s; ++sp)
+    if (fixed * sp * 4 >= slots * 5 && tiles / sp >= 32) best_s = sp;
+  if (!best_s) {
+    best_s = 1;
+    for (int sp = 2; sp <= 8; ++sp)
+      if (fixed * sp <= slots && tiles / sp >= 4) best_s = sp;
+    if (best_s == 8 && fixed * 8 * 2 <= slots)
+      for (int sp = 16; sp <= 1024 && fixed * sp <= slots && tiles / sp >= 8; sp *= 2) best_s = sp;
   }
   pl->n_splits = best_s;
   pl->cluster = pl->n_splits <= 8;

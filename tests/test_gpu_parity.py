@@ -195,6 +195,12 @@ ATTN_CASES = [
     ("proxy_tree", dict(B=2, L=64, Hq=8, Hkv=8), [64, 0]),                     # G = 1 (MHA)
     ("proxy_tree", dict(B=1, L=9300, Hq=4, Hkv=2), None),                      # > 8 KV splits: workspace merge
     ("long_paged", dict(B=3, L=5000, L_min=5000, Hq=4, Hkv=2), [5000, 40, 2300]),  # 8-CTA clusters with idle splits
+    # cluster sizes that do not divide 128: uneven row shares in the merge
+    ("tiny_chain", dict(B=1, L=900, Hq=4, Hkv=2), None),                       # 3 splits
+    ("tiny_chain", dict(B=1, L=1300, Hq=4, Hkv=2), None),                      # 5 splits
+    ("tiny_chain", dict(B=6, L=1800, Hq=16, Hkv=8), None),                     # 6 splits
+    ("proxy_tree", dict(B=1, L=1800, Hq=4, Hkv=2), None),                      # 7 splits, T = 61
+    ("tiny_chain", dict(B=5, L=2500, Hq=16, Hkv=8), [2500, 1000, 64, 2499, 7]),  # 7 splits, ragged
 ]
 
 
