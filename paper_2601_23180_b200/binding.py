@@ -163,8 +163,11 @@ STAT_F32 = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_log
 STAT_I32 = ("top1_idx", "top2_idx")
 
 
-def alloc_stats(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
-    st = {k: torch.full((B, T), float("nan"), dtype=torch.float32, device=device) for k in STAT_F32}
+def alloc_stats(B: int, T: int, device="cuda", entropy: bool = True) -> Dict[str, torch.Tensor]:
+    """Output buffers of the LM-head statistics. The entropy is optional in the C ABI (a null pointer
+    skips its computation, which saves two instructions per logit in the GEMM's epilogue)."""
+    st = {k: torch.full((B, T), float("nan"), dtype=torch.float32, device=device)
+          for k in STAT_F32 if entropy or k != "entropy"}
     st.update({k: torch.full((B, T), -1, dtype=torch.int32, device=device) for k in STAT_I32})
     return st
 

@@ -64,8 +64,10 @@ struct LmParams {
   int32_t* dev_status;
 };
 
-// Vocabulary range r of n_ranges, cut into tiles of at most 256 columns; all boundaries are
-// multiples of 32 columns so that each CTA of a pair takes a half that is a multiple of 16.
+// Vocabulary range r of n_ranges, cut into tiles of 256 columns plus one narrower tile for the
+// rest; all boundaries are multiples of 32 columns so that each CTA of a pair takes a half that
+// is a multiple of 16. (A tile of 224 columns costs as much as one of 256 - its k-loop is as long
+// and the MMA time does not shrink in proportion - so the rest is not spread over the tiles.)
 struct TileIter {
   int u0, units, n_tiles;
   __device__ TileIter(int V, int n_ranges, int r) {
@@ -76,12 +78,12 @@ struct TileIter {
     n_tiles = (units + 7) >> 3;
   }
   __device__ void tile(int t, int& n0, int& nw) const {
-    const int a = (units * t) / n_tiles, b = (units * (t + 1)) / n_tiles;
-    n0 = (u0 + a) << 5;
-    nw = (b - a) << 5;
+    n0 = (u0 + 8 * t) << 5;
+    nw = min(8, units - 8 * t) << 5;
   }
 };
 
+template <bool kEntropy>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                    const LmParams p) {
@@ -208,29 +210,63 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
         tc_wait_ld();
         const int nv = ncols - c0;  // >= 1
         float cmax = -INFINITY;
+        if (nv >= 32) {
+          // whole chunk valid: three-input max and packed fp32 pairs halve the instruction count
+          float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float v = __uint_as_float(r[j]);
-          if (j >= nv) { v = -INFINITY; r[j] = __float_as_uint(v); }
-          cmax = fmaxf(cmax, v);
-        }
-        if (cmax > m) {
-          const float f = ex2f((m - cmax) * c);
-          s *= f;
-          tz *= f;
-          m = cmax;
-        }
-        const float mc = m * c;
-        float acc = 0.f, acz = 0.f;
+          for (int j = 0; j < 32; j += 8) {
+            cm[0] = fmax3(cm[0], __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+            cm[1] = fmax3(cm[1], __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            cm[2] = fmax3(cm[2], __uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+            cm[3] = fmax3(cm[3], __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+          }
+          cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
+          if (cmax > m) {
+            const float f = ex2f((m - cmax) * c);
+            s *= f;
+            tz *= f;
+            m = cmax;
+          }
+          const float nmc = -m * c;
+          const float2 c2 = make_float2(c, c), nmc2 = make_float2(nmc, nmc);
+          float2 acc2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          float2 acz2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float e = ex2f(fmaf(__uint_as_float(r[j]), c, -mc));
-          acc += e;
-          // masked columns hold -inf with e = 0: keep 0 * inf out of the sum
-          acz = fmaf(e, (j < nv) ? __uint_as_float(r[j]) : 0.f, acz);
+          for (int j = 0; j < 32; j += 2) {
+            const float2 z = make_float2(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+            const float2 x = ffma2(z, c2, nmc2);
+            const float2 e = make_float2(ex2f(x.x), ex2f(x.y));
+            acc2[(j >> 1) & 1] = fadd2(acc2[(j >> 1) & 1], e);
+            if (kEntropy) acz2[(j >> 1) & 1] = ffma2(e, z, acz2[(j >> 1) & 1]);
+          }
+          s += (acc2[0].x + acc2[0].y) + (acc2[1].x + acc2[1].y);
+          if (kEntropy) tz += (acz2[0].x + acz2[0].y) + (acz2[1].x + acz2[1].y);
+        } else {
+          // ragged end of the vocabulary: columns past V count as -inf
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float v = __uint_as_float(r[j]);
+            if (j >= nv) { v = -INFINITY; r[j] = __float_as_uint(v); }
+            cmax = fmaxf(cmax, v);
+          }
+          if (cmax > m) {
+            const float f = ex2f((m - cmax) * c);
+            s *= f;
+            tz *= f;
+            m = cmax;
+          }
+          const float mc = m * c;
+          float acc = 0.f, acz = 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float e = ex2f(fmaf(__uint_as_float(r[j]), c, -mc));
+            acc += e;
+            // masked columns hold -inf with e = 0: keep 0 * inf out of the sum
+            if (kEntropy) acz = fmaf(e, (j < nv) ? __uint_as_float(r[j]) : 0.f, acz);
+          }
+          s += acc;
+          tz += acz;
         }
-        s += acc;
-        tz += acz;
         if (cmax > v2) {
           const int col0 = n0 + c0;
 #pragma unroll
@@ -290,61 +326,106 @@ __device__ __forceinline__ void lm_top2_insert(float v, int i, float& v1, int& i
   else if (lm_better(v, i, v2, i2)) { v2 = v; i2 = i; }
 }
 
-// log-sum-exp of one row from its per-range partials, computed by a whole warp
-__device__ __forceinline__ void lm_row_lse(const LmPartial* part, size_t stride, size_t prow, int n_ranges, float c,
-                                           int lane, float& M, float& S, float& TZ) {
-  float m = -INFINITY;
-  for (int r = lane; r < n_ranges; r += 32) m = fmaxf(m, part[r * stride + prow].m);
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  float sacc = 0.f, tacc = 0.f;
-  for (int r = lane; r < n_ranges; r += 32) {
-    const LmPartial q = part[r * stride + prow];
-    const float f = ex2f((q.m - m) * c);
-    sacc += q.s * f;
-    tacc += q.t * f;
-  }
-  for (int o = 16; o > 0; o >>= 1) {
-    sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
-    tacc += __shfl_xor_sync(0xffffffffu, tacc, o);
-  }
-  M = m; S = sacc; TZ = tacc;
+// running (max, sum of exponentials, sum of exponentials x logit) of a set of vocabulary ranges
+struct LmRowAcc { float m, s, t; };
+__device__ __forceinline__ void lm_fold(LmRowAcc& a, float m, float s, float t, float c) {
+  const float M = fmaxf(a.m, m);
+  const float fa = (a.m == -INFINITY) ? 0.f : ex2f((a.m - M) * c);
+  const float fb = (m == -INFINITY) ? 0.f : ex2f((m - M) * c);
+  a.s = a.s * fa + s * fb;
+  a.t = a.t * fa + t * fb;
+  a.m = M;
 }
 
 // One warp per (active sequence, node): merges the row's partial statistics and, for a child
 // node, computes the logit of its drafted token in its parent's row (a d-long dot product).
+// The dot product needs only the kernel's inputs, so it runs before the wait for the GEMM and
+// overlaps that kernel's tail; after the wait every lane loads its share of the partials of
+// the node's row and of the parent's row in one go and the warp folds them by shuffles.
 __global__ void __launch_bounds__(LM_FIN_THREADS)
 lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
   pdl_launch_dependents();
-  pdl_wait();
   const int lane = threadIdx.x & 31;
   const long long w = static_cast<long long>(blockIdx.x) * (LM_FIN_THREADS / 32) + (threadIdx.x >> 5);
   const int T = p.T;
-  if (w >= static_cast<long long>(n_seq) * T) return;
-  const int a = static_cast<int>(w / T), node = static_cast<int>(w % T);
+  const bool active = w < static_cast<long long>(n_seq) * T;
+  const int a = active ? static_cast<int>(w / T) : 0, node = active ? static_cast<int>(w % T) : 0;
   const int seq = p.seq_index ? __ldg(p.seq_index + a) : a;
   const long long row0 = static_cast<long long>(seq) * T;
-  const size_t stride = static_cast<size_t>(p.n_mt) * 2 * LM_BM;
-  const size_t prow = static_cast<size_t>(a) * 64 + node;
 
-  float M, S, TZ;
-  lm_row_lse(p.partial, stride, prow, p.n_ranges, p.c, lane, M, S, TZ);
+  // ---- drafted-token logit z[parent(node)][tok[node]]: inputs only
+  bool has_draft = false;
+  int par = 0;
+  float dot = 0.f;
+  if (active && node >= 1) {
+    par = __ldg(p.parent + row0 + node);
+    const int tk = __ldg(p.tok + row0 + node);
+    has_draft = par >= 0 && par < node && tk >= 0 && tk < p.V;
+    if (has_draft) {
+      const uint4* hv = reinterpret_cast<const uint4*>(p.h + (row0 + par) * p.d);
+      const uint4* wv = reinterpret_cast<const uint4*>(p.W + static_cast<long long>(tk) * p.d);
+      float acc[2] = {0.f, 0.f};
+#pragma unroll 4
+      for (int i = lane; i < p.d / 8; i += 32) {
+        const uint4 x = __ldg(hv + i), y = __ldg(wv + i);
+        acc[0] = fmaf(bf16_lo(x.x), bf16_lo(y.x), acc[0]); acc[1] = fmaf(bf16_hi(x.x), bf16_hi(y.x), acc[1]);
+        acc[0] = fmaf(bf16_lo(x.y), bf16_lo(y.y), acc[0]); acc[1] = fmaf(bf16_hi(x.y), bf16_hi(y.y), acc[1]);
+        acc[0] = fmaf(bf16_lo(x.z), bf16_lo(y.z), acc[0]); acc[1] = fmaf(bf16_hi(x.z), bf16_hi(y.z), acc[1]);
+        acc[0] = fmaf(bf16_lo(x.w), bf16_lo(y.w), acc[0]); acc[1] = fmaf(bf16_hi(x.w), bf16_hi(y.w), acc[1]);
+      }
+      dot = acc[0] + acc[1];
+      for (int o2 = 16; o2 > 0; o2 >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o2);
+    }
+  }
+  if (!has_draft) par = node;                    // a valid row to load; the result is not used
+
+  pdl_wait();                                    // the partials come from the GEMM kernel
+  if (!active) return;
+
+  // ---- merge of the per-range partials: own row (all statistics) and parent row (max, sum)
+  const size_t stride = static_cast<size_t>(p.n_mt) * 2 * LM_BM;
+  const LmPartial* own = p.partial + static_cast<size_t>(a) * 64 + node;
+  const LmPartial* parp = p.partial + static_cast<size_t>(a) * 64 + par;
+  LmRowAcc ro = {-INFINITY, 0.f, 0.f}, rp = {-INFINITY, 0.f, 0.f};
   float v1 = -INFINITY, v2 = -INFINITY;
   int i1 = -1, i2 = -1;
-  for (int r = lane; r < p.n_ranges; r += 32) {
-    const LmPartial q = p.partial[r * stride + prow];
-    lm_top2_insert(q.v1, q.i1, v1, i1, v2, i2);
-    lm_top2_insert(q.v2, q.i2, v1, i1, v2, i2);
+  for (int r0 = 0; r0 < p.n_ranges; r0 += 96) {  // three ranges per lane and round, loads first
+    float4 qa[3], qb[3];
+    float2 qp[3];
+#pragma unroll
+    for (int u = 0; u < 3; ++u) {
+      const int r = r0 + lane + 32 * u;
+      qa[u] = make_float4(-INFINITY, 0.f, -INFINITY, -INFINITY);
+      qb[u] = make_float4(__int_as_float(-1), __int_as_float(-1), 0.f, 0.f);
+      qp[u] = make_float2(-INFINITY, 0.f);
+      if (r < p.n_ranges) {
+        const float4* q4 = reinterpret_cast<const float4*>(own + r * stride);
+        qa[u] = q4[0];                           // m, s, v1, v2
+        qb[u] = q4[1];                           // i1, i2, t, pad
+        qp[u] = *reinterpret_cast<const float2*>(parp + r * stride);   // m, s of the parent's row
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 3; ++u) {
+      lm_fold(ro, qa[u].x, qa[u].y, qb[u].z, p.c);
+      lm_fold(rp, qp[u].x, qp[u].y, 0.f, p.c);
+      lm_top2_insert(qa[u].z, __float_as_int(qb[u].x), v1, i1, v2, i2);
+      lm_top2_insert(qa[u].w, __float_as_int(qb[u].y), v1, i1, v2, i2);
+    }
   }
   for (int o = 16; o > 0; o >>= 1) {
+    lm_fold(ro, __shfl_xor_sync(0xffffffffu, ro.m, o), __shfl_xor_sync(0xffffffffu, ro.s, o),
+            __shfl_xor_sync(0xffffffffu, ro.t, o), p.c);
+    lm_fold(rp, __shfl_xor_sync(0xffffffffu, rp.m, o), __shfl_xor_sync(0xffffffffu, rp.s, o), 0.f, p.c);
     const float ov1 = __shfl_xor_sync(0xffffffffu, v1, o), ov2 = __shfl_xor_sync(0xffffffffu, v2, o);
     const int oi1 = __shfl_xor_sync(0xffffffffu, i1, o), oi2 = __shfl_xor_sync(0xffffffffu, i2, o);
     lm_top2_insert(ov1, oi1, v1, i1, v2, i2);
     lm_top2_insert(ov2, oi2, v1, i1, v2, i2);
   }
-  const float lse = M * p.scale + logf(S);
-  const long long o = row0 + node;
   if (lane == 0) {
-    p.out.max[o] = M * p.scale;
+    const float lse = ro.m * p.scale + logf(ro.s);
+    const long long o = row0 + node;
+    p.out.max[o] = ro.m * p.scale;
     p.out.lse[o] = lse;
     p.out.top1_val[o] = v1 * p.scale;
     p.out.top2_val[o] = v2 * p.scale;
@@ -353,32 +434,12 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
     p.out.p_top1[o] = expf(v1 * p.scale - lse);
     p.out.p_top2[o] = expf(v2 * p.scale - lse);
     // entropy in nats: H = lse - E_p[z], E_p[z] = scale * sum(e * z_raw) / sum(e); never below 0
-    if (p.out.entropy) p.out.entropy[o] = fmaxf(lse - p.scale * (TZ / S), 0.f);
-  }
-  // drafted-token logit z[parent(node)][tok[node]]
-  float dl = __int_as_float(0x7fc00000), pd = dl;
-  if (node >= 1) {
-    const int par = __ldg(p.parent + row0 + node);
-    const int tk = __ldg(p.tok + row0 + node);
-    if (par >= 0 && par < node && tk >= 0 && tk < p.V) {
-      float Mp, Sp, Tp;
-      lm_row_lse(p.partial, stride, static_cast<size_t>(a) * 64 + par, p.n_ranges, p.c, lane, Mp, Sp, Tp);
-      const uint4* hv = reinterpret_cast<const uint4*>(p.h + (row0 + par) * p.d);
-      const uint4* wv = reinterpret_cast<const uint4*>(p.W + static_cast<long long>(tk) * p.d);
-      float acc = 0.f;
-      for (int i = lane; i < p.d / 8; i += 32) {
-        const uint4 x = __ldg(hv + i), y = __ldg(wv + i);
-        acc = fmaf(bf16_lo(x.x), bf16_lo(y.x), acc); acc = fmaf(bf16_hi(x.x), bf16_hi(y.x), acc);
-        acc = fmaf(bf16_lo(x.y), bf16_lo(y.y), acc); acc = fmaf(bf16_hi(x.y), bf16_hi(y.y), acc);
-        acc = fmaf(bf16_lo(x.z), bf16_lo(y.z), acc); acc = fmaf(bf16_hi(x.z), bf16_hi(y.z), acc);
-        acc = fmaf(bf16_lo(x.w), bf16_lo(y.w), acc); acc = fmaf(bf16_hi(x.w), bf16_hi(y.w), acc);
-      }
-      for (int o2 = 16; o2 > 0; o2 >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o2);
-      dl = acc * p.scale;
-      pd = expf(dl - (Mp * p.scale + logf(Sp)));
+    if (p.out.entropy) p.out.entropy[o] = fmaxf(lse - p.scale * (ro.t / ro.s), 0.f);
+    float dl = __int_as_float(0x7fc00000), pd = dl;
+    if (has_draft) {
+      dl = dot * p.scale;
+      pd = expf(dl - (rp.m * p.scale + logf(rp.s)));
     }
-  }
-  if (lane == 0) {
     p.out.draft_logit[o] = dl;
     p.out.p_draft[o] = pd;
   }
@@ -437,8 +498,12 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
     const uint32_t box[2] = {LM_BK, 64};
     if (!cached_tmap_bf16(&tm_w, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
   }
-  static bool smem_set[64] = {};
-  rc = ensure_smem_limit(reinterpret_cast<const void*>(lmhead_gemm_kernel), LM_SMEM_BYTES, smem_set);
+  // the entropy sum costs two more instructions per logit: only computed when it is asked for
+  const bool want_entropy = a->out.entropy != nullptr;
+  static bool smem_set[2][64] = {};
+  rc = want_entropy
+           ? ensure_smem_limit(reinterpret_cast<const void*>(lmhead_gemm_kernel<true>), LM_SMEM_BYTES, smem_set[1])
+           : ensure_smem_limit(reinterpret_cast<const void*>(lmhead_gemm_kernel<false>), LM_SMEM_BYTES, smem_set[0]);
   if (rc != TRISPEC_OK) return rc;
   LmParams p;
   p.T = a->T; p.d = a->d; p.V = a->V;
@@ -447,8 +512,13 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   p.seq_index = a->seq_index;
   p.partial = static_cast<LmPartial*>(a->workspace);
   p.dev_status = a->dev_status;
-  TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel, static_cast<unsigned>(2 * n_mt * n_ranges), LM_THREADS,
-                                   LM_SMEM_BYTES, st, 2, tm_h, tm_w, p));
+  if (want_entropy) {
+    TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel<true>, static_cast<unsigned>(2 * n_mt * n_ranges), LM_THREADS,
+                                     LM_SMEM_BYTES, st, 2, tm_h, tm_w, p));
+  } else {
+    TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel<false>, static_cast<unsigned>(2 * n_mt * n_ranges), LM_THREADS,
+                                     LM_SMEM_BYTES, st, 2, tm_h, tm_w, p));
+  }
   count_launch();
 
   LmFinalizeParams f;

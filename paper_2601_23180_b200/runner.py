@@ -26,7 +26,8 @@ def _i32_dev(x: np.ndarray) -> torch.Tensor:
 
 
 class VerifyPass:
-    def __init__(self, cfg: gen.VerifyConfig, inp: Dict[str, np.ndarray], with_attention: bool = True):
+    def __init__(self, cfg: gen.VerifyConfig, inp: Dict[str, np.ndarray], with_attention: bool = True,
+                 criterion: int = ts.CRIT_MARGIN):
         self.cfg = cfg
         B, T = cfg.B, cfg.T
         d: Dict[str, Optional[torch.Tensor]] = {}
@@ -43,7 +44,8 @@ class VerifyPass:
         self.mask = torch.zeros((B, T), dtype=torch.int64, device="cuda")
         self.depth = torch.zeros((B, T), dtype=torch.int32, device="cuda")
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
-        self.stats = ts.alloc_stats(B, T)
+        # the entropy is computed only for the routing criterion that reads it (the margin rule of Eq. 8 does not)
+        self.stats = ts.alloc_stats(B, T, entropy=(criterion == ts.CRIT_ENTROPY))
         self.scan_out = ts.alloc_scan_out(B, T)
         self.tree_args = ts.tree_args(d["parent"], self.mask, self.depth)
         self.attn_args = None
@@ -64,7 +66,7 @@ class VerifyPass:
         l.workspace, l.workspace_bytes = self.lm_ws.data_ptr(), self.lm_ws.numel()
         self.lm_args = l
         self.scan_args = ts.scan_args(self.stats, d["parent"], d["tok"], cfg.lam, cfg.mode, self.scan_out,
-                                      active=self.active)
+                                      active=self.active, criterion=criterion)
         self._host = None
 
     # one verify pass, inputs resident on the device

@@ -287,3 +287,35 @@ def test_bonus_sampling_follows_the_softmax_on_a_small_vocabulary():
     assert counts.sum() == n
     # counts are integers: allow two draws on top of 4.5 standard deviations (rare tokens)
     assert np.all(np.abs(counts - n * p) <= 4.5 * np.sqrt(n * p * (1 - p)) + 2.0)
+
+
+def test_fused_pass_with_entropy_routing():
+    """The fused pass asks the LM head for the entropy only when the routing criterion reads it. Here
+    it does: the entropies must match the oracle's, and the scan must be the oracle's entropy-routed
+    walk on the statistics the GPU produced (sequences with a feature on the threshold excepted)."""
+    import torch
+    import tests.gpu_helpers as H
+    from paper_2601_23180_b200 import binding as ts
+    from paper_2601_23180_b200 import runner
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=6, L=130, V=12000, d=256, lam=1.2,
+                            logit_scale=3.6 / (0.02 * 16.0), seed=11)
+    inp = gen.make_inputs(cfg)
+    margin_pass = runner.VerifyPass(cfg, inp)
+    assert "entropy" not in margin_pass.stats            # the margin rule does not pay for it
+    pas = runner.VerifyPass(cfg, inp, criterion=ts.CRIT_ENTROPY)
+    pas.run()
+    torch.cuda.synchronize()
+    got = pas.results()
+    assert got["status"] == 0
+    ref_st = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale)
+    H.check_stats(got["stats"], ref_st, pas.seqs, cfg.T)
+    st = got["stats"]
+    ref = orc.accept_scan(st["p_top1"].astype(np.float64), st["p_top2"].astype(np.float64),
+                          st["top1_idx"].astype(np.int64), inp["parent"], inp["tok"], cfg.lam, mode=cfg.mode,
+                          criterion=orc.CRIT_ENTROPY, entropy=st["entropy"].astype(np.float64))
+    clean = (ref["near_thr"] == 0) & (got["scan"]["near_thr"] == 0)
+    assert clean.sum() >= cfg.B - 2
+    for k in ("accept_len", "escalate", "bonus_tok", "last_node", "path"):
+        assert np.array_equal(got["scan"][k][clean], ref[k][clean]), k
+    # the entropy criterion must route both ways on this input, or the test says nothing
+    assert 0 < ref["escalate"].sum() < cfg.B
