@@ -328,6 +328,10 @@ int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
  * events (host resources, kept until the process exits); no device memory is allocated.
  * Host pointers should be page-locked for the copies to be asynchronous; the results are
  * valid once `stream` has been synchronised. NULL host input pointers skip that copy.
+ * Copies whose host AND device addresses follow each other are merged into one transfer, in
+ * these orders: (parent, tok, h), (q, k_tree, v_tree), (accept_len, bonus_tok, last_node,
+ * path, escalate). A caller that carves each group out of one host and one device buffer in
+ * that order pays three transfers per round instead of eleven.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
   const int32_t *parent, *tok;              /* host [B][T] */

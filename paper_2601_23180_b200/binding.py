@@ -10,6 +10,7 @@ import ctypes as C
 import os
 from typing import Dict, Optional
 
+import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
@@ -243,15 +244,49 @@ def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], activ
     return _hold(a, stats, parent, tok, out, active, start_node, q_draft, u_accept)
 
 
+def _nbytes(shape, dtype) -> int:
+    return int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+
+
+def _carve(buf: torch.Tensor, specs, align: int = 16):
+    """Views into one flat uint8 buffer in the given order: (name, shape, dtype). Every array starts
+    on a multiple of `align` bytes (the kernels want 16); where the sizes are multiples of it the arrays
+    follow each other without gaps, which is what lets the host-buffer entry point merge their copies."""
+    out, off = {}, 0
+    for name, shape, dtype in specs:
+        off = (off + align - 1) // align * align
+        n = _nbytes(shape, dtype)
+        out[name] = buf[off:off + n].view(dtype).view(*shape)
+        off += n
+    return out
+
+
+def _carve_bytes(specs, align: int = 16) -> int:
+    off = 0
+    for _, shape, dtype in specs:
+        off = (off + align - 1) // align * align + _nbytes(shape, dtype)
+    return off
+
+
+def scan_out_specs(B: int, T: int):
+    """The scan's outputs in the order `trispec_verify_host` copies them back (accept_len, bonus_tok,
+    last_node, path, escalate), then the ones that stay on the device."""
+    i32 = torch.int32
+    return [("accept_len", (B,), i32), ("bonus_tok", (B,), i32), ("last_node", (B,), i32), ("path", (B, T), i32),
+            ("escalate", (B,), torch.uint8)]
+
+
 def alloc_scan_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
+    """Output buffers of the scan. The five arrays a decode loop reads back are carved out of one
+    allocation, back to back, so that their device-to-host copies can be merged into one."""
+    specs = scan_out_specs(B, T)
+    out = _carve(torch.empty(_carve_bytes(specs), dtype=torch.uint8, device=device), specs)
+    for k, v in out.items():
+        v.fill_(9 if k == "escalate" else -7)
     i32 = dict(dtype=torch.int32, device=device)
-    return {
-        "accept_len": torch.full((B,), -7, **i32), "bonus_tok": torch.full((B,), -7, **i32),
-        "path": torch.full((B, T), -7, **i32), "last_node": torch.full((B,), -7, **i32),
-        "near_thr": torch.full((B,), -7, **i32), "n_escalated": torch.full((1,), -7, **i32),
-        "esc_index": torch.full((B,), -7, **i32),
-        "escalate": torch.full((B,), 9, dtype=torch.uint8, device=device),
-    }
+    out.update({"near_thr": torch.full((B,), -7, **i32), "n_escalated": torch.full((1,), -7, **i32),
+                "esc_index": torch.full((B,), -7, **i32)})
+    return out
 
 
 def prune_args(parent, tok, mask, root, out: Dict[str, torch.Tensor]) -> PruneArgs:

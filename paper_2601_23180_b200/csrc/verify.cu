@@ -56,9 +56,28 @@ extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree
   if (!io || !tree || !lm || !scan) return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t BT = static_cast<size_t>(tree->B) * tree->T;
-  auto h2d = [&](const void* dst, const void* src, size_t bytes, cudaStream_t s) -> cudaError_t {
-    if (!src || !dst) return cudaSuccess;
-    return cudaMemcpyAsync(const_cast<void*>(dst), src, bytes, cudaMemcpyHostToDevice, s);
+  // A copy list is issued with neighbours merged: requests whose source AND destination follow
+  // each other in memory become one transfer (each transfer costs a few microseconds of set-up
+  // whatever its size, and a pass moves eleven arrays). Callers get this by carving the arrays
+  // out of one host and one device buffer in the order used here.
+  struct CopyReq { void* dst; const void* src; size_t bytes; };
+  auto copy_list = [](CopyReq* r, int n, cudaMemcpyKind kind, cudaStream_t s) -> cudaError_t {
+    int i = 0;
+    while (i < n) {
+      if (!r[i].dst || !r[i].src || r[i].bytes == 0) { ++i; continue; }
+      size_t bytes = r[i].bytes;
+      int j = i + 1;
+      while (j < n && r[j].dst && r[j].src &&
+             static_cast<const char*>(r[j].dst) == static_cast<const char*>(r[i].dst) + bytes &&
+             static_cast<const char*>(r[j].src) == static_cast<const char*>(r[i].src) + bytes) {
+        bytes += r[j].bytes;
+        ++j;
+      }
+      cudaError_t e = cudaMemcpyAsync(r[i].dst, r[i].src, bytes, kind, s);
+      if (e != cudaSuccess) return e;
+      i = j;
+    }
+    return cudaSuccess;
   };
   HostPassStreams* hs = nullptr;
   if (attn) {
@@ -69,14 +88,18 @@ extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree
     TRISPEC_CUDA_OK(cudaEventRecord(hs->fork, st));
   }
   // what the LM head needs goes first through the copy engine
-  TRISPEC_CUDA_OK(h2d(tree->parent, io->parent, BT * 4, st));
-  TRISPEC_CUDA_OK(h2d(lm->tok, io->tok, BT * 4, st));
-  TRISPEC_CUDA_OK(h2d(lm->h, io->h, BT * static_cast<size_t>(lm->d) * 2, st));
+  {
+    CopyReq in[3] = {{const_cast<int32_t*>(tree->parent), io->parent, BT * 4},
+                     {const_cast<int32_t*>(lm->tok), io->tok, BT * 4},
+                     {const_cast<void*>(lm->h), io->h, BT * static_cast<size_t>(lm->d) * 2}};
+    TRISPEC_CUDA_OK(copy_list(in, 3, cudaMemcpyHostToDevice, st));
+  }
   if (attn) {
     TRISPEC_CUDA_OK(cudaStreamWaitEvent(hs->copy, hs->fork, 0));
-    TRISPEC_CUDA_OK(h2d(attn->q, io->q, BT * static_cast<size_t>(attn->Hq) * attn->D * 2, hs->copy));
-    TRISPEC_CUDA_OK(h2d(attn->k_tree, io->k_tree, BT * static_cast<size_t>(attn->Hkv) * attn->D * 2, hs->copy));
-    TRISPEC_CUDA_OK(h2d(attn->v_tree, io->v_tree, BT * static_cast<size_t>(attn->Hkv) * attn->D * 2, hs->copy));
+    CopyReq in[3] = {{const_cast<void*>(attn->q), io->q, BT * static_cast<size_t>(attn->Hq) * attn->D * 2},
+                     {const_cast<void*>(attn->k_tree), io->k_tree, BT * static_cast<size_t>(attn->Hkv) * attn->D * 2},
+                     {const_cast<void*>(attn->v_tree), io->v_tree, BT * static_cast<size_t>(attn->Hkv) * attn->D * 2}};
+    TRISPEC_CUDA_OK(copy_list(in, 3, cudaMemcpyHostToDevice, hs->copy));
     TRISPEC_CUDA_OK(cudaEventRecord(hs->copied, hs->copy));
   }
   int rc = trispec_build_tree_mask(tree, stream);
@@ -90,15 +113,12 @@ extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree
   }
   rc = trispec_accept_scan(scan, stream);
   if (rc != TRISPEC_OK) return rc;
-  auto d2h = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
-    if (!src || !dst) return cudaSuccess;
-    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st);
-  };
   const size_t B = static_cast<size_t>(scan->B);
-  TRISPEC_CUDA_OK(d2h(io->accept_len, scan->accept_len, B * 4));
-  TRISPEC_CUDA_OK(d2h(io->bonus_tok, scan->bonus_tok, B * 4));
-  TRISPEC_CUDA_OK(d2h(io->last_node, scan->last_node, B * 4));
-  TRISPEC_CUDA_OK(d2h(io->path, scan->path, B * static_cast<size_t>(scan->T) * 4));
-  TRISPEC_CUDA_OK(d2h(io->escalate, scan->escalate, B));
+  CopyReq out[5] = {{io->accept_len, scan->accept_len, B * 4},
+                    {io->bonus_tok, scan->bonus_tok, B * 4},
+                    {io->last_node, scan->last_node, B * 4},
+                    {io->path, scan->path, B * static_cast<size_t>(scan->T) * 4},
+                    {io->escalate, scan->escalate, B}};
+  TRISPEC_CUDA_OK(copy_list(out, 5, cudaMemcpyDeviceToHost, st));
   return TRISPEC_OK;
 }

@@ -25,16 +25,39 @@ def _i32_dev(x: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).cuda()
 
 
+def _pack_round_inputs(inp: Dict[str, np.ndarray], names):
+    """One flat byte tensor (CPU) holding the named arrays back to back, and the (name, shape, dtype)
+    list that carves it: int32 for the tree arrays, bf16 for the activations (stored as bit patterns)."""
+    arrays, specs = {}, []
+    for k in names:
+        if k in ("parent", "tok"):
+            arrays[k] = np.ascontiguousarray(inp[k], dtype=np.int32)
+            specs.append((k, arrays[k].shape, torch.int32))
+        else:
+            arrays[k] = np.ascontiguousarray(inp[k]).view(np.uint16)
+            specs.append((k, arrays[k].shape, torch.bfloat16))
+    flat = torch.zeros(ts._carve_bytes(specs), dtype=torch.uint8)
+    for k, view in ts._carve(flat, specs).items():
+        view.view(torch.uint8).copy_(torch.from_numpy(arrays[k].view(np.uint8).reshape(-1)).view(view.view(torch.uint8).shape))
+    return flat, specs
+
+
 class VerifyPass:
     def __init__(self, cfg: gen.VerifyConfig, inp: Dict[str, np.ndarray], with_attention: bool = True,
                  criterion: int = ts.CRIT_MARGIN):
         self.cfg = cfg
         B, T = cfg.B, cfg.T
         d: Dict[str, Optional[torch.Tensor]] = {}
-        for k in ("h", "W") + (("q", "k_tree", "v_tree", "k_cache", "v_cache") if with_attention else ()):
+        for k in ("W",) + (("k_cache", "v_cache") if with_attention else ()):
             d[k] = _bf16_dev(inp[k])
-        for k in ("parent", "tok", "ctx_len", "block_table", "seq_index"):
+        for k in ("ctx_len", "block_table", "seq_index"):
             d[k] = None if inp.get(k) is None else _i32_dev(inp[k])
+        # the per-round inputs sit back to back in two device buffers, in the order the host-buffer
+        # entry point copies them, so that each group arrives in one transfer
+        self._round_groups = [("parent", "tok", "h")] + ([("q", "k_tree", "v_tree")] if with_attention else [])
+        for group in self._round_groups:
+            flat, specs = _pack_round_inputs(inp, group)
+            d.update(ts._carve(flat.cuda(), specs))
         self.dev = d
         seqs = list(range(B)) if inp.get("seq_index") is None else [int(s) for s in inp["seq_index"]]
         self.seqs = seqs
@@ -75,15 +98,20 @@ class VerifyPass:
 
     # ---- the same pass with the per-round inputs and results in pinned host memory
     def prepare_host(self, inp: Dict[str, np.ndarray]):
-        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        """Pinned host copies of the per-round inputs and of the results, each group in one buffer
+        laid out like its device counterpart."""
         B, T = self.cfg.B, self.cfg.T
-        h = {"parent": pin(inp["parent"]), "tok": pin(inp["tok"]), "h": pin(inp["h"].view(np.int16))}
-        if self.attn_args is not None:
-            for k in ("q", "k_tree", "v_tree"):
-                h[k] = pin(inp[k].view(np.int16))
-        i32 = lambda *s: torch.zeros(s, dtype=torch.int32).pin_memory()
-        h.update(accept_len=i32(B), bonus_tok=i32(B), last_node=i32(B), path=i32(B, T),
-                 escalate=torch.zeros(B, dtype=torch.uint8).pin_memory())
+        h: Dict[str, torch.Tensor] = {}
+        self._host_flat = []
+        for group in self._round_groups:
+            flat, specs = _pack_round_inputs(inp, group)
+            flat = flat.pin_memory()
+            self._host_flat.append(flat)
+            h.update(ts._carve(flat, specs))
+        specs = ts.scan_out_specs(B, T)
+        out_flat = torch.zeros(ts._carve_bytes(specs), dtype=torch.uint8).pin_memory()
+        self._host_flat.append(out_flat)
+        h.update(ts._carve(out_flat, specs))
         self._host = h
         self._host_io = ts.host_io(**h)
         ins = ("parent", "tok", "h", "q", "k_tree", "v_tree")
