@@ -5,8 +5,8 @@
 // array once, coalesced (parent, token, top-1 index, the two probabilities); the margin test
 // of all nodes becomes two ballots, and the walk then runs on registers: the current node's
 // top-1 comes from a warp shuffle, the child match is a warp ballot. The accepted path is
-// collected in registers and stored as one row. A second kernel compacts the escalated
-// sequence ids in order.
+// collected in registers and stored as one row. The ordered list of escalated sequence ids is
+// made by the same block when the batch has at most 32 sequences, by a second kernel otherwise.
 #include "host_common.h"
 
 namespace trispec {
@@ -20,13 +20,8 @@ __device__ __forceinline__ float scan_feature(const trispec_scan_args& a, long l
   return __ldg(a.in.p_top1 + idx) - __ldg(a.in.p_top2 + idx);
 }
 
-__global__ void __launch_bounds__(kScanThreads)
-accept_scan_kernel(trispec_scan_args a) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int lane = threadIdx.x & 31;
-  const long long b = static_cast<long long>(blockIdx.x) * (kScanThreads / 32) + (threadIdx.x >> 5);
-  if (b >= a.B) return;
+// The walk of one sequence by one warp; writes the sequence's outputs and returns its escalation flag.
+__device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const long long b, const int lane) {
   const int T = a.T;
   const long long base = b * T;
   int32_t* path = a.path + base;
@@ -43,7 +38,7 @@ accept_scan_kernel(trispec_scan_args a) {
       if (a.near_thr) a.near_thr[b] = 0;
       if (a.esc_index) a.esc_index[b] = -1;
     }
-    return;
+    return 0;
   }
 
   // nodes `lane` and `lane + 32` of this sequence
@@ -125,6 +120,40 @@ accept_scan_kernel(trispec_scan_args a) {
     a.bonus_tok[b] = bonus;
     a.last_node[b] = cur;
     if (a.near_thr) a.near_thr[b] = near;
+  }
+  return esc;
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+accept_scan_kernel(trispec_scan_args a) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const long long b = static_cast<long long>(blockIdx.x) * (kScanThreads / 32) + (threadIdx.x >> 5);
+  if (b >= a.B) return;
+  scan_sequence(a, b, lane);
+}
+
+// Up to 32 sequences (a decode batch): one block, one warp per sequence, and the ordered list of
+// escalated sequences is made by the same block from a ballot of the flags, which saves the second
+// launch of the general path.
+constexpr int kScanSmallMax = 32;
+__global__ void __launch_bounds__(32 * kScanSmallMax)
+accept_scan_small_kernel(trispec_scan_args a) {
+  __shared__ int s_esc[kScanSmallMax];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int esc = (warp < a.B) ? scan_sequence(a, warp, lane) : 0;
+  if (lane == 0) s_esc[warp] = esc;
+  __syncthreads();
+  if (warp == 0 && a.esc_index) {
+    const bool flag = lane < a.B && lane < static_cast<int>(blockDim.x >> 5) && s_esc[lane] != 0;
+    const unsigned m = __ballot_sync(0xffffffffu, flag);
+    const int n = __popc(m);
+    if (flag) a.esc_index[__popc(m & ((1u << lane) - 1u))] = lane;
+    if (lane >= n && lane < a.B) a.esc_index[lane] = -1;
+    if (lane == 0) *a.n_escalated = n;
   }
 }
 
@@ -227,6 +256,11 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
   if ((a->q_draft == nullptr) != (a->u_accept == nullptr)) return TRISPEC_ERR_INVALID_ARG;
   if (a->q_draft && !a->in.p_draft) return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (a->B <= kScanSmallMax) {
+    TRISPEC_CUDA_OK(launch_dependent(accept_scan_small_kernel, 1u, static_cast<unsigned>(32 * a->B), 0, st, 1, *a));
+    count_launch();
+    return TRISPEC_OK;
+  }
   const int per_block = kScanThreads / 32;
   unsigned grid = static_cast<unsigned>((static_cast<long long>(a->B) + per_block - 1) / per_block);
   TRISPEC_CUDA_OK(launch_dependent(accept_scan_kernel, grid, kScanThreads, 0, st, 1, *a));
