@@ -14,13 +14,17 @@ namespace trispec {
 constexpr int kScanThreads = 256;  // 8 sequences per block
 
 // the proxy feature the routing criterion looks at (margin of Eq. 8 by default)
+template <int kCrit>
 __device__ __forceinline__ float scan_feature(const trispec_scan_args& a, long long idx) {
-  if (a.criterion == TRISPEC_CRIT_TOP1) return __ldg(a.in.p_top1 + idx);
-  if (a.criterion == TRISPEC_CRIT_ENTROPY) return __ldg(a.in.entropy + idx);
+  if (kCrit == TRISPEC_CRIT_TOP1) return __ldg(a.in.p_top1 + idx);
+  if (kCrit == TRISPEC_CRIT_ENTROPY) return __ldg(a.in.entropy + idx);
   return __ldg(a.in.p_top1 + idx) - __ldg(a.in.p_top2 + idx);
 }
 
 // The walk of one sequence by one warp; writes the sequence's outputs and returns its escalation flag.
+// The routing criterion and the acceptance rule are compile-time switches: the kernel is short and
+// latency-bound, and the plain case (margin rule, greedy acceptance) pays for nothing else.
+template <int kCrit, bool kStochastic>
 __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const long long b, const int lane) {
   const int T = a.T;
   const long long base = b * T;
@@ -49,8 +53,8 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
     par0 = __ldg(a.parent + base + lane); tok0 = __ldg(a.tok + base + lane);
     top0 = __ldg(a.in.top1_idx + base + lane);
     if (proxy) {
-      const float f = scan_feature(a, base + lane);
-      tr0 = (a.criterion == TRISPEC_CRIT_ENTROPY) ? (f <= a.lambda) : (f >= a.lambda);
+      const float f = scan_feature<kCrit>(a, base + lane);
+      tr0 = (kCrit == TRISPEC_CRIT_ENTROPY) ? (f <= a.lambda) : (f >= a.lambda);
       nr0 = fabsf(f - a.lambda) < 1e-3f;
     }
   }
@@ -58,8 +62,8 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
     par1 = __ldg(a.parent + base + lane + 32); tok1 = __ldg(a.tok + base + lane + 32);
     top1v = __ldg(a.in.top1_idx + base + lane + 32);
     if (proxy) {
-      const float f = scan_feature(a, base + lane + 32);
-      tr1 = (a.criterion == TRISPEC_CRIT_ENTROPY) ? (f <= a.lambda) : (f >= a.lambda);
+      const float f = scan_feature<kCrit>(a, base + lane + 32);
+      tr1 = (kCrit == TRISPEC_CRIT_ENTROPY) ? (f <= a.lambda) : (f >= a.lambda);
       nr1 = fabsf(f - a.lambda) < 1e-3f;
     }
   }
@@ -69,7 +73,7 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
   const unsigned long long near_bits =
       __ballot_sync(0xffffffffu, nr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, nr1)) << 32);
   // Bernoulli acceptance of Eq. 6 for every node at once: bit c = child c passes its test
-  const bool stochastic = a.q_draft != nullptr;
+  constexpr bool stochastic = kStochastic;
   unsigned long long passes = ~0ull;
   if (stochastic) {
     bool ps0 = false, ps1 = false;
@@ -124,6 +128,7 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
   return esc;
 }
 
+template <int kCrit, bool kStochastic>
 __global__ void __launch_bounds__(kScanThreads)
 accept_scan_kernel(trispec_scan_args a) {
   pdl_launch_dependents();
@@ -131,20 +136,21 @@ accept_scan_kernel(trispec_scan_args a) {
   const int lane = threadIdx.x & 31;
   const long long b = static_cast<long long>(blockIdx.x) * (kScanThreads / 32) + (threadIdx.x >> 5);
   if (b >= a.B) return;
-  scan_sequence(a, b, lane);
+  scan_sequence<kCrit, kStochastic>(a, b, lane);
 }
 
 // Up to 32 sequences (a decode batch): one block, one warp per sequence, and the ordered list of
 // escalated sequences is made by the same block from a ballot of the flags, which saves the second
 // launch of the general path.
 constexpr int kScanSmallMax = 32;
+template <int kCrit, bool kStochastic>
 __global__ void __launch_bounds__(32 * kScanSmallMax)
 accept_scan_small_kernel(trispec_scan_args a) {
   __shared__ int s_esc[kScanSmallMax];
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int esc = (warp < a.B) ? scan_sequence(a, warp, lane) : 0;
+  const int esc = (warp < a.B) ? scan_sequence<kCrit, kStochastic>(a, warp, lane) : 0;
   if (lane == 0) s_esc[warp] = esc;
   __syncthreads();
   if (warp == 0 && a.esc_index) {
@@ -256,14 +262,26 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
   if ((a->q_draft == nullptr) != (a->u_accept == nullptr)) return TRISPEC_ERR_INVALID_ARG;
   if (a->q_draft && !a->in.p_draft) return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // kernel instance for (criterion, acceptance rule); TARGET mode reads no feature: margin instance
+  const int crit = (a->mode == TRISPEC_MODE_PROXY) ? a->criterion : TRISPEC_CRIT_MARGIN;
+  const int which = crit * 2 + (a->q_draft ? 1 : 0);
+  typedef void (*ScanKernel)(trispec_scan_args);
+  static const ScanKernel small_k[6] = {
+      accept_scan_small_kernel<TRISPEC_CRIT_MARGIN, false>,  accept_scan_small_kernel<TRISPEC_CRIT_MARGIN, true>,
+      accept_scan_small_kernel<TRISPEC_CRIT_TOP1, false>,    accept_scan_small_kernel<TRISPEC_CRIT_TOP1, true>,
+      accept_scan_small_kernel<TRISPEC_CRIT_ENTROPY, false>, accept_scan_small_kernel<TRISPEC_CRIT_ENTROPY, true>};
+  static const ScanKernel big_k[6] = {
+      accept_scan_kernel<TRISPEC_CRIT_MARGIN, false>,  accept_scan_kernel<TRISPEC_CRIT_MARGIN, true>,
+      accept_scan_kernel<TRISPEC_CRIT_TOP1, false>,    accept_scan_kernel<TRISPEC_CRIT_TOP1, true>,
+      accept_scan_kernel<TRISPEC_CRIT_ENTROPY, false>, accept_scan_kernel<TRISPEC_CRIT_ENTROPY, true>};
   if (a->B <= kScanSmallMax) {
-    TRISPEC_CUDA_OK(launch_dependent(accept_scan_small_kernel, 1u, static_cast<unsigned>(32 * a->B), 0, st, 1, *a));
+    TRISPEC_CUDA_OK(launch_dependent(small_k[which], 1u, static_cast<unsigned>(32 * a->B), 0, st, 1, *a));
     count_launch();
     return TRISPEC_OK;
   }
   const int per_block = kScanThreads / 32;
   unsigned grid = static_cast<unsigned>((static_cast<long long>(a->B) + per_block - 1) / per_block);
-  TRISPEC_CUDA_OK(launch_dependent(accept_scan_kernel, grid, kScanThreads, 0, st, 1, *a));
+  TRISPEC_CUDA_OK(launch_dependent(big_k[which], grid, kScanThreads, 0, st, 1, *a));
   count_launch();
   if (a->esc_index) {
     TRISPEC_CUDA_OK(launch_dependent(esc_compact_kernel, 1, kCompactThreads, 0, st, 1,
