@@ -362,33 +362,21 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         }
       }
       const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
-      if (i > 0) {
-        mbar_wait(o_bar, (i - 1) & 1u, p.dev_status);   // P V of the previous tile is complete
-        tc_fence_after();
-      }
+      // new reference maximum (lazy: only when the running one is exceeded by more than the
+      // threshold); the rescaling of O it implies is applied further down, after P V of the
+      // previous tile, so that the exponentials below do not wait for that MMA
+      bool need = false;
+      float f = 1.f;
       if (i == 0) {
         m_ref = tmax;
       } else {
-        const bool need = tmax > m_ref + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-          float f = 1.f;
-          if (need) { f = (m_ref == -INFINITY) ? 0.f : ex2f(m_ref - tmax); m_ref = tmax; l *= f; }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * f);
-            tmem_st32(tmem_base + lane_base + AT_TM_O + c * 32, o);
-          }
-          tc_wait_st();
-        }
+        need = tmax > m_ref + kRescaleThreshold;
+        if (need) { f = (m_ref == -INFINITY) ? 0.f : ex2f(m_ref - tmax); m_ref = tmax; l *= f; }
       }
       const float nmu = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nmu2 = make_float2(nmu, nmu);
-      uint8_t* prow = sP + row * 128;
+      uint4 pk[8];
 #pragma unroll
       for (int cch = 0; cch < 8; ++cch) {
         float e[8];
@@ -401,11 +389,28 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
           e[j + 1] = ex2f(t.y);
           ls[(j >> 1) & 1] = fadd2(ls[(j >> 1) & 1], make_float2(e[j], e[j + 1]));
         }
-        uint4 pk;
-        pk.x = pack_bf16(e[0], e[1]); pk.y = pack_bf16(e[2], e[3]);
-        pk.z = pack_bf16(e[4], e[5]); pk.w = pack_bf16(e[6], e[7]);
-        *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk;
+        pk[cch].x = pack_bf16(e[0], e[1]); pk[cch].y = pack_bf16(e[2], e[3]);
+        pk[cch].z = pack_bf16(e[4], e[5]); pk[cch].w = pack_bf16(e[6], e[7]);
       }
+      if (i > 0) {
+        mbar_wait(o_bar, (i - 1) & 1u, p.dev_status);   // P V of the previous tile is complete: P is free, O stable
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_base + lane_base + AT_TM_O + c * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * f);
+            tmem_st32(tmem_base + lane_base + AT_TM_O + c * 32, o);
+          }
+          tc_wait_st();
+        }
+      }
+      uint8_t* prow = sP + row * 128;
+#pragma unroll
+      for (int cch = 0; cch < 8; ++cch) *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk[cch];
       l += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
       if (nvalid < AT_BN) {
         // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)

@@ -24,6 +24,7 @@ struct HostPassStreams {
   cudaStream_t copy = nullptr;
   cudaEvent_t fork = nullptr, copied = nullptr;
   bool ready = false;
+  std::mutex enqueue;   // the stream and the events are shared by every caller on this device
 };
 static int host_pass_streams(HostPassStreams** out) {
   static HostPassStreams per_dev[64];
@@ -80,9 +81,13 @@ extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree
     return cudaSuccess;
   };
   HostPassStreams* hs = nullptr;
+  std::unique_lock<std::mutex> enqueue_lock;
   if (attn) {
     int rc = host_pass_streams(&hs);
     if (rc != TRISPEC_OK) return rc;
+    // one caller at a time records and waits on the shared events (host threads driving
+    // different streams of one device would otherwise pick up each other's records)
+    enqueue_lock = std::unique_lock<std::mutex>(hs->enqueue);
     // the side stream may not overwrite q / k_tree / v_tree before earlier work on `stream`
     // (a previous pass reading them) is done
     TRISPEC_CUDA_OK(cudaEventRecord(hs->fork, st));
