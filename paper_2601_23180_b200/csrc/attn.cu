@@ -35,9 +35,10 @@ namespace trispec {
 constexpr int AT_BM = 128;      // rows per M tile
 constexpr int AT_BN = 64;       // keys per tile (= paged block size)
 constexpr int AT_D = 128;
-constexpr int AT_STAGES = 3;
+constexpr int AT_STAGES = 3;        // K ring; the V ring has 3 slots with one P buffer, 2 with two
 constexpr int AT_BOX_BYTES = 64 * 64 * 2;               // 64 rows x 64 elements
-constexpr int AT_KV_STAGE_BYTES = 4 * AT_BOX_BYTES;     // K (2 boxes) + V (2 boxes) = 32 KB
+constexpr int AT_KV_STAGE_BYTES = 4 * AT_BOX_BYTES;     // one K slot + one V slot = 32 KB
+constexpr int AT_TILE_BYTES = 2 * AT_BOX_BYTES;         // a K tile or a V tile: 64 keys x 128 dims bf16 = 16 KB
 constexpr int AT_P_BYTES = AT_BM * AT_BN * 2;           // 16 KB
 constexpr int AT_THREADS = 192;
 constexpr int AT_SMEM_USED = AT_STAGES * AT_KV_STAGE_BYTES + AT_P_BYTES + 256;
@@ -52,7 +53,8 @@ constexpr int AT_PART_PITCH = AT_D * 2 + 16;             // bytes per row of the
 constexpr int AT_PART_ML_OFF = AT_BM * AT_PART_PITCH;    // (m, l) pairs follow the partial rows
 constexpr int AT_PART_ML2_OFF = AT_PART_ML_OFF + AT_BM * 8;   // gathered (m, l) of every split for this CTA's rows
 constexpr int AT_PART_ML2_MAX = AT_BM + 2 * 8;                // n_splits x rows per CTA, rows rounded up to even
-static_assert(AT_PART_ML2_OFF + AT_PART_ML2_MAX * 8 <= AT_STAGES * AT_KV_STAGE_BYTES, "partial must fit in the K/V ring");
+static_assert(AT_PART_ML2_OFF + AT_PART_ML2_MAX * 8 <= (AT_STAGES + 2) * AT_TILE_BYTES,
+              "partial must fit in the K ring plus the shorter V ring");
 
 struct AttnParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits;
@@ -86,7 +88,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
-template <bool kCluster>
+// NP = number of P buffers. With one, the softmax of tile i waits for O += P V of tile i - 1 before
+// it may overwrite P; with two (and a V ring of two slots instead of three, same shared memory) it
+// waits for tile i - 2, which has long completed: the variant for short tile loops, which are bound
+// by the S -> softmax -> P V chain of a CTA rather than by the bytes in flight.
+template <bool kCluster, int NP>
 __global__ void __launch_bounds__(AT_THREADS, 2)
 verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                          const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt,
@@ -121,19 +127,21 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   const bool idle_cta = (split > last_split) || misaligned;
   if (!kCluster && idle_cta) return;           // the merge kernel skips it too
 
-  uint8_t* sKV = smem;
-  uint8_t* sP = sKV + AT_STAGES * AT_KV_STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + AT_P_BYTES);
+  constexpr int NV = (NP == 2) ? 2 : 3;         // V ring slots: K ring + V ring + P buffers = 112 KB either way
+  uint8_t* sK = smem;                           // [AT_STAGES] K tiles
+  uint8_t* sV = sK + AT_STAGES * AT_TILE_BYTES; // [NV] V tiles
+  uint8_t* sP = sV + NV * AT_TILE_BYTES;        // [NP] P tiles
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + AT_STAGES * AT_KV_STAGE_BYTES + AT_P_BYTES);
   uint64_t* k_full = bars;                      // [3]  K tile landed
   uint64_t* k_empty = bars + AT_STAGES;         // [3]  S = Q K^T has consumed it
-  uint64_t* v_full = bars + 2 * AT_STAGES;      // [3]  V tile landed
-  uint64_t* v_empty = bars + 3 * AT_STAGES;     // [3]  O += P V has consumed it
+  uint64_t* v_full = bars + 2 * AT_STAGES;      // [NV] V tile landed
+  uint64_t* v_empty = bars + 3 * AT_STAGES;     // [NV] O += P V has consumed it
   uint64_t* s_bar = bars + 4 * AT_STAGES;       // S ready in TMEM
   uint64_t* s_free = s_bar + 1;                 // S read into registers by the 128 softmax threads
-  uint64_t* o_bar = s_bar + 2;                  // O += P V complete (P buffer free, O stable)
-  uint64_t* p_bar = s_bar + 3;                  // P written by the 128 softmax threads
-  uint64_t* q_bar = s_bar + 4;                  // Q stored to TMEM by the 128 softmax threads
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_bar + 5);
+  uint64_t* q_bar = s_bar + 2;                  // Q stored to TMEM by the 128 softmax threads
+  uint64_t* o_bar = s_bar + 3;                  // [NP] O += P V of a tile using P buffer b complete (buffer free)
+  uint64_t* p_bar = s_bar + 5;                  // [NP] P buffer b written by the 128 softmax threads
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_bar + 7);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t* sPartO = smem;                                               // reuses the K/V ring at the end
@@ -145,16 +153,16 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     // the loader owns the ring barriers: it signals the set-up barrier without waiting on it
     // and starts streaming while the other warps are still allocating TMEM and storing Q
     if (lane == 0) {
-      for (int i = 0; i < AT_STAGES; ++i) {
-        mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
-      }
+      for (int i = 0; i < AT_STAGES; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
+      for (int i = 0; i < NV; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
       fence_mbar_init();
     }
     __syncwarp();
     asm volatile("bar.arrive 1, 192;" ::: "memory");
   } else {
     if (threadIdx.x == 0) {
-      mbar_init(s_bar, 1); mbar_init(s_free, 128); mbar_init(o_bar, 1); mbar_init(p_bar, 128); mbar_init(q_bar, 128);
+      mbar_init(s_bar, 1); mbar_init(s_free, 128); mbar_init(q_bar, 128);
+      for (int i = 0; i < NP; ++i) { mbar_init(o_bar + i, 1); mbar_init(p_bar + i, 128); }
       fence_mbar_init();
     }
     if (warp == 5) {
@@ -183,9 +191,9 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       };
       auto load_tile = [&](int i, bool is_v, int blk) {
         const bool tree = has_tree && (i == n_tiles - 1);
-        const int stage = i % AT_STAGES;
+        const int stage = is_v ? i % NV : i % AT_STAGES;
         uint64_t* full = (is_v ? v_full : k_full) + stage;
-        uint8_t* dst = sKV + stage * AT_KV_STAGE_BYTES + (is_v ? 2 * AT_BOX_BYTES : 0);
+        uint8_t* dst = (is_v ? sV : sK) + stage * AT_TILE_BYTES;
         mbar_expect_tx(full, 2 * AT_BOX_BYTES);
         if (tree) {
           const CUtensorMap* tm = is_v ? &tm_vt : &tm_kt;
@@ -212,7 +220,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
           ++next_k;
           progressed = true;
         }
-        if (mbar_test(v_empty + next_v % AT_STAGES, ((next_v / AT_STAGES) & 1u) ^ 1u)) {
+        if (mbar_test(v_empty + next_v % NV, ((next_v / NV) & 1u) ^ 1u)) {
           load_tile(next_v, true, vblk0);
           vblk0 = vblk1;
           vblk1 = block_id(t_begin + next_v + 2);
@@ -237,7 +245,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(AT_BM, AT_BN, false, false);
       const uint32_t idesc_o = idesc_bf16(AT_BM, AT_D, false, true);
-      const uint32_t sKV_u = base_u32, sP_u = sKV_u + AT_STAGES * AT_KV_STAGE_BYTES;
+      const uint32_t sK_u = base_u32, sV_u = sK_u + AT_STAGES * AT_TILE_BYTES, sP_u = sV_u + NV * AT_TILE_BYTES;
       mbar_wait(q_bar, 0, p.dev_status);
       tc_fence_after();
       int next_s = 0, next_pv = 0;
@@ -248,7 +256,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             mbar_test(k_full + next_s % AT_STAGES, (next_s / AT_STAGES) & 1u)) {
           const int stage = next_s % AT_STAGES;
           tc_fence_after();
-          const uint32_t sk = sKV_u + stage * AT_KV_STAGE_BYTES;
+          const uint32_t sk = sK_u + stage * AT_TILE_BYTES;
 #pragma unroll
           for (int kk = 0; kk < AT_D / 16; ++kk) {
             const uint64_t bd = smem_desc_sw128(sk + (kk >> 2) * AT_BOX_BYTES + (kk & 3) * 32, 1024, 16);
@@ -259,20 +267,21 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
           ++next_s;
           progressed = true;
         }
-        if (next_pv < next_s && mbar_test(p_bar, next_pv & 1u) &&
-            mbar_test(v_full + next_pv % AT_STAGES, (next_pv / AT_STAGES) & 1u)) {
-          const int stage = next_pv % AT_STAGES;
+        if (next_pv < next_s && mbar_test(p_bar + next_pv % NP, (next_pv / NP) & 1u) &&
+            mbar_test(v_full + next_pv % NV, (next_pv / NV) & 1u)) {
+          const int stage = next_pv % NV;
           tc_fence_after();
-          const uint32_t sv = sKV_u + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
+          const uint32_t sv = sV_u + stage * AT_TILE_BYTES;
+          const uint32_t sp = sP_u + (next_pv % NP) * AT_P_BYTES;
 #pragma unroll
           for (int kk = 0; kk < AT_BN / 16; ++kk) {
-            const uint64_t ad = smem_desc_sw128(sP_u + kk * 32, 1024, 16);
+            const uint64_t ad = smem_desc_sw128(sp + kk * 32, 1024, 16);
             // V: MN-major, 64-dim blocks 8 KB apart (LBO), 8-key groups 1 KB apart (SBO)
             const uint64_t bd = smem_desc_sw128(sv + kk * 2048, 1024, AT_BOX_BYTES);
             tc_mma_ss(tmem_base + AT_TM_O, ad, bd, idesc_o, (next_pv | kk) != 0);
           }
           tc_commit(v_empty + stage);
-          tc_commit(o_bar);
+          tc_commit(o_bar + next_pv % NP);
           ++next_pv;
           progressed = true;
         }
@@ -316,7 +325,6 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     float m_ref = -INFINITY, l = 0.f;
 
     for (int i = 0; i < n_tiles; ++i) {
-      const int stage = i % AT_STAGES;
       const bool tree = has_tree && (i == n_tiles - 1);
       mbar_wait(s_bar, i & 1u, p.dev_status);
       tc_fence_after();
@@ -392,10 +400,17 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         pk[cch].x = pack_bf16(e[0], e[1]); pk[cch].y = pack_bf16(e[2], e[3]);
         pk[cch].z = pack_bf16(e[4], e[5]); pk[cch].w = pack_bf16(e[6], e[7]);
       }
-      if (i > 0) {
-        mbar_wait(o_bar, (i - 1) & 1u, p.dev_status);   // P V of the previous tile is complete: P is free, O stable
+      if (i >= NP) {
+        // the P buffer is free once O += P V of the tile that used it last is complete
+        mbar_wait(o_bar + i % NP, ((i / NP) - 1) & 1u, p.dev_status);
         tc_fence_after();
+      }
+      if (i > 0) {
         if (__any_sync(0xffffffffu, need)) {
+          if (NP > 1) {   // O is stable only after the previous tile's P V
+            mbar_wait(o_bar + (i - 1) % NP, ((i - 1) / NP) & 1u, p.dev_status);
+            tc_fence_after();
+          }
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t o[32];
@@ -408,14 +423,14 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
           tc_wait_st();
         }
       }
-      uint8_t* prow = sP + row * 128;
+      uint8_t* prow = sP + (i % NP) * AT_P_BYTES + row * 128;
 #pragma unroll
       for (int cch = 0; cch < 8; ++cch) *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk[cch];
       l += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
       if (nvalid < AT_BN) {
         // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
-        mbar_wait(v_full + stage, (i / AT_STAGES) & 1u, p.dev_status);
-        uint8_t* sv = sKV + stage * AT_KV_STAGE_BYTES + 2 * AT_BOX_BYTES;
+        mbar_wait(v_full + i % NV, (i / NV) & 1u, p.dev_status);
+        uint8_t* sv = sV + (i % NV) * AT_TILE_BYTES;
         for (int e = threadIdx.x; e < (AT_BN - nvalid) * 16; e += 128) {
           const int r = nvalid + (e >> 4), c16 = e & 15;
           *reinterpret_cast<uint4*>(sv + (c16 >> 3) * AT_BOX_BYTES + r * 128 + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
@@ -423,10 +438,10 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       }
       fence_async_smem();
       tc_fence_before();
-      mbar_arrive(p_bar);
+      mbar_arrive(p_bar + i % NP);
     }
     // ---------------------------------------------------------------- epilogue
-    mbar_wait(o_bar, (n_tiles - 1) & 1u, p.dev_status);
+    mbar_wait(o_bar + (n_tiles - 1) % NP, ((n_tiles - 1) / NP) & 1u, p.dev_status);   // the last P V, hence all of them
     tc_fence_after();
     if (kCluster && p.n_splits == 1) {
       // a single split is the whole result: normalise and store it straight from tensor memory
@@ -741,10 +756,16 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
     tm_k = tm_kt;   // never dereferenced: every sequence has zero context tiles
     tm_v = tm_vt;
   }
-  static bool smem_set_c[64] = {}, smem_set_w[64] = {};
-  rc = pl.cluster
-           ? ensure_smem_limit(reinterpret_cast<const void*>(verify_attn_split_kernel<true>), AT_SMEM_BYTES, smem_set_c)
-           : ensure_smem_limit(reinterpret_cast<const void*>(verify_attn_split_kernel<false>), AT_SMEM_BYTES, smem_set_w);
+  // Two P buffers for CTAs with few tiles (their time is the S -> softmax -> P V chain, tile after
+  // tile, and never reaches the HBM-bound steady state); one P buffer and the deeper V ring for long
+  // tile loops. Measured: proxy_tree (16 tiles per CTA) 45.1 -> 43.2 us with two; long_paged
+  // (128-512) 1005 -> 1023 us, target_escalated (64) 150 -> 154 us, llama_tree (129) unchanged.
+  const bool two_p = pl.tiles_max / pl.n_splits <= 32;
+  typedef void (*AttnKernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, AttnParams);
+  const AttnKernel kernel = pl.cluster ? (two_p ? verify_attn_split_kernel<true, 2> : verify_attn_split_kernel<true, 1>)
+                                       : (two_p ? verify_attn_split_kernel<false, 2> : verify_attn_split_kernel<false, 1>);
+  static bool smem_set[4][64] = {};
+  rc = ensure_smem_limit(reinterpret_cast<const void*>(kernel), AT_SMEM_BYTES, smem_set[(pl.cluster ? 2 : 0) + (two_p ? 1 : 0)]);
   if (rc != TRISPEC_OK) return rc;
   AttnParams p;
   p.T = a->T; p.Hq = a->Hq; p.Hkv = a->Hkv; p.G = pl.G; p.NPT = pl.NPT; p.n_mt = pl.n_mt;
@@ -760,13 +781,13 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   p.lse = a->lse;
   p.dev_status = a->dev_status;
   if (pl.cluster) {
-    TRISPEC_CUDA_OK(launch_dependent(verify_attn_split_kernel<true>, static_cast<unsigned>(pl.items), AT_THREADS,
+    TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(pl.items), AT_THREADS,
                                      AT_SMEM_BYTES, st, static_cast<unsigned>(pl.n_splits), tm_k, tm_v, tm_kt, tm_vt,
                                      p));
     count_launch();
     return TRISPEC_OK;
   }
-  TRISPEC_CUDA_OK(launch_dependent(verify_attn_split_kernel<false>, static_cast<unsigned>(pl.items), AT_THREADS,
+  TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(pl.items), AT_THREADS,
                                    AT_SMEM_BYTES, st, 1, tm_k, tm_v, tm_kt, tm_vt, p));
   count_launch();
 
