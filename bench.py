@@ -398,9 +398,15 @@ def run_only(args, cfg):
         inp.update({k: v for k, v in gen.make_inputs(small, with_attention=False).items() if k in ("h", "W")})
         pas = runner.VerifyPass(small, inp)
         Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
-        byts = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 4 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
+        rows = cfg.T
+        if args.tree_nodes is not None:          # pruned trees: fewer query rows per sequence
+            rows = max(0, min(cfg.T, args.tree_nodes))
+            n_nodes = torch.full((cfg.B,), rows, dtype=torch.int32, device="cuda")
+            pas.attn_args.n_nodes = n_nodes.data_ptr()
+            out["config"]["tree_nodes"] = rows
+        byts = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 4 + 2 * n_seq * rows * cfg.Hq * cfg.D * 2
         ms = timed(lambda: ts.trispec_verify_attn(pas.attn_args), byts)
-        flops = 4.0 * cfg.T * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
+        flops = 4.0 * rows * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
         roof = _roof(peaks, flops, byts, ms)
         roof["kernel"] = "verify_attn_split_kernel"
     else:
@@ -457,6 +463,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan", "prune", "commit", "sample"],
                     help="time one entry point alone (L2 flushed before each call) instead of the pass")
+    ap.add_argument("--tree-nodes", type=int, default=None,
+                    help="with --only attention: every tree keeps only its first N nodes (a pruned tree)")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the number of sequences of the workload (reduced copies for profiler captures)")
     args = ap.parse_args()

@@ -95,6 +95,11 @@ int trispec_build_tree_mask(const trispec_tree_args* a, void* stream);
  *    seq_index (optional, int32 [B_active], device): only these sequences are computed;
  *      NULL = all B (then B_active is ignored).
  *    lse (optional) f32 [B][Hq][T]: log-sum-exp of the scaled scores.
+ *    n_nodes (optional, int32 [B], device): sequence b has only its first n_nodes[b] tree
+ *      nodes (a pruned tree: n_keep of trispec_prune_tree, the branches that are passed on to
+ *      the target in routing case (ii)); rows o[b][i] and lse of nodes i >= n_nodes[b] are
+ *      neither computed nor written, and whole 128-row tiles past them cost nothing. The
+ *      mask rows of the remaining nodes must not name nodes >= n_nodes[b]. NULL = T nodes.
  *    workspace: device scratch of at least trispec_verify_attn_workspace(a) bytes,
  *      256-byte aligned; contents are undefined before and after the call. The query
  *      returns 0 (and workspace may be NULL) whenever the context is cut into at most 8
@@ -118,6 +123,7 @@ typedef struct {
   void* workspace;
   size_t workspace_bytes;
   int32_t* dev_status;
+  const int32_t* n_nodes;
 } trispec_attn_args;
 size_t trispec_verify_attn_workspace(const trispec_attn_args* a);
 int trispec_verify_attn(const trispec_attn_args* a, void* stream);

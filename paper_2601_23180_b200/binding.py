@@ -40,7 +40,7 @@ class AttnArgs(C.Structure):
                 ("block_size", _i), ("max_blocks_per_seq", _i), ("block_table", _vp),
                 ("ctx_len", _vp), ("mask", _vp), ("seq_index", _vp), ("B_active", _i),
                 ("o", _vp), ("lse", _vp), ("workspace", _vp), ("workspace_bytes", _sz),
-                ("dev_status", _vp)]
+                ("dev_status", _vp), ("n_nodes", _vp)]
 
 
 class Stats(C.Structure):
@@ -187,7 +187,7 @@ def tree_args(parent: torch.Tensor, mask: torch.Tensor, depth: Optional[torch.Te
 
 
 def attn_args(q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, scale, o, workspace=None,
-              block_table=None, block_size=64, seq_index=None, lse=None, dev_status=None) -> AttnArgs:
+              block_table=None, block_size=64, seq_index=None, lse=None, dev_status=None, n_nodes=None) -> AttnArgs:
     B, T, Hq, D = q.shape
     Hkv = k_tree.shape[2]
     a = AttnArgs()
@@ -208,8 +208,9 @@ def attn_args(q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, scale, o, work
     a.workspace = _p(workspace)
     a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     a.dev_status = _p(dev_status)
+    a.n_nodes = _p(n_nodes)
     return _hold(a, q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, o, workspace, block_table, seq_index, lse,
-                 dev_status)
+                 dev_status, n_nodes)
 
 
 def lmhead_args(h, W, parent, tok, logit_scale, stats, workspace=None, seq_index=None,

@@ -62,6 +62,7 @@ struct AttnParams {
   float scale_log2;
   const uint16_t* q;
   const int32_t *block_table, *ctx_len, *seq_index;
+  const int32_t* n_nodes;   // tree nodes per sequence (a pruned tree), or null = T
   const uint64_t* mask;
   float* part_o;    // [items][128][128]   (workspace mode only)
   float* part_ml;   // [items][128][2]
@@ -107,6 +108,8 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   const int a = idx / p.Hkv;
   const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
   const int L = __ldg(p.ctx_len + b);
+  // a pruned tree has fewer nodes: rows past them are not computed, M tiles past them do nothing
+  const int nn = p.n_nodes ? max(0, min(p.T, __ldg(p.n_nodes + b))) : p.T;
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
   // every sequence spreads its own context tiles evenly over the splits, so that the CTAs that
   // merge with each other finish together whatever the sequence's length
@@ -124,7 +127,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   if (misaligned && threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 7);   // shared window misaligned
   // a split past the end of this sequence's context has nothing to do; in cluster mode it
   // still takes part in the merge (with weight zero), so it may not leave early
-  const bool idle_cta = (split > last_split) || misaligned;
+  const bool idle_cta = (split > last_split) || misaligned || (mtile * p.NPT >= nn);
   if (!kCluster && idle_cta) return;           // the merge kernel skips it too
 
   constexpr int NV = (NP == 2) ? 2 : 3;         // V ring slots: K ring + V ring + P buffers = 112 KB either way
@@ -300,7 +303,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     // ------------------------------------------------------------------ softmax (warps 0-3)
     const int row = warp * 32 + lane;
     const int node = mtile * p.NPT + row / p.G;
-    const bool row_valid = (row < p.NPT * p.G) && (node < p.T);
+    const bool row_valid = (row < p.NPT * p.G) && (node < nn);
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     // Q row -> TMEM (A operand of S = Q K^T): lane = row, column c = dims (2c, 2c + 1)
     {
@@ -549,7 +552,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
       const int rl = 2 * pr + half;               // row within this CTA's slice
       const int row = split * rpc + rl;
       const int node = mtile * p.NPT + row / p.G;
-      const bool ok = (row < AT_BM) && (row < p.NPT * p.G) && (node < p.T);
+      const bool ok = (row < AT_BM) && (row < p.NPT * p.G) && (node < nn);
       uint4 v[8];
       float2 ml[8];
 #pragma unroll
@@ -602,7 +605,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 // ---------------------------------------------------------------------------------------
 struct AttnMergeParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits, n_seq;
-  const int32_t *ctx_len, *seq_index;
+  const int32_t *ctx_len, *seq_index, *n_nodes;
   const float *part_o, *part_ml;
   uint16_t* o;   // bf16 [B][T][Hq][128]
   float* lse;    // [B][Hq][T] or null
@@ -620,6 +623,7 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
   const int node = static_cast<int>((w / p.Hq) % p.T);
   const int a = static_cast<int>(w / (static_cast<long long>(p.Hq) * p.T));
   const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
+  if (p.n_nodes && node >= __ldg(p.n_nodes + b)) return;   // not a node of this (pruned) tree
   const int g = hq / p.G, j = hq % p.G;
   const int mtile = node / p.NPT;
   const int row = (node % p.NPT) * p.G + j;
@@ -775,6 +779,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   p.scale_log2 = a->scale * kLog2e;
   p.q = static_cast<const uint16_t*>(a->q);
   p.block_table = a->block_table; p.ctx_len = a->ctx_len; p.seq_index = a->seq_index; p.mask = a->mask;
+  p.n_nodes = a->n_nodes;
   p.part_o = static_cast<float*>(a->workspace);
   p.part_ml = p.part_o + pl.items * AT_BM * AT_D;
   p.o = static_cast<uint16_t*>(a->o);
@@ -794,7 +799,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   AttnMergeParams m;
   m.T = a->T; m.Hq = a->Hq; m.Hkv = a->Hkv; m.G = pl.G; m.NPT = pl.NPT; m.n_mt = pl.n_mt;
   m.n_splits = pl.n_splits; m.n_seq = pl.n_seq;
-  m.ctx_len = a->ctx_len; m.seq_index = a->seq_index;
+  m.ctx_len = a->ctx_len; m.seq_index = a->seq_index; m.n_nodes = a->n_nodes;
   m.part_o = p.part_o; m.part_ml = p.part_ml;
   m.o = static_cast<uint16_t*>(a->o); m.lse = a->lse;
   const long long rows = static_cast<long long>(pl.n_seq) * a->T * a->Hq;

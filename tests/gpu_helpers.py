@@ -80,7 +80,7 @@ def run_scan(stats_np, parent, tok, lam, mode, active=None, start_node=None, cri
     return {k: v.cpu().numpy() for k, v in out.items()}
 
 
-def run_attn(dev, cfg: gen.VerifyConfig, mask_dev, want_lse=True):
+def run_attn(dev, cfg: gen.VerifyConfig, mask_dev, want_lse=True, n_nodes=None):
     from paper_2601_23180_b200 import binding as ts
     B, T, Hq, D = dev["q"].shape
     o = torch.full((B, T, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
@@ -88,7 +88,8 @@ def run_attn(dev, cfg: gen.VerifyConfig, mask_dev, want_lse=True):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     a = ts.attn_args(dev["q"], dev["k_tree"], dev["v_tree"], mask_dev, dev["k_cache"], dev["v_cache"],
                      dev["ctx_len"], 1.0 / math.sqrt(D), o, block_table=dev.get("block_table"),
-                     block_size=cfg.block_size, seq_index=dev.get("seq_index"), lse=lse, dev_status=status)
+                     block_size=cfg.block_size, seq_index=dev.get("seq_index"), lse=lse, dev_status=status,
+                     n_nodes=None if n_nodes is None else i32_dev(n_nodes))
     ws = ts.alloc_workspace(ts.trispec_verify_attn_workspace(a))
     a.workspace, a.workspace_bytes = ws.data_ptr(), ws.numel()
     ts.trispec_verify_attn(a)

@@ -319,3 +319,32 @@ def test_fused_pass_with_entropy_routing():
         assert np.array_equal(got["scan"][k][clean], ref[k][clean]), k
     # the entropy criterion must route both ways on this input, or the test says nothing
     assert 0 < ref["escalate"].sum() < cfg.B
+
+
+@pytest.mark.parametrize("name,over,n_nodes", [
+    # G = 8: four M tiles of 16 nodes; whole tiles, part of a tile and nothing at all are left out
+    ("target_escalated", dict(B=5, n_active=5, L=700), [61, 30, 16, 5, 0]),
+    # one M tile, cluster merge over several splits
+    ("proxy_tree", dict(B=3, L=2000), [61, 1, 40]),
+    # more than 8 splits: the workspace merge kernel skips the rows too
+    ("proxy_tree", dict(B=2, L=9300, Hq=4, Hkv=2), [7, 61]),
+])
+def test_attention_of_pruned_trees(name, over, n_nodes):
+    """With n_nodes, a sequence's tree ends after its first n_nodes[b] nodes (parents precede children, so
+    a prefix of the nodes is a tree): those rows equal the oracle's, the others are never written."""
+    import tests.gpu_helpers as H
+    cfg = gen.small_variant(gen.CONFIGS[name], **over)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    dev = H.to_device(inp)
+    mask_dev, _ = H.run_tree_mask(dev["parent"])
+    o, lse = H.run_attn(dev, cfg, mask_dev, n_nodes=np.array(n_nodes, dtype=np.int32))
+    ref_mask, _ = orc.build_tree_mask(inp["parent"])
+    ref_o, ref_lse = orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], ref_mask, inp["k_cache"],
+                                     inp["v_cache"], inp["ctx_len"], 1.0 / math.sqrt(cfg.D),
+                                     block_table=inp.get("block_table"), block_size=cfg.block_size)
+    for b in range(cfg.B):
+        n = n_nodes[b]
+        if n:
+            assert np.abs(o[b, :n] - ref_o[b, :n]).max() <= 2e-2, b
+            assert np.abs(lse[b, :, :n] - ref_lse[b, :, :n]).max() <= 1e-3 * max(1.0, np.abs(ref_lse[b, :, :n]).max())
+        assert np.isnan(o[b, n:]).all() and np.isnan(lse[b, :, n:]).all(), b
