@@ -21,10 +21,16 @@
 // reads of the MMAs, P), which is why Q is kept out of shared memory: per tile the MMAs read
 // K, P and V only.
 // Warps 0-3: softmax. Warp 4: one thread streams K and V by TMA (no multicast) through two
-// independent 3-slot rings (a K slot is free once S has read it, a V slot after O += P V); it
+// independent rings (a K slot is free once S has read it, a V slot after O += P V); it
 // initialises the ring barriers itself and starts loading before the CTA-wide set-up barrier.
 // Warp 5: one thread issues the MMAs, polling for whichever of S(i+1) / P V(i) can go.
-// Two CTAs fit on one SM (~112 KB shared memory, 256 TMEM columns each).
+// A softmax thread computes and packs the exponentials of tile i before it waits for the P
+// buffer to be free, so that only the 16-byte stores of P sit behind that wait.
+// Two CTAs fit on one SM (~112 KB shared memory, 256 TMEM columns each). The 112 KB are either
+// K ring 3 + V ring 3 + one P buffer (long tile loops: bytes in flight) or K ring 3 + V ring 2 +
+// two P buffers (short loops: tile i waits for P V of tile i - 2 only).
+// A sequence may carry fewer than T tree nodes (a pruned tree): rows past its count are not
+// computed and M tiles past it do nothing.
 #include <math.h>
 
 #include "host_common.h"

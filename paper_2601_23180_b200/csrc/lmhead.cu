@@ -3,13 +3,14 @@
 // never reach global memory: each CTA streams a slice of the vocabulary through
 // tcgen05.mma (bf16 x bf16 -> fp32 in tensor memory) and its epilogue keeps, per row, a
 // running (max, sum of exponentials, top-1, top-2) in registers across all of its vocabulary
-// tiles. A small second kernel merges the per-slice partials and computes the drafted-token
-// probabilities.
+// tiles (and the sum the entropy needs, when the caller asks for the entropy). A small second
+// kernel merges the per-slice partials and computes the drafted-token probabilities.
 //
 // GEMM kernel layout (two CTAs on two SMs work as a pair on one 256 x 256 tile)
 //   M tile  = 256 rows = 4 sequence slots x 64 node slots, 128 rows per CTA of the pair
 //             (T <= 64; missing nodes are zero-filled by the TMA out-of-bounds rule)
-//   N tile  = up to 256 vocabulary entries, a multiple of 32; each CTA loads one half of it
+//   N tile  = 256 vocabulary entries, plus one narrower tile (a multiple of 32) for the rest of
+//             the CTA pair's vocabulary range; each CTA loads one half of a tile
 //   K block = 64 bf16 = one 128-byte swizzle row; 4 MMAs of K = 16 per block
 //   Per k-block a CTA stages its own 128 rows of H (16 KB) and half of the W tile (16 KB):
 //   32 KB for 128 x 256 x 64 multiply-adds per SM, against 48 KB when every SM works
