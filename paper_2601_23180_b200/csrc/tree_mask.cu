@@ -58,6 +58,83 @@ tree_mask_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask
   }
 }
 
+// Large batches (thousands of sequences): one THREAD per sequence. Parents precede children, so a
+// node's mask is its parent's mask plus its own bit, and one pass over the nodes in order does it:
+// about ten instructions per node for one thread, against a whole warp climbing level by level
+// above (which is the better shape for a decode batch, where sequences are few). A block takes 64
+// sequences: all 256 threads load their parents (16-byte loads) into shared memory, 64 threads walk,
+// all 256 threads write masks and depths back, coalesced.
+constexpr int kMaskBlockSeqs = 64, kMaskBlockThreads = 256;
+constexpr int kMaskParPitch = kMaskBlockSeqs + 4;   // bytes per node row of the parent table (bank spread)
+constexpr int kMaskRowPitch = kMaskBlockSeqs + 1;   // masks per node row
+
+__global__ void __launch_bounds__(kMaskBlockThreads)
+tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask, int32_t* __restrict__ depth,
+                       long long n_seq, int T) {
+  __shared__ signed char sPar[64 * kMaskParPitch];
+  __shared__ unsigned long long sMask[64 * kMaskRowPitch];
+  pdl_launch_dependents();
+  pdl_wait();
+  const long long s0 = static_cast<long long>(blockIdx.x) * kMaskBlockSeqs;
+  const int n_here = static_cast<int>(min(static_cast<long long>(kMaskBlockSeqs), n_seq - s0));
+  const int n_elem = n_here * T;
+  const int32_t* src = parent + s0 * T;
+  // parents -> shared memory as bytes ([node][sequence]); anything outside [-1, 62] becomes -2
+  auto put = [&](int e, int v) {
+    const int seq = e / T, node = e - seq * T;
+    sPar[node * kMaskParPitch + seq] = static_cast<signed char>((v >= -1 && v < 63) ? v : -2);
+  };
+  if ((n_elem & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    const int4* src4 = reinterpret_cast<const int4*>(src);
+#pragma unroll 2
+    for (int q = threadIdx.x; q < (n_elem >> 2); q += kMaskBlockThreads) {
+      const int4 v = __ldg(src4 + q);
+      put(4 * q, v.x); put(4 * q + 1, v.y); put(4 * q + 2, v.z); put(4 * q + 3, v.w);
+    }
+  } else {
+    for (int e = threadIdx.x; e < n_elem; e += kMaskBlockThreads) put(e, __ldg(src + e));
+  }
+  __syncthreads();
+  if (threadIdx.x < n_here) {
+    const int t = threadIdx.x;
+    for (int i = 0; i < T; ++i) {
+      const int par = sPar[i * kMaskParPitch + t];
+      unsigned long long m;
+      if (par == -1) {
+        m = 1ull << i;                                      // a root
+      } else if (par < 0 || par >= i) {
+        m = 0ull;                                           // malformed: flagged, not followed
+      } else {
+        const unsigned long long pm = sMask[par * kMaskRowPitch + t];
+        m = pm ? (pm | (1ull << i)) : 0ull;                 // a malformed ancestor spoils the walk
+      }
+      sMask[i * kMaskRowPitch + t] = m;
+    }
+  }
+  __syncthreads();
+  uint64_t* dst = mask + s0 * T;
+  int32_t* ddst = depth ? depth + s0 * T : nullptr;
+  auto get = [&](int e) -> unsigned long long {
+    const int seq = e / T, node = e - seq * T;
+    return sMask[node * kMaskRowPitch + seq];
+  };
+  if ((n_elem & 1) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0 &&
+      (!ddst || (reinterpret_cast<uintptr_t>(ddst) & 7u) == 0)) {
+#pragma unroll 2
+    for (int q = threadIdx.x; q < (n_elem >> 1); q += kMaskBlockThreads) {   // two masks = 16 bytes per store
+      const unsigned long long m0 = get(2 * q), m1 = get(2 * q + 1);
+      reinterpret_cast<ulonglong2*>(dst)[q] = make_ulonglong2(m0, m1);
+      if (ddst) reinterpret_cast<int2*>(ddst)[q] = make_int2(__popcll(m0) - 1, __popcll(m1) - 1);
+    }
+  } else {
+    for (int e = threadIdx.x; e < n_elem; e += kMaskBlockThreads) {
+      const unsigned long long m = get(e);
+      dst[e] = m;
+      if (ddst) ddst[e] = __popcll(m) - 1;
+    }
+  }
+}
+
 }  // namespace trispec
 
 extern "C" int trispec_build_tree_mask(const trispec_tree_args* a, void* stream) {
@@ -65,6 +142,13 @@ extern "C" int trispec_build_tree_mask(const trispec_tree_args* a, void* stream)
   if (!a || !a->parent || !a->mask || a->B <= 0 || a->T <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->T > 64) return TRISPEC_ERR_UNSUPPORTED;
   const long long n = a->B;
+  if (n >= 2048) {   // enough sequences to fill the chip with a thread each
+    unsigned grid = static_cast<unsigned>((n + kMaskBlockSeqs - 1) / kMaskBlockSeqs);
+    TRISPEC_CUDA_OK(launch_dependent(tree_mask_block_kernel, grid, kMaskBlockThreads, 0,
+                                     static_cast<cudaStream_t>(stream), 1, a->parent, a->mask, a->depth, n, a->T));
+    count_launch();
+    return TRISPEC_OK;
+  }
   const int per_block = (kMaskThreads / 32) * kMaskSeqPerWarp;
   unsigned grid = static_cast<unsigned>((n + per_block - 1) / per_block);
   TRISPEC_CUDA_OK(launch_dependent(tree_mask_kernel, grid, kMaskThreads, 0, static_cast<cudaStream_t>(stream), 1,

@@ -1,5 +1,6 @@
 """GPU parity of token pruning and KV commit against the oracle (bit-exact: integer and byte work),
 through the C ABI, plus a proxy round -> prune -> commit composition on one stream."""
+import dataclasses
 import math
 
 import numpy as np
@@ -348,3 +349,36 @@ def test_attention_of_pruned_trees(name, over, n_nodes):
             assert np.abs(o[b, :n] - ref_o[b, :n]).max() <= 2e-2, b
             assert np.abs(lse[b, :, :n] - ref_lse[b, :, :n]).max() <= 1e-3 * max(1.0, np.abs(ref_lse[b, :, :n]).max())
         assert np.isnan(o[b, n:]).all() and np.isnan(lse[b, :, n:]).all(), b
+
+
+def test_tree_mask_large_batch_matches_oracle():
+    """Batches of 2048 sequences and more take the thread-per-sequence mask kernel: bit-exact against the
+    oracle on the workload's trees, on a chain of 64 nodes, and with malformed parents flagged as in the
+    warp-per-sequence kernel (mask 0, depth -1, for the node and everything below it)."""
+    import tests.gpu_helpers as H
+    cfg = gen.CONFIGS["proxy_tree"]
+    distinct = np.stack([gen.make_tree(dataclasses.replace(cfg, seed=cfg.seed + s), 0) for s in range(300)])
+    ref_mask, ref_depth = orc.build_tree_mask(distinct)
+    B = 2048 + 37                                             # a ragged last block
+    idx = np.arange(B) % len(distinct)
+    parent = distinct[idx].copy()
+    bad_rows = [5, 64, 2000, B - 1]
+    for b in bad_rows:
+        parent[b, 7] = 9                                      # parent after the child
+    mask, depth = H.run_tree_mask(H.i32_dev(parent))
+    mask, depth = mask.cpu().numpy().view(np.uint64), depth.cpu().numpy()
+    good = np.ones(B, dtype=bool); good[bad_rows] = False
+    assert np.array_equal(mask[good], ref_mask[idx][good]) and np.array_equal(depth[good], ref_depth[idx][good])
+    for b in bad_rows:
+        below = [i for i in range(cfg.T) if (int(ref_mask[idx[b], i]) >> 7) & 1]   # node 7 and its descendants
+        assert len(below) >= 1
+        for i in range(cfg.T):
+            if i in below:
+                assert mask[b, i] == 0 and depth[b, i] == -1
+            else:
+                assert mask[b, i] == ref_mask[idx[b], i] and depth[b, i] == ref_depth[idx[b], i]
+    chain = np.tile(np.arange(-1, 63, dtype=np.int32), (2048, 1))
+    m, d = H.run_tree_mask(H.i32_dev(chain))
+    cm, cd = orc.build_tree_mask(chain[:1])
+    assert np.array_equal(m.cpu().numpy().view(np.uint64), np.tile(cm, (2048, 1)))
+    assert np.array_equal(d.cpu().numpy(), np.tile(cd, (2048, 1)))
