@@ -323,7 +323,7 @@ def run_only(args, cfg):
             "scan_with_compaction": {"kernel": "accept_scan_kernel + esc_compact_kernel (one block)", "ms": ms_both,
                                      "achieved": (scan_bytes + compact_bytes) / ms_both / 1e6, "unit": "GB/s",
                                      "frac": (scan_bytes + compact_bytes) / ms_both / 1e6 / hb},
-            "tree_mask_roofline": {"kernel": "tree_mask_kernel", "bound": "hbm", "achieved": mask_bytes / ms_mask / 1e6,
+            "tree_mask_roofline": {"kernel": "tree_mask_block_kernel", "bound": "hbm", "achieved": mask_bytes / ms_mask / 1e6,
                                    "peak": hb, "unit": "GB/s", "frac": mask_bytes / ms_mask / 1e6 / hb,
                                    "work_per_launch": mask_bytes, "ms_per_launch": ms_mask}})
         print(json.dumps(out), flush=True)
