@@ -382,3 +382,36 @@ def test_tree_mask_large_batch_matches_oracle():
     cm, cd = orc.build_tree_mask(chain[:1])
     assert np.array_equal(m.cpu().numpy().view(np.uint64), np.tile(cm, (2048, 1)))
     assert np.array_equal(d.cpu().numpy(), np.tile(cd, (2048, 1)))
+
+
+def test_host_pass_with_separately_allocated_host_buffers():
+    """The host-buffer entry point merges copies only where host and device addresses both follow each
+    other; with every host array in an allocation of its own it must fall back to one transfer per array
+    and give the same results as the device-resident pass."""
+    import torch
+    from paper_2601_23180_b200 import binding as ts
+    from paper_2601_23180_b200 import runner
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=3, L=300, V=6000, d=128, logit_scale=3.6 / (0.02 * math.sqrt(128)))
+    inp = gen.make_inputs(cfg)
+    pas = runner.VerifyPass(cfg, inp)
+    pas.run()
+    torch.cuda.synchronize()
+    want = {k: v.clone() for k, v in pas.scan_out.items()}
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    B, T = cfg.B, cfg.T
+    host = {"parent": pin(inp["parent"]), "tok": pin(inp["tok"])}
+    for k in ("h", "q", "k_tree", "v_tree"):
+        host[k] = pin(inp[k].view(np.int16))
+    for k in ("accept_len", "bonus_tok", "last_node"):
+        host[k] = torch.full((B,), -9, dtype=torch.int32).pin_memory()
+    host["path"] = torch.full((B, T), -9, dtype=torch.int32).pin_memory()
+    host["escalate"] = torch.full((B,), 7, dtype=torch.uint8).pin_memory()
+    for k in ("q", "k_tree", "v_tree", "h"):
+        pas.dev[k].zero_()                                   # the pass must bring them from the host
+    pas.dev["parent"].fill_(-1)
+    pas.dev["tok"].zero_()
+    ts.trispec_verify_host(ts.host_io(**host), pas.tree_args, pas.attn_args, pas.lm_args, pas.scan_args)
+    torch.cuda.synchronize()
+    assert int(pas.status.item()) == 0
+    for k in ("accept_len", "bonus_tok", "last_node", "path", "escalate"):
+        assert torch.equal(host[k], want[k].cpu()), k
