@@ -226,23 +226,28 @@ sample_gemm_kernel(const __grid_constant__ CUtensorMap tmap_hc, const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------
-// Few sequences (B <= 32): operands swapped. W is the M-side operand (128 vocabulary rows per
-// MMA), the compact rows are the N side (16 or 32 columns), so a pipeline stage is 16 KB of W
-// plus 2-4 KB of Hc and the ring (up to 11 stages) carries almost only W: enough bytes in
+// Few sequences (B <= 64): operands swapped. W is the M-side operand (128 vocabulary rows per
+// MMA), the compact rows are the N side (16, 32 or 64 columns), so a pipeline stage is 16 KB of W
+// plus 2-8 KB of Hc and the ring (9-12 stages) carries almost only W: enough bytes in
 // flight to keep HBM busy, which the 128 x 256 tile above cannot do with its 48 KB stages.
 // TMEM lane = vocabulary entry, column = sequence; each epilogue thread keeps a running best
-// per sequence in registers and the CTA reduces them at the end.
+// per sequence in registers and the CTA reduces them at the end. One group of four epilogue warps
+// serves 32 sequence columns (64 columns: two groups, 320 threads); the loader and the MMA issuer
+// are the two warps after the epilogue warps.
 // ---------------------------------------------------------------------------------------
-constexpr int SW_BM = 128, SW_BK = 64, SW_MAX_STAGES = 12, SW_MAX_SEQ = 32;
+constexpr int SW_BM = 128, SW_BK = 64, SW_MAX_STAGES = 12, SW_MAX_SEQ = 32;   // SW_MAX_SEQ: sequences per epilogue group
+constexpr int SW_MAX_GROUPS = 2, SW_MAX_THREADS = (4 * SW_MAX_GROUPS + 2) * 32, SW_TMEM_COLS = 128;
 constexpr int SW_A_BYTES = SW_BM * SW_BK * 2;           // 16 KB of W per stage
 
 struct SampleSwapParams {
   SampleParams base;
-  int N;            // sequence columns: 16 or 32
+  int N;            // sequence columns: 16, 32 or 64
+  int groups;       // epilogue warp groups: ceil(N / 32)
   int stages, stage_bytes;
 };
 
-__global__ void __launch_bounds__(SM_THREADS, 1)
+template <int kGroups>
+__global__ void __launch_bounds__((4 * kGroups + 2) * 32, 1)
 sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_hc,
                            const SampleSwapParams sp) {
   pdl_launch_dependents();
@@ -256,8 +261,9 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
   uint64_t* tmem_full = bars + 2 * SW_MAX_STAGES;
   uint64_t* tmem_empty = bars + 2 * SW_MAX_STAGES + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * SW_MAX_STAGES + 4);
-  float* red_y = reinterpret_cast<float*>(bars + 2 * SW_MAX_STAGES + 6);    // [4 warps][32 sequences]
-  int* red_i = reinterpret_cast<int*>(red_y + 4 * SW_MAX_SEQ);
+  float* red_y = reinterpret_cast<float*>(bars + 2 * SW_MAX_STAGES + 6);    // [epilogue warps][32 sequences]
+  int* red_i = reinterpret_cast<int*>(red_y + 4 * SW_MAX_GROUPS * SW_MAX_SEQ);
+  constexpr int loader_warp = 4 * kGroups, issuer_warp = loader_warp + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int range = blockIdx.x;
@@ -271,21 +277,21 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < sp.stages; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 4 * kGroups); }
     fence_mbar_init();
   }
-  if (warp == 5) {
-    tmem_alloc(tmem_slot, 64);                    // two accumulators of at most 32 columns
+  if (warp == issuer_warp) {
+    tmem_alloc(tmem_slot, SW_TMEM_COLS);          // two accumulators of at most 64 columns
     tmem_relinquish();
   }
-  if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_hc); prefetch_tmap(&tmap_w); }
+  if (warp == loader_warp && lane == 0) { prefetch_tmap(&tmap_hc); prefetch_tmap(&tmap_w); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();   // the compact rows come from the gather kernel
 
-  if (warp == 4) {
+  if (warp == loader_warp) {
     if (lane == 0) {   // ---------------------------------------------------------- TMA producer
       int stage = 0;
       uint32_t phase = 0;
@@ -301,7 +307,7 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == issuer_warp) {
     if (lane == 0) {   // ---------------------------------------------------------- MMA issuer
       int stage = 0;
       uint32_t phase = 0;
@@ -310,7 +316,7 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
         const int buf = t & 1;
         mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * 32);
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * 64);
         for (int kb = 0; kb < n_kb; ++kb) {
           mbar_wait(full_bar + stage, phase, p.dev_status);
           tc_fence_after();
@@ -326,11 +332,13 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 0-3)
-    const int row = warp * 32 + lane;             // TMEM lane = vocabulary entry of the tile
-    unsigned int live_mask = 0;                   // bit b: sequence b wants a sample
-    for (int b = 0; b < p.B; ++b)
-      if (__ldg(p.bonus_tok + b) == -2) live_mask |= 1u << b;
+    // ------------------------------------------------------------------ epilogue (4 warps per 32 sequences)
+    const int grp = warp >> 2, wq = warp & 3;     // sequence group, TMEM lane quarter
+    const int b0 = grp * SW_MAX_SEQ;              // first sequence of this group
+    const int row = wq * 32 + lane;               // TMEM lane = vocabulary entry of the tile
+    unsigned int live_mask = 0;                   // bit j: sequence b0 + j wants a sample
+    for (int j = 0; j < SW_MAX_SEQ && b0 + j < p.B; ++j)
+      if (__ldg(p.bonus_tok + b0 + j) == -2) live_mask |= 1u << j;
     float best[SW_MAX_SEQ];
     int best_idx[SW_MAX_SEQ];
 #pragma unroll
@@ -341,7 +349,7 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
       mbar_wait(tmem_full + buf, (t >> 1) & 1u, p.dev_status);
       tc_fence_after();
       uint32_t r[32];
-      tmem_ld32(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(buf * 32), r);
+      tmem_ld32(tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + static_cast<uint32_t>(buf * 64 + b0), r);
       tc_wait_ld();
       tc_fence_before();
       __syncwarp();
@@ -351,7 +359,7 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
 #pragma unroll
         for (int b = 0; b < SW_MAX_SEQ; ++b) {
           if ((live_mask >> b) & 1u) {
-            const uint4 w = philox4x32_10(make_uint4(static_cast<unsigned>(v >> 2), static_cast<unsigned>(b),
+            const uint4 w = philox4x32_10(make_uint4(static_cast<unsigned>(v >> 2), static_cast<unsigned>(b0 + b),
                                                      p.step_lo, p.step_hi), key);
             const unsigned int word = (v & 2) ? ((v & 1) ? w.w : w.z) : ((v & 1) ? w.y : w.x);
             const float y = fmaf(__uint_as_float(r[b]), p.scale, gumbel_from_word(word));
@@ -373,25 +381,25 @@ sample_gemm_swapped_kernel(const __grid_constant__ CUtensorMap tmap_w, const __g
       }
       if (lane == 0) { red_y[warp * SW_MAX_SEQ + b] = y; red_i[warp * SW_MAX_SEQ + b] = i; }
     }
-    asm volatile("bar.sync 2, 128;" ::: "memory");   // the four epilogue warps
-    if (warp == 0 && lane < p.B && ((live_mask >> lane) & 1u)) {
-      float y = red_y[lane];
-      int i = red_i[lane];
+    asm volatile("bar.sync 2, %0;" ::"n"(128 * kGroups) : "memory");   // all epilogue warps
+    if (wq == 0 && b0 + lane < p.B && ((live_mask >> lane) & 1u)) {
+      float y = red_y[warp * SW_MAX_SEQ + lane];
+      int i = red_i[warp * SW_MAX_SEQ + lane];
       for (int w2 = 1; w2 < 4; ++w2) {
-        const float oy = red_y[w2 * SW_MAX_SEQ + lane];
-        const int oi = red_i[w2 * SW_MAX_SEQ + lane];
+        const float oy = red_y[(warp + w2) * SW_MAX_SEQ + lane];
+        const int oi = red_i[(warp + w2) * SW_MAX_SEQ + lane];
         if (oi >= 0 && (i < 0 || oy > y || (oy == y && oi < i))) { y = oy; i = oi; }
       }
       SamplePartial out;
       out.y = y; out.idx = i;
-      p.partial[static_cast<size_t>(range) * (p.n_mt * SM_BM) + lane] = out;
+      p.partial[static_cast<size_t>(range) * (p.n_mt * SM_BM) + b0 + lane] = out;
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == issuer_warp) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 64);
+    tmem_dealloc(tmem_base, SW_TMEM_COLS);
   }
 }
 
@@ -482,15 +490,16 @@ extern "C" int trispec_sample_bonus(const trispec_sample_args* a, void* stream) 
   }
   TRISPEC_CUDA_OK(launch_dependent(sample_gather_kernel, static_cast<unsigned>(n_mt * SM_BM), 256, 0, st, 1, p));
   count_launch();
-  if (a->B <= SW_MAX_SEQ) {
+  if (a->B <= SW_MAX_SEQ * SW_MAX_GROUPS) {
     // few sequences: W on the M side, deep ring of small stages
     SampleSwapParams sp;
     sp.base = p;
-    sp.N = a->B <= 16 ? 16 : 32;
+    sp.N = a->B <= 16 ? 16 : (a->B <= 32 ? 32 : 64);
+    sp.groups = (sp.N + SW_MAX_SEQ - 1) / SW_MAX_SEQ;
     sp.stage_bytes = SW_A_BYTES + sp.N * SW_BK * 2;
     sp.stages = (224 * 1024) / sp.stage_bytes;
     if (sp.stages > SW_MAX_STAGES) sp.stages = SW_MAX_STAGES;
-    const int smem_bytes = sp.stages * sp.stage_bytes + 1024 + 2048;
+    const int smem_bytes = sp.stages * sp.stage_bytes + 1024 + 3072;
     CUtensorMap tm_w128, tm_hcn;
     {
       const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
@@ -504,10 +513,13 @@ extern "C" int trispec_sample_bonus(const trispec_sample_args* a, void* stream) 
       const uint32_t box[2] = {SW_BK, static_cast<uint32_t>(sp.N)};
       if (!cached_tmap_bf16(&tm_hcn, p.hc, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
     }
-    static bool smem_set_sw[64] = {};
-    rc = ensure_smem_limit(reinterpret_cast<const void*>(sample_gemm_swapped_kernel), 227 * 1024, smem_set_sw);
+    typedef void (*SwapKernel)(CUtensorMap, CUtensorMap, SampleSwapParams);
+    const SwapKernel kernel = sp.groups == 1 ? sample_gemm_swapped_kernel<1> : sample_gemm_swapped_kernel<2>;
+    static bool smem_set_sw[2][64] = {};
+    rc = ensure_smem_limit(reinterpret_cast<const void*>(kernel), 227 * 1024, smem_set_sw[sp.groups - 1]);
     if (rc != TRISPEC_OK) return rc;
-    TRISPEC_CUDA_OK(launch_dependent(sample_gemm_swapped_kernel, static_cast<unsigned>(n_ranges), SM_THREADS,
+    TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(n_ranges),
+                                     static_cast<unsigned>((4 * sp.groups + 2) * 32),
                                      static_cast<size_t>(smem_bytes), st, 1, tm_w128, tm_hcn, sp));
     count_launch();
   } else {
