@@ -72,10 +72,15 @@ struct LmParams {
 struct TileIter {
   int u0, units, n_tiles;
   __device__ TileIter(int V, int n_ranges, int r) {
+    // Every range gets V32 / n_ranges units of 32 columns. What is left over goes to the first ranges in
+    // chunks that cost as few extra tiles as possible: a tile costs a whole k-loop whatever its width, so
+    // a chunk first fills up a range's last, partial tile (no extra tile), and where the ranges consist of
+    // whole tiles it is a whole tile (few ranges run one tile longer, instead of many).
     const int V32 = (V + 31) >> 5;
-    u0 = static_cast<int>((static_cast<long long>(V32) * r) / n_ranges);
-    const int u1 = static_cast<int>((static_cast<long long>(V32) * (r + 1)) / n_ranges);
-    units = u1 - u0;
+    const int base = V32 / n_ranges, rem = V32 - base * n_ranges;
+    const int chunk = 8 - (base & 7);               // 1..8
+    u0 = r * base + min(rem, r * chunk);
+    units = base + min(chunk, max(0, rem - r * chunk));
     n_tiles = (units + 7) >> 3;
   }
   __device__ void tile(int t, int& n0, int& nw) const {

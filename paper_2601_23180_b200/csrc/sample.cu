@@ -236,7 +236,7 @@ sample_gemm_kernel(const __grid_constant__ CUtensorMap tmap_hc, const __grid_con
 // are the two warps after the epilogue warps.
 // ---------------------------------------------------------------------------------------
 constexpr int SW_BM = 128, SW_BK = 64, SW_MAX_STAGES = 12, SW_MAX_SEQ = 32;   // SW_MAX_SEQ: sequences per epilogue group
-constexpr int SW_MAX_GROUPS = 2, SW_MAX_THREADS = (4 * SW_MAX_GROUPS + 2) * 32, SW_TMEM_COLS = 128;
+constexpr int SW_MAX_GROUPS = 2, SW_TMEM_COLS = 128;
 constexpr int SW_A_BYTES = SW_BM * SW_BK * 2;           // 16 KB of W per stage
 
 struct SampleSwapParams {
