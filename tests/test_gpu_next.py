@@ -225,7 +225,10 @@ def _run_sample(dev, cfg, last_node, bonus_in, seed, step):
 
 @pytest.mark.parametrize("name,over", [("proxy_tree", dict(B=5, V=20011, d=256)),        # few sequences: W on the M side
                                        ("llama_tree", dict(B=19, V=128256 // 8, d=512)),  # 32 sequence columns
-                                       ("proxy_tree", dict(B=40, V=9000, d=128))])        # sequences on the M side
+                                       ("proxy_tree", dict(B=40, V=9000, d=128)),         # 64 sequence columns, two epilogue groups
+                                       ("proxy_tree", dict(B=33, V=5000, d=64)),          # one sequence in the second group
+                                       ("proxy_tree", dict(B=64, V=7000, d=128)),         # both groups full
+                                       ("proxy_tree", dict(B=70, V=6000, d=64))])         # sequences on the M side
 def test_bonus_sampling_matches_gumbel_max_oracle(name, over):
     """The sampled token is argmax_v (z_v + G_v) with the oracle's counter-based noise. fp32 logits
     can flip the arg-max only where the two best perturbed logits are closer than the LM-head
