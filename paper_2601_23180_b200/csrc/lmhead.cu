@@ -309,6 +309,7 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
 // ---------------------------------------------------------------------------------------
 struct LmFinalizeParams {
   int T, d, V, n_mt, n_ranges;
+  int stride;       // partial rows per vocabulary range
   float scale, c;
   const int32_t* seq_index;
   const LmPartial* partial;
@@ -389,7 +390,7 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
   if (!active) return;
 
   // ---- merge of the per-range partials: own row (all statistics) and parent row (max, sum)
-  const size_t stride = static_cast<size_t>(p.n_mt) * 2 * LM_BM;
+  const size_t stride = static_cast<size_t>(p.stride);
   const LmPartial* own = p.partial + static_cast<size_t>(a) * 64 + node;
   const LmPartial* parp = p.partial + static_cast<size_t>(a) * 64 + par;
   LmRowAcc ro = {-INFINITY, 0.f, 0.f}, rp = {-INFINITY, 0.f, 0.f};
@@ -451,11 +452,250 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// One sequence (batch-1 decoding, the paper's own setting): operands swapped. With at most 64
+// rows the GEMM is bound by streaming W, and the pair kernel above spends half of its ring
+// on H tiles. Here W is the M-side operand (128 vocabulary entries per MMA), the sequence's
+// rows are the N side (16-64 columns), one CTA per SM, and a stage is 16 KB of W plus 2-8 KB of
+// H: up to 12 stages, almost all of them W. TMEM lane = vocabulary entry, column = tree node.
+// Epilogue: per tile a warp reduces 32 columns at once over its 32 vocabulary entries with
+// transposing shuffle butterflies (top-2 with indices, then the sums of exponentials), after which
+// lane l holds column l's result and folds it into the running statistics it keeps for that column.
+// ---------------------------------------------------------------------------------------
+constexpr int LW_BM = 128, LW_BK = 64, LW_MAX_STAGES = 12, LW_THREADS = 192;
+constexpr int LW_A_BYTES = LW_BM * LW_BK * 2;           // 16 KB of W per stage
+constexpr int LW_ROWS = 64;                              // partial rows per vocabulary range
+
+struct LmRowsParams {
+  LmParams base;
+  int N;            // node columns: T rounded up to 16
+  int stages, stage_bytes;
+};
+
+struct LmColStats { float m, s, t, v1, v2; int i1, i2; };
+
+template <bool kEntropy>
+__global__ void __launch_bounds__(LW_THREADS, 1)
+lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
+                   const LmRowsParams sp) {
+  pdl_launch_dependents();
+  const LmParams& p = sp.base;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sp.stages * sp.stage_bytes);
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = bars + LW_MAX_STAGES;
+  uint64_t* tmem_full = bars + 2 * LW_MAX_STAGES;
+  uint64_t* tmem_empty = bars + 2 * LW_MAX_STAGES + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LW_MAX_STAGES + 4);
+  LmColStats* red = reinterpret_cast<LmColStats*>(bars + 2 * LW_MAX_STAGES + 6);   // [4 warps][64 columns]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int range = blockIdx.x;
+  const int V16 = (p.V + 15) >> 4;
+  const int u0 = static_cast<int>((static_cast<long long>(V16) * range) / p.n_ranges);
+  const int u1 = static_cast<int>((static_cast<long long>(V16) * (range + 1)) / p.n_ranges);
+  const int v_begin = u0 << 4, v_end = min(u1 << 4, p.V);
+  const int n_tiles = (v_end - v_begin + LW_BM - 1) / LW_BM;
+  const int n_kb = p.d / LW_BK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < sp.stages; ++i) { mbar_init(full_bar + i, 1); mbar_init(empty_bar + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tmem_full + i, 1); mbar_init(tmem_empty + i, 4); }
+    fence_mbar_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, 128);                   // two accumulators of at most 64 columns
+    tmem_relinquish();
+  }
+  if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_h); prefetch_tmap(&tmap_w); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 4) {
+    if (lane == 0) {   // ---------------------------------------------------------- TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t tx = static_cast<uint32_t>(LW_A_BYTES + sp.N * LW_BK * 2);
+      const int seq = p.seq_index ? __ldg(p.seq_index) : 0;     // the one active sequence
+      for (int t = 0; t < n_tiles; ++t) {
+        for (int kb = 0; kb < n_kb; ++kb) {
+          mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
+          uint8_t* sa = smem + stage * sp.stage_bytes;
+          mbar_expect_tx(full_bar + stage, tx);
+          tma_load_2d(sa, &tmap_w, full_bar + stage, kb * LW_BK, v_begin + t * LW_BM);   // rows past V: zero fill
+          tma_load_3d(sa + LW_A_BYTES, &tmap_h, full_bar + stage, kb * LW_BK, 0, seq);     // nodes past T: zero fill
+          if (++stage == sp.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {   // ---------------------------------------------------------- MMA issuer
+      int stage = 0;
+      uint32_t phase = 0;
+      const uint32_t idesc = idesc_bf16(LW_BM, sp.N, false, false);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int buf = t & 1;
+        mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * 64);
+        for (int kb = 0; kb < n_kb; ++kb) {
+          mbar_wait(full_bar + stage, phase, p.dev_status);
+          tc_fence_after();
+          const uint32_t sa = base_u32 + stage * sp.stage_bytes;
+          const uint64_t adesc = smem_desc_sw128(sa, 1024, 16);
+          const uint64_t bdesc = smem_desc_sw128(sa + LW_A_BYTES, 1024, 16);
+#pragma unroll
+          for (int k = 0; k < LW_BK / 16; ++k) tc_mma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
+          tc_commit(empty_bar + stage);
+          if (++stage == sp.stages) { stage = 0; phase ^= 1u; }
+        }
+        tc_commit(tmem_full + buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 0-3)
+    // this lane keeps the running statistics of columns `lane` and `lane + 32`
+    LmColStats run[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      run[h].m = -INFINITY; run[h].s = 0.f; run[h].t = 0.f;
+      run[h].v1 = -INFINITY; run[h].v2 = -INFINITY; run[h].i1 = -1; run[h].i2 = -1;
+    }
+    const float c = p.c;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      mbar_wait(tmem_full + buf, (t >> 1) & 1u, p.dev_status);
+      tc_fence_after();
+      const int v_lane0 = v_begin + t * LW_BM + warp * 32;    // vocabulary entry of lane 0
+      const bool valid = v_lane0 + lane < v_end;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h * 32 >= sp.N) break;
+        uint32_t r[32];
+        tmem_ld32(tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(buf * 64 + h * 32), r);
+        tc_wait_ld();
+        if (h * 32 + 32 >= sp.N) {                // last chunk read: the accumulator may be overwritten
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tmem_empty + buf);
+        }
+        // Per column: top-2 (value, vocabulary index) and the sum of exponentials over this warp's 32
+        // vocabulary entries. A transposing butterfly does all 32 columns at once: in the step with
+        // distance o a lane keeps half of the columns it still holds, hands the other half to its
+        // partner and merges what it receives, so that after five steps lane l holds column l.
+        const int my_v = v_lane0 + lane;
+        float v1[32], v2[32];
+        int i1[32], i2[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const bool on = valid && (h * 32 + j < sp.N);
+          v1[j] = on ? __uint_as_float(r[j]) : -INFINITY;
+          i1[j] = on ? my_v : -1;
+          v2[j] = -INFINITY;
+          i2[j] = -1;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const bool up = (lane & o) != 0;
+#pragma unroll
+          for (int i = 0; i < o; ++i) {
+            const float sv1 = up ? v1[i] : v1[i + o], sv2 = up ? v2[i] : v2[i + o];
+            const int si1 = up ? i1[i] : i1[i + o], si2 = up ? i2[i] : i2[i + o];
+            float kv1 = up ? v1[i + o] : v1[i], kv2 = up ? v2[i + o] : v2[i];
+            int ki1 = up ? i1[i + o] : i1[i], ki2 = up ? i2[i + o] : i2[i];
+            const float rv1 = __shfl_xor_sync(0xffffffffu, sv1, o), rv2 = __shfl_xor_sync(0xffffffffu, sv2, o);
+            const int ri1 = __shfl_xor_sync(0xffffffffu, si1, o), ri2 = __shfl_xor_sync(0xffffffffu, si2, o);
+            lm_top2_insert(rv1, ri1, kv1, ki1, kv2, ki2);
+            lm_top2_insert(rv2, ri2, kv1, ki1, kv2, ki2);
+            v1[i] = kv1; v2[i] = kv2; i1[i] = ki1; i2[i] = ki2;
+          }
+        }
+        const float m_t = v1[0];                  // this lane's column: h * 32 + lane
+        // every lane needs every column's maximum for its exponentials
+        float es[32], et[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float mj = __shfl_sync(0xffffffffu, m_t, j);
+          const bool on = valid && (h * 32 + j < sp.N);
+          const float z = __uint_as_float(r[j]);
+          es[j] = on ? ex2f((z - mj) * c) : 0.f;
+          et[j] = (kEntropy && on) ? es[j] * z : 0.f;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const bool up = (lane & o) != 0;
+#pragma unroll
+          for (int i = 0; i < o; ++i) {
+            const float ss = up ? es[i] : es[i + o], ks = up ? es[i + o] : es[i];
+            es[i] = ks + __shfl_xor_sync(0xffffffffu, ss, o);
+            if (kEntropy) {
+              const float st2 = up ? et[i] : et[i + o], kt = up ? et[i + o] : et[i];
+              et[i] = kt + __shfl_xor_sync(0xffffffffu, st2, o);
+            }
+          }
+        }
+        // fold the tile's statistics of column h * 32 + lane into the running ones
+        {
+          LmRowAcc a = {run[h].m, run[h].s, run[h].t};
+          lm_fold(a, m_t, es[0], et[0], c);
+          run[h].m = a.m; run[h].s = a.s; run[h].t = a.t;
+          lm_top2_insert(v1[0], i1[0], run[h].v1, run[h].i1, run[h].v2, run[h].i2);
+          lm_top2_insert(v2[0], i2[0], run[h].v1, run[h].i1, run[h].v2, run[h].i2);
+        }
+      }
+    }
+    // the four warps covered different vocabulary entries of every tile: merge through shared memory
+    red[warp * 64 + lane] = run[0];
+    red[warp * 64 + 32 + lane] = run[1];
+    asm volatile("bar.sync 2, 128;" ::: "memory");   // the four epilogue warps
+    if (warp == 0) {
+      pdl_wait();   // the partials of the previous pass may still be read until earlier kernels are done
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int col = h * 32 + lane;
+        if (col >= p.T) continue;
+        LmColStats q = red[col];
+        LmRowAcc a = {q.m, q.s, q.t};
+        for (int w2 = 1; w2 < 4; ++w2) {
+          const LmColStats o2 = red[w2 * 64 + col];
+          lm_fold(a, o2.m, o2.s, o2.t, c);
+          lm_top2_insert(o2.v1, o2.i1, q.v1, q.i1, q.v2, q.i2);
+          lm_top2_insert(o2.v2, o2.i2, q.v1, q.i1, q.v2, q.i2);
+        }
+        LmPartial out;
+        out.m = a.m; out.s = a.s; out.v1 = q.v1; out.v2 = q.v2; out.i1 = q.i1; out.i2 = q.i2; out.t = a.t; out.pad = 0;
+        p.partial[static_cast<size_t>(range) * LW_ROWS + col] = out;
+      }
+    }
+  }
+  pdl_wait();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 128);
+  }
+}
+
+// One active sequence takes the W-on-M kernel (lmhead_rows_kernel): one CTA and one vocabulary range
+// per SM, LW_ROWS partial rows per range.
+static bool lm_rows_path(int n_seq) { return n_seq == 1; }
+
 static int lm_plan(const trispec_lmhead_args* a, int* n_seq, int* n_mt, int* n_ranges) {
   if (!a || a->B <= 0 || a->T <= 0 || a->d <= 0 || a->V <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->T > 64 || (a->d % LM_BK) != 0 || a->V < 2) return TRISPEC_ERR_UNSUPPORTED;
   *n_seq = a->seq_index ? a->B_active : a->B;
   if (*n_seq <= 0 || *n_seq > a->B) return TRISPEC_ERR_INVALID_ARG;
+  if (lm_rows_path(*n_seq)) {
+    *n_mt = 1;
+    const int V16 = (a->V + 15) / 16;
+    *n_ranges = device_sm_count() < V16 ? device_sm_count() : V16;
+    return TRISPEC_OK;
+  }
   *n_mt = (*n_seq + 3) / 4;
   const int pairs = device_sm_count() / 2;       // one CTA pair per two SMs
   int r = pairs / *n_mt;
@@ -472,6 +712,7 @@ extern "C" size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a) {
   using namespace trispec;
   int n_seq, n_mt, n_ranges;
   if (lm_plan(a, &n_seq, &n_mt, &n_ranges) != TRISPEC_OK) return 0;
+  if (lm_rows_path(n_seq)) return static_cast<size_t>(n_ranges) * LW_ROWS * sizeof(LmPartial);
   return static_cast<size_t>(n_ranges) * n_mt * 2 * LM_BM * sizeof(LmPartial);
 }
 
@@ -506,6 +747,55 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   }
   // the entropy sum costs two more instructions per logit: only computed when it is asked for
   const bool want_entropy = a->out.entropy != nullptr;
+  LmFinalizeParams f;
+  f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges;
+  f.scale = a->logit_scale; f.c = a->logit_scale * kLog2e;
+  f.seq_index = a->seq_index;
+  f.partial = static_cast<LmPartial*>(a->workspace);
+  f.h = static_cast<const uint16_t*>(a->h);
+  f.W = static_cast<const uint16_t*>(a->W);
+  f.parent = a->parent; f.tok = a->tok;
+  f.out = a->out;
+  if (lm_rows_path(n_seq)) {
+    LmRowsParams sp;
+    sp.base.T = a->T; sp.base.d = a->d; sp.base.V = a->V;
+    sp.base.n_seq = 1; sp.base.n_mt = 1; sp.base.n_ranges = n_ranges;
+    sp.base.c = f.c;
+    sp.base.seq_index = a->seq_index;
+    sp.base.partial = static_cast<LmPartial*>(a->workspace);
+    sp.base.dev_status = a->dev_status;
+    sp.N = ((a->T + 15) / 16) * 16;
+    sp.stage_bytes = LW_A_BYTES + sp.N * LW_BK * 2;
+    sp.stages = (216 * 1024) / sp.stage_bytes;
+    if (sp.stages > LW_MAX_STAGES) sp.stages = LW_MAX_STAGES;
+    const int smem_bytes = sp.stages * sp.stage_bytes + 1024 + 8192;
+    CUtensorMap tm_w128, tm_hn;
+    {
+      const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
+      const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
+      const uint32_t box[2] = {LW_BK, LW_BM};
+      if (!cached_tmap_bf16(&tm_w128, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+    }
+    {
+      const uint64_t dims[3] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->T), static_cast<uint64_t>(a->B)};
+      const uint64_t strides[2] = {static_cast<uint64_t>(a->d) * 2, static_cast<uint64_t>(a->d) * 2 * a->T};
+      const uint32_t box[3] = {LW_BK, static_cast<uint32_t>(sp.N), 1};
+      if (!cached_tmap_bf16(&tm_hn, a->h, 3, dims, strides, box)) return TRISPEC_ERR_CUDA;
+    }
+    typedef void (*RowsKernel)(CUtensorMap, CUtensorMap, LmRowsParams);
+    const RowsKernel kernel = want_entropy ? lmhead_rows_kernel<true> : lmhead_rows_kernel<false>;
+    static bool smem_set_rows[2][64] = {};
+    rc = ensure_smem_limit(reinterpret_cast<const void*>(kernel), 227 * 1024, smem_set_rows[want_entropy ? 1 : 0]);
+    if (rc != TRISPEC_OK) return rc;
+    TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(n_ranges), LW_THREADS,
+                                     static_cast<size_t>(smem_bytes), st, 1, tm_w128, tm_hn, sp));
+    count_launch();
+    f.stride = LW_ROWS;
+    TRISPEC_CUDA_OK(launch_dependent(lmhead_finalize_kernel, static_cast<unsigned>((a->T + 7) / 8),
+                                     LM_FIN_THREADS, 0, st, 1, f, 1));
+    count_launch();
+    return TRISPEC_OK;
+  }
   static bool smem_set[2][64] = {};
   rc = want_entropy
            ? ensure_smem_limit(reinterpret_cast<const void*>(lmhead_gemm_kernel<true>), LM_SMEM_BYTES, smem_set[1])
@@ -527,15 +817,7 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   }
   count_launch();
 
-  LmFinalizeParams f;
-  f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges;
-  f.scale = a->logit_scale; f.c = p.c;
-  f.seq_index = a->seq_index;
-  f.partial = p.partial;
-  f.h = static_cast<const uint16_t*>(a->h);
-  f.W = static_cast<const uint16_t*>(a->W);
-  f.parent = a->parent; f.tok = a->tok;
-  f.out = a->out;
+  f.stride = n_mt * 2 * LM_BM;
   TRISPEC_CUDA_OK(launch_dependent(lmhead_finalize_kernel, static_cast<unsigned>((n_seq * a->T + 7) / 8),
                                    LM_FIN_THREADS, 0, st, 1, f, n_seq));
   count_launch();
