@@ -131,6 +131,12 @@ LM_CASES = [
     ("proxy_tree", dict(B=5, V=151936 // 8, d=192, logit_scale=3.6 / (0.02 * math.sqrt(192)))),
     ("target_escalated", dict(B=7, n_active=3, V=9000, d=320, logit_scale=3.6 / (0.02 * math.sqrt(320)))),
     ("llama_tree", dict(B=2, V=128256 // 4, d=1024, logit_scale=3.6 / (0.02 * 32.0))),
+    # one active sequence: the kernel with W on the M side and the tree's nodes as columns
+    ("proxy_tree", dict(B=1, V=40011, d=512)),                                   # 61 nodes: two column chunks
+    ("llama_tree", dict(B=1, V=9000, d=256)),                                    # 49 nodes
+    ("target_escalated", dict(B=4, n_active=1, V=7000, d=320)),                  # the one sequence is picked by seq_index
+    ("tiny_chain", dict(k=15, V=3000, d=128)),                                   # 16 nodes: exactly one 16-column block
+    ("tiny_chain", dict(k=31, V=200, d=64)),                                     # 32 nodes, fewer vocabulary units than SMs
 ]
 
 
