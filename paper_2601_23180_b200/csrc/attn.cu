@@ -710,6 +710,19 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   }
   pl->n_splits = best_s;
   pl->cluster = pl->n_splits <= 8;
+  // Clusters do not reach every CTA slot (measured: 142 of the 148 SMs take clusters of 3 or 4, 284 slots), and
+  // a grid a little larger than that runs as two waves. When plain CTAs would fill the chip in ONE wave
+  // (at least 92 % of all slots, long enough tile loops), that wave plus the small merge kernel is faster than
+  // the clustered choice: target_escalated (96 items x 3 splits = 288 CTAs) 148 -> 118 us.
+  {
+    const long long cluster_slots = slots * 96 / 100;
+    const int sp_full = fixed > 0 ? static_cast<int>(slots / fixed) : 0;
+    if (pl->cluster && fixed * best_s > cluster_slots && sp_full >= 2 && fixed * sp_full * 100 >= slots * 92 &&
+        tiles / sp_full >= 16) {
+      pl->n_splits = sp_full;
+      pl->cluster = false;
+    }
+  }
   pl->items = static_cast<size_t>(fixed) * pl->n_splits;
   if (pl->items > 0x7fffffffull) return TRISPEC_ERR_UNSUPPORTED;
   return TRISPEC_OK;
