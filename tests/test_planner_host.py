@@ -1,0 +1,51 @@
+"""Host-side planning that can be observed without a GPU: the workspace queries.
+
+`trispec_verify_attn_workspace` returns 0 when the KV splits of a sequence are merged inside a thread-block
+cluster, and the size of the fp32 partials when plain CTAs and the merge kernel are used instead;
+`trispec_lmhead_stats_workspace` shows which LM-head kernel a call takes. Without a device the planners
+assume 148 SMs."""
+from paper_2601_23180_b200 import binding as ts
+from paper_2601_23180_b200 import inputs as gen
+
+
+def _attn_args(cfg, n_active=None):
+    a = ts.AttnArgs()
+    a.B, a.T, a.Hq, a.Hkv, a.D, a.scale = cfg.B, cfg.T, cfg.Hq, cfg.Hkv, cfg.D, 1.0
+    a.kv_layout, a.Lmax = ts.KV_CONTIGUOUS, cfg.L
+    a.B_active = 0 if n_active is None else n_active
+    a.seq_index = None if n_active is None else 1     # any non-null value: only its presence is looked at
+    return a
+
+
+def test_attention_workspace_follows_the_split_plan():
+    # proxy_tree: 64 (sequence, KV head) items x 4 splits in clusters: merged on chip, no workspace
+    assert ts.trispec_verify_attn_workspace(_attn_args(gen.CONFIGS["proxy_tree"])) == 0
+    # llama_tree: 256 items, no split
+    assert ts.trispec_verify_attn_workspace(_attn_args(gen.CONFIGS["llama_tree"])) == 0
+    # target_escalated: 3 active sequences x 8 KV heads x 4 M tiles = 96 items; 4 clustered splits would be 384
+    # CTAs (two waves), 3 plain splits are 288 CTAs (one wave of the 296 slots): partials go to the workspace
+    cfg = gen.CONFIGS["target_escalated"]
+    ws = ts.trispec_verify_attn_workspace(_attn_args(cfg, n_active=3))
+    assert ws == 96 * 3 * 128 * (128 + 2) * 4
+    # one sequence with a very long context: more than 8 splits, workspace as well
+    long1 = gen.small_variant(gen.CONFIGS["proxy_tree"], B=1, L=65536, Hq=4, Hkv=2)
+    assert ts.trispec_verify_attn_workspace(_attn_args(long1)) > 0
+
+
+def test_lmhead_workspace_shows_the_kernel_choice():
+    def args(B, T, d, V, n_active=None):
+        a = ts.LmheadArgs()
+        a.B, a.T, a.d, a.V, a.logit_scale = B, T, d, V, 1.0
+        a.B_active = 0 if n_active is None else n_active
+        a.seq_index = None if n_active is None else 1
+        return a
+    # batches: CTA pairs, 74 // n_mt vocabulary ranges x n_mt M tiles x 256 rows x 32 bytes
+    assert ts.trispec_lmhead_stats_workspace(args(8, 61, 2048, 151936)) == 37 * 2 * 256 * 32
+    assert ts.trispec_lmhead_stats_workspace(args(64, 61, 2048, 151936)) == 4 * 16 * 256 * 32
+    # one active sequence: one range per SM x 64 rows x 32 bytes
+    assert ts.trispec_lmhead_stats_workspace(args(1, 9, 2048, 32000)) == 148 * 64 * 32
+    assert ts.trispec_lmhead_stats_workspace(args(8, 61, 5120, 151936, n_active=1)) == 148 * 64 * 32
+    # fewer 16-row vocabulary units than SMs
+    assert ts.trispec_lmhead_stats_workspace(args(1, 9, 64, 200)) == 13 * 64 * 32
+    # unsupported shapes plan nothing
+    assert ts.trispec_lmhead_stats_workspace(args(1, 65, 2048, 32000)) == 0
