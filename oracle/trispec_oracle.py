@@ -19,6 +19,12 @@ What each function follows:
                    the "standard left-to-right acceptance rule" applied after Eq. 10.
   prune_tree       token pruning of routing case (ii) ("prune these tokens from the draft tree
                    and pass the remaining branches to the target"; ablation on token pruning).
+  accept_scan_token_specific
+                   the token-specific deferral rule of the SpecCascade baselines (appendix
+                   "Baseline Implementation Details: SpecCascade") as an acceptance rule.
+  accept_scan_stochastic, sample_bonus
+                   Eq. 6 at temperature 1 and the bonus draw of Algorithm 1 (Gumbel-max with
+                   counter-based Philox noise).
   commit_kv        X <- X + Y of Algorithm 1 as the KV cache sees it: the keys/values of the
                    last committed token and of the accepted draft tokens are appended.
 
@@ -382,22 +388,27 @@ def commit_kv(k_cache: np.ndarray, v_cache: np.ndarray, ctx_len: np.ndarray, k_t
 def accept_scan_stochastic(p_top1: np.ndarray, p_top2: np.ndarray, p_draft: np.ndarray,
                            q_draft: np.ndarray, u: np.ndarray, parent: np.ndarray, tok: np.ndarray,
                            lam: float, mode: int = MODE_PROXY, active: Optional[np.ndarray] = None,
-                           near_eps: float = 1e-3) -> Dict[str, np.ndarray]:
+                           near_eps: float = 1e-3, near_accept_eps: float = 1e-6) -> Dict[str, np.ndarray]:
     """The walk of accept_scan with the Bernoulli acceptance of Eq. 6 in place of the arg-max
     match: a drafted child c is accepted iff u[c] < min(1, p_draft[c] / q_draft[c]), where
     p_draft[c] is the verifier's probability of tok[c] at c's parent, q_draft[c] the drafter's,
-    and u[c] a uniform number in [0, 1) supplied by the caller.
+    and u[c] a uniform number in [0, 1) supplied by the caller. The decision is taken in fp64
+    whatever the precision of the arrays; a drafter probability of 0 counts as ratio 1.
     Readings: the paper states the rule for a chain; on a tree the children of the current node
     are tried in node order and the first accepted one is taken. When no child is accepted the
     round ends in case (i) and the bonus token has to be SAMPLED from the current node's
     distribution (Algorithm 1), which this function cannot do from statistics: it returns
     bonus_tok = -2 for "sample at last_node". The margin test precedes the children as in
-    accept_scan. Outputs as accept_scan (without the escalation list)."""
+    accept_scan. Outputs as accept_scan (without the escalation list), plus near_accept [B]: the
+    number of children tested along the walk whose uniform number lies within near_accept_eps of
+    the acceptance ratio (a decision that an implementation dividing in lower precision may
+    take the other way; such sequences are counted, not compared)."""
     parent = np.asarray(parent)
     B, T = parent.shape
     res = {"accept_len": np.zeros(B, dtype=np.int32), "escalate": np.zeros(B, dtype=np.uint8),
            "bonus_tok": np.full(B, -1, dtype=np.int32), "path": np.full((B, T), -1, dtype=np.int32),
-           "last_node": np.full(B, -1, dtype=np.int32), "near_thr": np.zeros(B, dtype=np.int32)}
+           "last_node": np.full(B, -1, dtype=np.int32), "near_thr": np.zeros(B, dtype=np.int32),
+           "near_accept": np.zeros(B, dtype=np.int32)}
     for b in range(B):
         if active is not None and not active[b]:
             continue
@@ -414,14 +425,76 @@ def accept_scan_stochastic(p_top1: np.ndarray, p_top2: np.ndarray, p_draft: np.n
             for c in range(cur + 1, T):
                 if int(parent[b, c]) != cur:
                     continue
-                # in the arrays' own precision (fp32 inputs give the fp32 decision the kernel takes)
-                one = p_draft.dtype.type(1)
-                ratio = min(one, p_draft[b, c] / q_draft[b, c]) if q_draft[b, c] > 0 else one
-                if u[b, c] < ratio:
+                qc = float(q_draft[b, c])
+                ratio = min(1.0, float(p_draft[b, c]) / qc) if qc > 0.0 else 1.0
+                if abs(float(u[b, c]) - ratio) < near_accept_eps:
+                    res["near_accept"][b] += 1
+                if float(u[b, c]) < ratio:
                     nxt = c
                     break
             if nxt < 0:
                 res["bonus_tok"][b] = -2
+                break
+            res["path"][b, n] = nxt
+            n += 1
+            cur = nxt
+        res["accept_len"][b] = n
+        res["last_node"][b] = cur
+    return res
+
+
+# ----------------------------------------------------------------------------------------
+# token-specific deferral rule (appendix "Baseline Implementation Details: SpecCascade")
+# ----------------------------------------------------------------------------------------
+def accept_scan_token_specific(p_top1: np.ndarray, p_top2: np.ndarray, top1_idx: np.ndarray,
+                               p_draft: np.ndarray, parent: np.ndarray, tok: np.ndarray, lam: float,
+                               alpha: float, mode: int = MODE_PROXY, active: Optional[np.ndarray] = None,
+                               near_eps: float = 1e-3, near_accept_eps: float = 1e-6) -> Dict[str, np.ndarray]:
+    """The walk of accept_scan with the token-specific deferral rule in place of the arg-max
+    match: the rule compares the verifier's probability of the candidate token with the
+    verifier's maximum probability and never looks at the drafter's distribution. A drafted
+    child c of the current node is accepted iff
+        p_draft[c] >= (1 - alpha) * p_top1[current node],
+    p_draft[c] being the verifier's probability of tok[c] at c's parent (the paper runs the rule
+    with alpha = 0.2). alpha = 0 accepts only a token as probable as the arg-max (greedy
+    acceptance); alpha = 1 accepts any drafted token.
+    Readings: on a tree the children of the current node are tried in node order and the first
+    that passes is taken (as for duplicate siblings and for the stochastic rule); when none
+    passes the round ends in case (i) with the verifier's arg-max token as the bonus token, as in
+    greedy acceptance. In PROXY mode the margin test of Eq. 8 precedes the children as in
+    accept_scan. The comparison is made in fp64; near_accept [B] counts the tested children with
+    |p_draft - (1 - alpha) p_top1| < near_accept_eps. Outputs as accept_scan, without the
+    escalation list."""
+    parent = np.asarray(parent)
+    B, T = parent.shape
+    res = {"accept_len": np.zeros(B, dtype=np.int32), "escalate": np.zeros(B, dtype=np.uint8),
+           "bonus_tok": np.full(B, -1, dtype=np.int32), "path": np.full((B, T), -1, dtype=np.int32),
+           "last_node": np.full(B, -1, dtype=np.int32), "near_thr": np.zeros(B, dtype=np.int32),
+           "near_accept": np.zeros(B, dtype=np.int32)}
+    for b in range(B):
+        if active is not None and not active[b]:
+            continue
+        cur, n = 0, 0
+        while True:
+            if mode == MODE_PROXY:
+                margin = float(p_top1[b, cur]) - float(p_top2[b, cur])
+                if abs(margin - lam) < near_eps:
+                    res["near_thr"][b] += 1
+                if not (margin >= lam):
+                    res["escalate"][b] = 1
+                    break
+            bar = (1.0 - float(alpha)) * float(p_top1[b, cur])
+            nxt = -1
+            for c in range(cur + 1, T):
+                if int(parent[b, c]) != cur:
+                    continue
+                if abs(float(p_draft[b, c]) - bar) < near_accept_eps:
+                    res["near_accept"][b] += 1
+                if float(p_draft[b, c]) >= bar:
+                    nxt = c
+                    break
+            if nxt < 0:
+                res["bonus_tok"][b] = int(top1_idx[b, cur])
                 break
             res["path"][b, n] = nxt
             n += 1
@@ -452,15 +525,23 @@ def philox4x32_10(counter: Sequence[int], key: Sequence[int]) -> Tuple[int, int,
     return c0, c1, c2, c3
 
 
+def gumbel_from_word(w: int) -> float:
+    """Standard Gumbel variate from one 32-bit word of the generator: the word's upper 23 bits
+    give u = ((w >> 9) + 0.5) / 2^23, a point strictly inside (0, 1) that a single-precision
+    float holds exactly, and G = -ln(-ln u). Dropping the lower 9 bits bounds the variate:
+    G lies in [-ln(-ln(2^-24)), -ln(-ln(1 - 2^-24))] = [-2.812, 16.636], so an entry more than
+    19.45 below the largest logit can never be drawn (its probability is below 4e-9)."""
+    uu = ((int(w) >> 9) + 0.5) / 8388608.0
+    return float(-np.log(-np.log(uu)))
+
+
 def gumbel_noise(seed: int, step: int, b: int, v: int) -> float:
     """Standard Gumbel variate of vocabulary entry v of sequence b in round `step`:
-    word (v mod 4) of philox4x32_10(counter = (v div 4, b, step low, step high), key = seed) is
-    turned into u = ((word >> 9) + 0.5) / 2^23, which lies strictly inside (0, 1) and is exact in
-    fp32 as well, and G = -ln(-ln u)."""
+    word (v mod 4) of philox4x32_10(counter = (v div 4, b, step low, step high), key = seed),
+    turned into a variate by gumbel_from_word."""
     w = philox4x32_10((v >> 2, b, step & 0xFFFFFFFF, (step >> 32) & 0xFFFFFFFF),
                       (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))[v & 3]
-    uu = ((w >> 9) + 0.5) / 8388608.0
-    return -np.log(-np.log(uu))
+    return gumbel_from_word(w)
 
 
 def gumbel_noise_row(seed: int, step: int, b: int, V: int) -> np.ndarray:

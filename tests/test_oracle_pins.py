@@ -451,3 +451,45 @@ def test_verify_end_to_end_small():
         else:
             assert np.isnan(out["o"][b]).all() and out["scan"]["last_node"][b] == -1
     assert out["scan"]["escalate"].sum() == 0     # TARGET mode never escalates
+
+
+def test_verify_hands_the_four_steps_the_right_arrays():
+    """The whole-pass function against its four steps called by hand on a batch where only a
+    subset of the sequences is verified (seq_index): the subset must reach the attention and the
+    LM head as `seqs`, the scan as the `active` flags, and the scan must read the statistics the
+    LM head produced; a sequence outside the subset yields NaN / -1 everywhere."""
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=5, n_active=3, k=12, max_depth=4, L=70, V=300, d=64,
+                            Hq=4, Hkv=2, rho=0.3, logit_scale=3.6 / (0.02 * 8.0), seed=21)
+    inp = gen.make_inputs(cfg)
+    seqs = [int(s) for s in inp["seq_index"]]
+    assert 0 < len(seqs) < cfg.B
+    scale = 1.0 / math.sqrt(cfg.D)
+    out = orc.verify(inp, scale, cfg.logit_scale, cfg.lam, mode=orc.MODE_PROXY)
+    mask, depth = orc.build_tree_mask(inp["parent"])
+    assert np.array_equal(out["mask"], mask) and np.array_equal(out["depth"], depth)
+    o, lse = orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], mask, inp["k_cache"], inp["v_cache"],
+                             inp["ctx_len"], scale, seqs=seqs)
+    assert np.array_equal(out["o"], o, equal_nan=True) and np.array_equal(out["attn_lse"], lse, equal_nan=True)
+    st = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale, seqs=seqs)
+    for k in st:
+        assert np.array_equal(out["stats"][k], st[k], equal_nan=True), k
+    active = np.zeros(cfg.B, dtype=np.uint8)
+    active[seqs] = 1
+    sc = orc.accept_scan(st["p_top1"], st["p_top2"], st["top1_idx"], inp["parent"], inp["tok"], cfg.lam,
+                         mode=orc.MODE_PROXY, active=active)
+    for k in sc:
+        assert np.array_equal(out["scan"][k], sc[k]), k
+    # the subset matters: a verified sequence has finite outputs and a walk, the others have neither
+    for b in range(cfg.B):
+        if b in seqs:
+            assert np.isfinite(out["o"][b]).all() and np.isfinite(out["stats"]["lse"][b]).all()
+            assert out["scan"]["last_node"][b] >= 0
+        else:
+            assert np.isnan(out["o"][b]).all() and np.isnan(out["stats"]["lse"][b]).all()
+            assert out["scan"]["last_node"][b] == -1 and out["scan"]["accept_len"][b] == 0
+    # and the outcome is not degenerate: both routing cases occur, something is accepted
+    assert out["scan"]["escalate"][seqs].sum() + (out["scan"]["bonus_tok"][seqs] >= 0).sum() == len(seqs)
+    # TARGET mode of the same call never escalates and accepts at least as much on every sequence
+    tgt = orc.verify(inp, scale, cfg.logit_scale, cfg.lam, mode=orc.MODE_TARGET, with_attention=False)
+    assert "o" not in tgt and tgt["scan"]["escalate"].sum() == 0
+    assert (tgt["scan"]["accept_len"][seqs] >= out["scan"]["accept_len"][seqs]).all()

@@ -2,6 +2,7 @@
 cases that reduce to the identity or to a plain slice, invariants that tie them to the tree mask
 and to the attention oracle, and brute force on small random trees."""
 import itertools
+import math
 
 import numpy as np
 import pytest
@@ -360,3 +361,195 @@ def test_stochastic_scan_special_cases_and_acceptance_probability():
     for j in range(1, Tc):
         pj = surv[j - 1]
         assert abs(lens[j:].sum() / n - pj) < 4 * np.sqrt(pj * (1 - pj) / n) + 1e-9
+
+
+def test_stochastic_scan_decides_in_double_precision_and_counts_near_ties():
+    """Eq. 6 compares u with min(1, p/q). A single-precision division rounds 0.1f/0.3f up to
+    0.33333334; a uniform number just below that but above the exact quotient must be REJECTED,
+    and counted as lying on the boundary (near_accept), whatever precision the arrays have."""
+    parent = np.array([[-1, 0]], dtype=np.int32)
+    tok = np.array([[0, 7]], dtype=np.int32)
+    one, zero = np.ones((1, 2), dtype=np.float32), np.zeros((1, 2), dtype=np.float32)
+    p = np.array([[0.0, 0.1]], dtype=np.float32)
+    q = np.array([[0.0, 0.3]], dtype=np.float32)
+    exact = float(p[0, 1]) / float(q[0, 1])
+    rounded = float(np.float32(p[0, 1]) / np.float32(q[0, 1]))
+    assert rounded != exact
+    lo, hi = min(exact, rounded), max(exact, rounded)
+    u_between = np.array([[0.0, (lo + hi) / 2]], dtype=np.float64)
+    r = orc.accept_scan_stochastic(one, zero, p, q, u_between, parent, tok, 0.5)
+    assert r["accept_len"][0] == (1 if u_between[0, 1] < exact else 0)
+    assert r["near_accept"][0] == 1
+    # far from the ratio on either side: decided, not counted
+    for uu, want in ((0.2, 1), (0.5, 0)):
+        r = orc.accept_scan_stochastic(one, zero, p, q, np.array([[0.0, uu]]), parent, tok, 0.5)
+        assert r["accept_len"][0] == want and r["near_accept"][0] == 0
+    # only children that are actually tested count: after the first accepted child the siblings are not
+    parent3 = np.array([[-1, 0, 0]], dtype=np.int32)
+    tok3 = np.array([[0, 7, 8]], dtype=np.int32)
+    p3 = np.array([[0.0, 0.5, 0.1]]); q3 = np.array([[0.0, 0.5, 0.3]])
+    u3 = np.array([[0.0, 0.9, exact]])
+    r = orc.accept_scan_stochastic(np.ones((1, 3)), np.zeros((1, 3)), p3, q3, u3, parent3, tok3, 0.5)
+    assert r["path"][0, 0] == 1 and r["near_accept"][0] == 0
+
+
+def test_gumbel_variate_range_is_bounded_by_the_23_bit_uniform():
+    """The uniform number keeps the upper 23 bits of a word, so the variate cannot leave
+    [-ln(-ln 2^-24), -ln(-ln(1 - 2^-24))]; an entry 19.45 below the best logit is out of reach."""
+    g_min, g_max = orc.gumbel_from_word(0), orc.gumbel_from_word(0xFFFFFFFF)
+    assert abs(g_min - (-math.log(24 * math.log(2)))) < 1e-12
+    assert abs(g_max - (-math.log(-math.log1p(-2.0 ** -24)))) < 1e-9
+    assert -2.813 < g_min < -2.811 and 16.63 < g_max < 16.64
+    assert g_max - g_min < 19.45
+    for w in (1, 0x1FF, 0x200, 0x7FFFFFFF, 0x80000000, 0xFFFFFE00):
+        assert g_min <= orc.gumbel_from_word(w) <= g_max
+    # words that differ only in the dropped 9 bits give the same variate; the next one up differs
+    assert orc.gumbel_from_word(0x200) == orc.gumbel_from_word(0x3FF) != orc.gumbel_from_word(0x400)
+    # monotone in the word
+    ws = [0, 0x200, 0x12345600, 0x80000000, 0xFFFFFFFF]
+    gs = [orc.gumbel_from_word(w) for w in ws]
+    assert all(a < b for a, b in zip(gs, gs[1:]))
+
+
+def _one_hot_rows(B, T, d, hot):
+    """bf16 hidden states that are unit vectors: row (b, i) = e_{hot[b][i]}."""
+    h = np.zeros((B, T, d), dtype=np.float32)
+    for b in range(B):
+        for i in range(T):
+            h[b, i, hot[b][i]] = 1.0
+    return gen.f32_to_bf16_bits(h)
+
+
+def test_sample_bonus_on_hand_set_logits():
+    """Algorithm 1's x_bonus ~ p: with one-hot hidden states the logits of row (b, node) are a
+    column of W, set by hand to bf16-exact values; the expected token is the arg-max of
+    z + noise with the noise taken from the scalar generator (counter (v div 4, b, step))."""
+    V, d, B, T = 7, 4, 4, 3
+    Wf = np.array([[0.0, 2.0, -1.0, 0.5],
+                   [1.0, 0.0, -1.0, 0.5],
+                   [0.5, -2.0, 3.0, 0.5],
+                   [0.0, 0.0, 0.0, 0.5],
+                   [-1.0, 1.0, 0.0, 0.5],
+                   [2.0, 1.5, 0.25, 0.5],
+                   [0.0, -0.5, 1.0, 0.5]], dtype=np.float32)
+    W = gen.f32_to_bf16_bits(Wf)
+    hot = [[0, 1, 2], [1, 2, 3], [2, 0, 1], [3, 3, 0]]
+    h = _one_hot_rows(B, T, d, hot)
+    scale = 1.5
+    node = np.array([2, 0, -1, 1])                 # sequence 2 is skipped
+    seed, step = 0xDEADBEEF12345678, (1 << 33) + 5  # both halves of the 64-bit step are used
+    tok, best, gap = orc.sample_bonus(h, W, scale, node, seed, step)
+    flipped = 0
+    for b in range(B):
+        if node[b] < 0:
+            assert tok[b] == -1 and np.isnan(best[b]) and np.isnan(gap[b])
+            continue
+        z = scale * Wf[:, hot[b][node[b]]].astype(np.float64)
+        y = np.array([z[v] + orc.gumbel_noise(seed, step, b, v) for v in range(V)])
+        order = np.argsort(-y, kind="stable")
+        assert tok[b] == order[0]
+        assert abs(best[b] - y[order[0]]) < 1e-12 and abs(gap[b] - (y[order[0]] - y[order[1]])) < 1e-12
+        flipped += int(order[0] != int(np.argmax(z)))
+    # sequence 3, node 1 has all logits equal (column 3): the winner is the arg-max of the noise alone
+    noise3 = [orc.gumbel_noise(seed, step, 3, v) for v in range(V)]
+    assert tok[3] == int(np.argmax(noise3))
+    # the noise must be able to overturn the arg-max of the logits: over rounds, it does, and the
+    # round index, the sequence index and the seed all change the draw
+    n_flip, draws = 0, set()
+    for st in range(200):
+        t2, _, _ = orc.sample_bonus(h, W, scale, node, seed, st)
+        n_flip += int(t2[0] != int(np.argmax(Wf[:, hot[0][2]])))
+        draws.add(tuple(int(x) for x in t2))
+    assert 5 < n_flip < 195 and len(draws) > 20
+    same_rows = _one_hot_rows(2, 1, d, [[0], [0]])
+    t3 = [tuple(orc.sample_bonus(same_rows, W, scale, np.array([0, 0]), seed, st)[0]) for st in range(50)]
+    assert any(a != b for a, b in t3)              # sequence index enters the counter
+    t4 = [orc.sample_bonus(same_rows, W, scale, np.array([0, 0]), seed + 1, st)[0][0] for st in range(50)]
+    assert [a for a, _ in t3] != t4                # so does the seed
+
+
+def test_sample_bonus_draws_follow_the_softmax():
+    """20 000 draws through sample_bonus itself (8 sequences x 2500 rounds, the same row in every
+    sequence): every frequency within 4 standard deviations of softmax(z)."""
+    V, d, B = 6, 2, 8
+    Wf = np.array([[1.0, 0.0], [0.0, 0.0], [-1.0, 0.0], [2.0, 0.0], [0.5, 0.0], [-3.0, 0.0]], dtype=np.float32)
+    W = gen.f32_to_bf16_bits(Wf)
+    h = _one_hot_rows(B, 1, d, [[0]] * B)
+    z = Wf[:, 0].astype(np.float64)
+    p = np.exp(z) / np.exp(z).sum()
+    W64 = orc.bf16_to_f64(W)
+    counts = np.zeros(V)
+    rounds = 2500
+    node = np.zeros(B, dtype=np.int64)
+    for step in range(rounds):
+        tok, _, _ = orc.sample_bonus(h, W, 1.0, node, 7, step, W64=W64)
+        counts += np.bincount(tok, minlength=V)
+    n = rounds * B
+    assert counts.sum() == n
+    assert np.all(np.abs(counts / n - p) < 4 * np.sqrt(p * (1 - p) / n))
+
+
+# ------------------------------------------------------------------------------ token-specific deferral rule
+def test_token_specific_rule_hand_chain():
+    """Chain 0 -> 1 -> 2 -> 3, alpha = 0.2 (the paper's setting): a drafted token is accepted iff
+    its probability is at least 0.8 of the verifier's maximum at that position."""
+    parent = np.array([[-1, 0, 1, 2]], dtype=np.int32)
+    tok = np.array([[0, 5, 6, 7]], dtype=np.int32)
+    p1 = np.array([[0.50, 0.60, 0.90, 0.70]])
+    p2 = np.zeros((1, 4))
+    top1 = np.array([[9, 6, 8, 4]], dtype=np.int64)      # only node 1's arg-max is the drafted token
+    # child probabilities at the parent's position: 0.45 >= 0.8*0.50 (accepted though not the arg-max),
+    # 0.60 >= 0.8*0.60 (the arg-max itself), 0.70 < 0.8*0.90 = 0.72 (deferred)
+    pd = np.array([[np.nan, 0.45, 0.60, 0.70]])
+    r = orc.accept_scan_token_specific(p1, p2, top1, pd, parent, tok, 0.0, 0.2, mode=orc.MODE_TARGET)
+    assert r["accept_len"][0] == 2 and r["path"][0, :3].tolist() == [1, 2, -1]
+    assert r["last_node"][0] == 2 and r["bonus_tok"][0] == 8 and r["escalate"][0] == 0
+    # greedy acceptance on the same statistics stops at the root: token 5 is not the arg-max 9
+    g = orc.accept_scan(p1, p2, top1, parent, tok, 0.0, mode=orc.MODE_TARGET)
+    assert g["accept_len"][0] == 0 and g["bonus_tok"][0] == 9
+    # the threshold itself: 0.72 exactly passes (>=), and is counted as lying on the boundary
+    pd_edge = np.array([[np.nan, 0.45, 0.60, 0.8 * 0.90]])
+    e = orc.accept_scan_token_specific(p1, p2, top1, pd_edge, parent, tok, 0.0, 0.2, mode=orc.MODE_TARGET)
+    assert e["accept_len"][0] == 3 and e["bonus_tok"][0] == 4 and e["near_accept"][0] == 1
+    # PROXY mode: the margin test comes first; node 2 untrusted (0.9 - 0.5 < 0.45) -> escalate with 2 accepted
+    p2m = np.array([[0.0, 0.0, 0.5, 0.0]])
+    m = orc.accept_scan_token_specific(p1, p2m, top1, pd, parent, tok, 0.45, 0.2, mode=orc.MODE_PROXY)
+    assert m["escalate"][0] == 1 and m["accept_len"][0] == 2 and m["bonus_tok"][0] == -1
+
+
+def test_token_specific_rule_limits_reduce_to_greedy_and_to_accept_everything():
+    """alpha = 0 on real softmax statistics is greedy acceptance (a token reaches the maximum
+    probability only by being the arg-max); alpha = 1 accepts the first child at every node
+    down to a leaf; the accepted length on a chain never shrinks as alpha grows."""
+    cfg = _cfg(B=6, k=14, max_depth=5, V=200, d=64, rho=0.3, logit_scale=3.6 / (0.02 * 8.0), seed=31)
+    inp = gen.make_inputs(cfg, with_attention=False)
+    st = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale)
+    parent, tok = inp["parent"], inp["tok"]
+    for mode in (orc.MODE_PROXY, orc.MODE_TARGET):
+        g = orc.accept_scan(st["p_top1"], st["p_top2"], st["top1_idx"], parent, tok, cfg.lam, mode=mode)
+        r0 = orc.accept_scan_token_specific(st["p_top1"], st["p_top2"], st["top1_idx"], st["p_draft"], parent, tok,
+                                            cfg.lam, 0.0, mode=mode)
+        for k in ("accept_len", "escalate", "bonus_tok", "path", "last_node", "near_thr"):
+            assert np.array_equal(g[k], r0[k]), (k, mode)
+    assert (g["accept_len"] > 0).any()
+    r1 = orc.accept_scan_token_specific(st["p_top1"], st["p_top2"], st["top1_idx"], st["p_draft"], parent, tok,
+                                        cfg.lam, 1.0, mode=orc.MODE_TARGET)
+    for b in range(cfg.B):
+        cur, want = 0, []
+        while (parent[b] == cur).any():
+            cur = int(np.nonzero(parent[b] == cur)[0][0])
+            want.append(cur)
+        assert r1["path"][b, :len(want)].tolist() == want and r1["accept_len"][b] == len(want)
+        assert r1["bonus_tok"][b] == st["top1_idx"][b, cur]
+    # chain: monotone in alpha
+    ccfg = gen.small_variant(gen.CONFIGS["tiny_chain"], B=5, V=200, d=64, logit_scale=3.6 / (0.02 * 8.0), seed=32)
+    cin = gen.make_inputs(ccfg, with_attention=False)
+    cst = orc.lmhead_stats(cin["h"], cin["W"], cin["parent"], cin["tok"], ccfg.logit_scale)
+    prev = None
+    for alpha in (0.0, 0.2, 0.5, 0.9, 1.0):
+        r = orc.accept_scan_token_specific(cst["p_top1"], cst["p_top2"], cst["top1_idx"], cst["p_draft"],
+                                           cin["parent"], cin["tok"], 0.5, alpha, mode=orc.MODE_TARGET)
+        if prev is not None:
+            assert (r["accept_len"] >= prev).all()
+        prev = r["accept_len"].copy()
+    assert (prev == ccfg.k).all()
