@@ -147,7 +147,8 @@ def verify_attn(q: np.ndarray, k_tree: np.ndarray, v_tree: np.ndarray, mask: np.
 # ----------------------------------------------------------------------------------------
 # LM-head softmax statistics (Eq. 5 distributions; top_1/top_2 of Eq. 8)
 # ----------------------------------------------------------------------------------------
-STAT_F = ("max", "lse", "top1_val", "top2_val", "p_top1", "p_top2", "draft_logit", "p_draft", "entropy")
+STAT_F = ("max", "lse", "top1_val", "top2_val", "top3_val", "p_top1", "p_top2", "draft_logit", "p_draft",
+          "entropy")
 STAT_I = ("top1_idx", "top2_idx")
 
 
@@ -161,7 +162,9 @@ def lmhead_stats(h: np.ndarray, W: np.ndarray, parent: np.ndarray, tok: np.ndarr
                  W64: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
     """Per row r = (b, node): p = softmax(z) over the vocabulary, reduced to
     max z, lse = log sum exp z, the largest entry (top1_val, top1_idx; ties -> lowest index),
-    the largest entry among the other indices (top2_val, top2_idx), p_top1, p_top2; and for
+    the largest entry among the other indices (top2_val, top2_idx), the largest entry among the
+    rest (top3_val; reported so that a comparison can tell when top2_idx sits on a tie), p_top1,
+    p_top2; and for
     each child node c the logit of its drafted token in its parent's row (draft_logit[b][c])
     and the probability p_draft[b][c] = p_{parent(c)}(tok[c]). Entries of node 0 in
     draft_logit / p_draft are NaN. entropy = -sum_v p ln p (nats), the feature of the entropy
@@ -181,6 +184,9 @@ def lmhead_stats(h: np.ndarray, W: np.ndarray, parent: np.ndarray, tok: np.ndarr
             z_wo = z.copy()
             z_wo[i1] = -np.inf
             i2 = int(np.argmax(z_wo))
+            z_wo[i2] = -np.inf
+            # third largest entry: only for the parity tests' accounting of near-ties behind top_2
+            out["top3_val"][b, r] = z_wo.max() if len(z) > 2 else np.nan
             out["max"][b, r] = m
             out["lse"][b, r] = lse
             out["top1_val"][b, r] = z[i1]

@@ -242,6 +242,7 @@ def test_stats_against_exact_rational_logits_and_full_sort():
         assert abs(st["lse"][0, r] - lse) < 1e-13
         assert abs(st["p_top1"][0, r] - math.exp(z[order[0]] - lse)) < 1e-13
         assert abs(st["p_top2"][0, r] - math.exp(z[order[1]] - lse)) < 1e-13
+        assert abs(st["top3_val"][0, r] - z[order[2]]) < 1e-13
         # probabilities over the vocabulary sum to one
         assert abs(math.fsum(math.exp(x - st["lse"][0, r]) for x in z) - 1.0) < 1e-12
     # drafted-token probability is read in the PARENT's row
