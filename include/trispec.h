@@ -30,7 +30,18 @@
  *     T <= 64, Hq / Hkv in {1, 2, 4, 8, 16}.
  *   - Rows of per-node arrays are indexed row = b * T + node.
  *   - `dev_status` (optional, int32 on the device, caller zeroes it): receives a non-zero
- *     code if a bounded device-side wait gave up; the kernels never trap.
+ *     trispec_status code when a kernel meets a condition it has to work around (a bounded wait
+ *     that gave up, an index or length outside its range, a malformed tree); the kernels never
+ *     trap and never read or write outside the caller's arrays because of such a value.
+ *   - Ordering. A call may read any of its inputs as soon as its first kernel starts, and that
+ *     kernel is an ordinary stream-ordered launch: whatever was enqueued on `stream` before the
+ *     call - the caller's own kernels and copies, or an earlier call of this library such as a
+ *     KV commit, a pruning step or the scan that wrote an escalation list - has completed by
+ *     then. One exception is the caller's to avoid: a kernel that uses programmatic dependent
+ *     launch and signals completion before its last write to q, k_tree, v_tree, h, the KV
+ *     cache or an index array must not be the last thing on the stream before a call.
+ *     Inside one call the library's kernels overlap their prologues and tails (programmatic
+ *     dependent launch); seen from the stream a call is one ordered unit of work.
  */
 #ifndef TRISPEC_H_
 #define TRISPEC_H_
@@ -48,8 +59,13 @@ typedef enum {
   TRISPEC_ERR_UNSUPPORTED = 2,     /* D != 128, T > 64, unsupported group size, ... */
   TRISPEC_ERR_WORKSPACE = 3,       /* workspace_bytes smaller than the *_workspace() query */
   TRISPEC_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed */
-  TRISPEC_ERR_DEVICE_TIMEOUT = 5,  /* value written to dev_status by a bounded wait */
-  TRISPEC_ERR_TOO_LARGE = 8        /* problem needs more than the library's built-in scratch */
+  TRISPEC_ERR_DEVICE_TIMEOUT = 5,  /* dev_status: a bounded device-side wait gave up; results are invalid */
+  TRISPEC_ERR_BAD_BLOCK = 6,       /* dev_status: block_table entry outside [0, num_blocks), read as block 0 */
+  TRISPEC_ERR_SMEM_ALIGN = 7,      /* dev_status: a kernel's shared-memory window was not where it must be */
+  TRISPEC_ERR_TOO_LARGE = 8,       /* problem needs more than the library's built-in scratch */
+  TRISPEC_ERR_NO_ROOM = 9,         /* dev_status: a KV commit would exceed a sequence's capacity; skipped */
+  TRISPEC_ERR_BAD_LENGTH = 10,     /* dev_status: ctx_len[b] outside [0, capacity], clamped to it */
+  TRISPEC_ERR_BAD_TREE = 11        /* dev_status: parent[] of some sequence is not a tree (see entry 1) */
 } trispec_status;
 
 #define TRISPEC_MODE_PROXY 0   /* margin rule of Eq. 8-9 applied (proxy verifier) */
@@ -59,6 +75,12 @@ typedef enum {
 #define TRISPEC_CRIT_MARGIN 0   /* p_top1 - p_top2 >= lambda (Eq. 8; the paper's default) */
 #define TRISPEC_CRIT_TOP1 1     /* p_top1 >= lambda */
 #define TRISPEC_CRIT_ENTROPY 2  /* entropy <= lambda (plain Shannon entropy in nats) */
+
+/* acceptance rules: a drafted child c of the current node is accepted iff */
+#define TRISPEC_ACCEPT_GREEDY 0          /* tok[c] is the arg-max token (greedy form of Eq. 6) */
+#define TRISPEC_ACCEPT_STOCHASTIC 1      /* u < min(1, p(tok[c]) / q(tok[c])) (Eq. 6 at temperature 1) */
+#define TRISPEC_ACCEPT_TOKEN_SPECIFIC 2  /* p(tok[c]) >= (1 - alpha) * max p (token-specific deferral
+                                            rule, appendix "Baseline Implementation Details: SpecCascade") */
 
 #define TRISPEC_KV_CONTIGUOUS 0 /* k_cache, v_cache: [B][Lmax][Hkv][D] */
 #define TRISPEC_KV_PAGED 1      /* pool [num_blocks][block_size][Hkv][D] + block_table */
@@ -73,13 +95,17 @@ long long trispec_launch_count(void);
  *    parent [B][T] int32: parent[b][0] = -1, 0 <= parent[b][i] < i.
  *    mask   [B][T] uint64: bit j of mask[b][i] is 1 iff j is an ancestor of i or j == i.
  *    depth  [B][T] int32 : edges from the root (may be NULL).
- *    Malformed parents (>= i or < -1) are not dereferenced: the row gets mask 0 and depth -1.
+ *    Malformed parents (>= i or < -1, or parent[b][0] != -1) are not dereferenced: the node and
+ *    every node below it get mask 0 and depth -1 (such a node attends to no tree key),
+ *    and dev_status (optional) receives TRISPEC_ERR_BAD_TREE, which is
+ *    how a caller of the fused pass learns of it after the pass.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
   int B, T;
   const int32_t* parent;
   uint64_t* mask;
   int32_t* depth;
+  int32_t* dev_status;
 } trispec_tree_args;
 int trispec_build_tree_mask(const trispec_tree_args* a, void* stream);
 
@@ -91,7 +117,8 @@ int trispec_build_tree_mask(const trispec_tree_args* a, void* stream);
  *    kv_layout CONTIGUOUS: k_cache/v_cache [B][Lmax][Hkv][D] bf16.
  *    kv_layout PAGED: pool [num_blocks][block_size=64][Hkv][D]; token t of sequence b is in
  *      block block_table[b][t / 64] (int32 [B][max_blocks_per_seq]), slot t % 64.
- *    ctx_len [B] int32, 0 <= ctx_len[b] <= Lmax (contiguous) or 64 * max_blocks_per_seq.
+ *    ctx_len [B] int32, 0 <= ctx_len[b] <= Lmax (contiguous) or 64 * max_blocks_per_seq; a
+ *      value outside that range is clamped to it and dev_status receives TRISPEC_ERR_BAD_LENGTH.
  *    seq_index (optional, int32 [B_active], device): only these sequences are computed;
  *      NULL = all B (then B_active is ignored).
  *    lse (optional) f32 [B][Hq][T]: log-sum-exp of the scaled scores.
@@ -99,7 +126,8 @@ int trispec_build_tree_mask(const trispec_tree_args* a, void* stream);
  *      nodes (a pruned tree: n_keep of trispec_prune_tree, the branches that are passed on to
  *      the target in routing case (ii)); rows o[b][i] and lse of nodes i >= n_nodes[b] are
  *      neither computed nor written, and whole 128-row tiles past them cost nothing. The
- *      mask rows of the remaining nodes must not name nodes >= n_nodes[b]. NULL = T nodes.
+ *      mask rows of the remaining nodes must not name nodes >= n_nodes[b]; rows of q, k_tree
+ *      and v_tree past the count may hold anything (they are never used). NULL = T nodes.
  *    workspace: device scratch of at least trispec_verify_attn_workspace(a) bytes,
  *      256-byte aligned; contents are undefined before and after the call. The query
  *      returns 0 (and workspace may be NULL) whenever the context is cut into at most 8
@@ -201,6 +229,13 @@ int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream);
  *      node order and the first accepted one is taken. When none is accepted the round ends in
  *      case (i) with bonus_tok = -2: the bonus token has to be sampled at last_node
  *      (trispec_sample_bonus). The decision is taken in fp32 (IEEE division).
+ *    Token-specific deferral rule (accept_rule = TRISPEC_ACCEPT_TOKEN_SPECIFIC; the rule of the
+ *      SpecCascade baselines that looks only at the verifier's distribution; the paper runs it
+ *      with alpha = 0.2): child c of the current node is accepted iff
+ *      in.p_draft[c] >= (1 - alpha) * in.p_top1[current node], 0 <= alpha <= 1, compared in fp32;
+ *      the children are tried in node order and the first that passes is taken; when none
+ *      passes the round ends in case (i) with bonus_tok = top1_idx of the current node.
+ *      alpha = 0 is greedy acceptance, alpha = 1 accepts any drafted token.
  *    active (optional uint8 [B]): sequences with 0 are skipped (outputs: accept_len 0,
  *      escalate 0, bonus -1, last_node -1, path -1).
  *    Outputs: accept_len, bonus_tok, last_node, near_thr int32 [B]; escalate uint8 [B];
@@ -221,6 +256,8 @@ typedef struct {
   const uint8_t* active;
   const int32_t* start_node;
   const float *q_draft, *u_accept;  /* both NULL: greedy acceptance; both set: Eq. 6 at temperature 1 */
+  int accept_rule;                  /* TRISPEC_ACCEPT_*; GREEDY with q_draft/u_accept set means STOCHASTIC */
+  float alpha;                      /* slack of the token-specific rule; ignored by the other rules */
   int32_t *accept_len, *bonus_tok, *path, *last_node, *near_thr, *n_escalated, *esc_index;
   uint8_t* escalate;
 } trispec_scan_args;
@@ -338,6 +375,11 @@ int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
  * these orders: (parent, tok, h), (q, k_tree, v_tree), (accept_len, bonus_tok, last_node,
  * path, escalate). A caller that carves each group out of one host and one device buffer in
  * that order pays three transfers per round instead of eleven.
+ * The device buffers behind tree->parent, lm->tok, lm->h, attn->q, attn->k_tree and
+ * attn->v_tree are WRITTEN by this call although the argument structs declare them const (they
+ * are inputs of the pass proper). The structs must describe one pass: tree->parent, lm->parent
+ * and scan->parent have to be the same pointer, and so do lm->tok and scan->tok; otherwise the
+ * call returns TRISPEC_ERR_INVALID_ARG and does nothing.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
   const int32_t *parent, *tok;              /* host [B][T] */

@@ -30,7 +30,7 @@ _vp, _i, _f, _sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
 
 
 class TreeArgs(C.Structure):
-    _fields_ = [("B", _i), ("T", _i), ("parent", _vp), ("mask", _vp), ("depth", _vp)]
+    _fields_ = [("B", _i), ("T", _i), ("parent", _vp), ("mask", _vp), ("depth", _vp), ("dev_status", _vp)]
 
 
 class AttnArgs(C.Structure):
@@ -57,7 +57,7 @@ class LmheadArgs(C.Structure):
 class ScanArgs(C.Structure):
     _fields_ = [("B", _i), ("T", _i), ("lam", _f), ("mode", _i), ("criterion", _i), ("parent", _vp), ("tok", _vp),
                 ("stats", Stats), ("active", _vp), ("start_node", _vp), ("q_draft", _vp), ("u_accept", _vp),
-                ("accept_len", _vp),
+                ("accept_rule", _i), ("alpha", _f), ("accept_len", _vp),
                 ("bonus_tok", _vp), ("path", _vp), ("last_node", _vp), ("near_thr", _vp),
                 ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
 
@@ -181,9 +181,10 @@ def _stats_struct(st: Dict[str, torch.Tensor]) -> Stats:
 
 
 # ------------------------------------------------------------------------------ argument builders
-def tree_args(parent: torch.Tensor, mask: torch.Tensor, depth: Optional[torch.Tensor]) -> TreeArgs:
+def tree_args(parent: torch.Tensor, mask: torch.Tensor, depth: Optional[torch.Tensor],
+              dev_status: Optional[torch.Tensor] = None) -> TreeArgs:
     B, T = parent.shape
-    return _hold(TreeArgs(B, T, _p(parent), _p(mask), _p(depth)), parent, mask, depth)
+    return _hold(TreeArgs(B, T, _p(parent), _p(mask), _p(depth), _p(dev_status)), parent, mask, depth, dev_status)
 
 
 def attn_args(q, k_tree, v_tree, mask, k_cache, v_cache, ctx_len, scale, o, workspace=None,
@@ -229,10 +230,12 @@ def lmhead_args(h, W, parent, tok, logit_scale, stats, workspace=None, seq_index
 
 
 CRIT_MARGIN, CRIT_TOP1, CRIT_ENTROPY = 0, 1, 2
+ACCEPT_GREEDY, ACCEPT_STOCHASTIC, ACCEPT_TOKEN_SPECIFIC = 0, 1, 2
 
 
 def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], active=None,
-              start_node=None, criterion=CRIT_MARGIN, q_draft=None, u_accept=None) -> ScanArgs:
+              start_node=None, criterion=CRIT_MARGIN, q_draft=None, u_accept=None,
+              accept_rule=ACCEPT_GREEDY, alpha=0.0) -> ScanArgs:
     B, T = parent.shape
     a = ScanArgs()
     a.B, a.T, a.lam, a.mode, a.criterion = B, T, float(lam), int(mode), int(criterion)
@@ -240,6 +243,7 @@ def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], activ
     a.stats = _stats_struct(stats)
     a.active, a.start_node = _p(active), _p(start_node)
     a.q_draft, a.u_accept = _p(q_draft), _p(u_accept)
+    a.accept_rule, a.alpha = int(accept_rule), float(alpha)
     for k in ("accept_len", "bonus_tok", "path", "last_node", "near_thr", "n_escalated", "esc_index", "escalate"):
         setattr(a, k, _p(out.get(k)))
     return _hold(a, stats, parent, tok, out, active, start_node, q_draft, u_accept)

@@ -24,7 +24,9 @@ __device__ __forceinline__ float scan_feature(const trispec_scan_args& a, long l
 // The walk of one sequence by one warp; writes the sequence's outputs and returns its escalation flag.
 // The routing criterion and the acceptance rule are compile-time switches: the kernel is short and
 // latency-bound, and the plain case (margin rule, greedy acceptance) pays for nothing else.
-template <int kCrit, bool kStochastic>
+// kAccept: TRISPEC_ACCEPT_GREEDY (arg-max match), _STOCHASTIC (Eq. 6 at temperature 1) or
+// _TOKEN_SPECIFIC (the token-specific deferral rule of the SpecCascade baselines).
+template <int kCrit, int kAccept>
 __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const long long b, const int lane) {
   const int T = a.T;
   const long long base = b * T;
@@ -49,6 +51,15 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
   const bool proxy = (a.mode == TRISPEC_MODE_PROXY);
   int par0 = -2, par1 = -2, tok0 = 0, tok1 = 0, top0 = -1, top1v = -1;
   bool tr0 = true, tr1 = true, nr0 = false, nr1 = false;   // margin >= lambda / within 1e-3 of it
+  constexpr bool stochastic = (kAccept == TRISPEC_ACCEPT_STOCHASTIC);
+  constexpr bool token_rule = (kAccept == TRISPEC_ACCEPT_TOKEN_SPECIFIC);
+  // token-specific rule: top-1 probability of this lane's nodes (the bar a child has to reach is
+  // (1 - alpha) times its parent's) and the probability of the nodes' own drafted tokens
+  float pt0 = 0.f, pt1 = 0.f, pd0 = -1.f, pd1 = -1.f;
+  if (token_rule) {
+    if (has0) { pt0 = __ldg(a.in.p_top1 + base + lane); if (lane > 0) pd0 = __ldg(a.in.p_draft + base + lane); }
+    if (has1) { pt1 = __ldg(a.in.p_top1 + base + lane + 32); pd1 = __ldg(a.in.p_draft + base + lane + 32); }
+  }
   if (has0) {
     par0 = __ldg(a.parent + base + lane); tok0 = __ldg(a.tok + base + lane);
     top0 = __ldg(a.in.top1_idx + base + lane);
@@ -73,7 +84,6 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
   const unsigned long long near_bits =
       __ballot_sync(0xffffffffu, nr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, nr1)) << 32);
   // Bernoulli acceptance of Eq. 6 for every node at once: bit c = child c passes its test
-  constexpr bool stochastic = kStochastic;
   unsigned long long passes = ~0ull;
   if (stochastic) {
     bool ps0 = false, ps1 = false;
@@ -103,9 +113,18 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
       near += static_cast<int>((near_bits >> cur) & 1ull);
       if (!((trusted >> cur) & 1ull)) { esc = 1; break; }
     }
-    // greedy: the child whose token is the arg-max; stochastic: the first child that passed
-    unsigned m0 = __ballot_sync(0xffffffffu, par0 == cur && (stochastic || tok0 == top1));
-    unsigned m1 = __ballot_sync(0xffffffffu, par1 == cur && (stochastic || tok1 == top1));
+    // greedy: the child whose token is the arg-max; stochastic: the first child that passed its
+    // Bernoulli test; token-specific: the first child at least (1 - alpha) as probable as the arg-max
+    unsigned m0, m1;
+    if (token_rule) {
+      const float p_lo = __shfl_sync(0xffffffffu, pt0, src), p_hi = __shfl_sync(0xffffffffu, pt1, src);
+      const float bar = (1.f - a.alpha) * ((cur < 32) ? p_lo : p_hi);
+      m0 = __ballot_sync(0xffffffffu, par0 == cur && pd0 >= bar);
+      m1 = __ballot_sync(0xffffffffu, par1 == cur && pd1 >= bar);
+    } else {
+      m0 = __ballot_sync(0xffffffffu, par0 == cur && (stochastic || tok0 == top1));
+      m1 = __ballot_sync(0xffffffffu, par1 == cur && (stochastic || tok1 == top1));
+    }
     if (stochastic) { m0 &= static_cast<unsigned>(passes); m1 &= static_cast<unsigned>(passes >> 32); }
     int nxt = -1;
     if (m0) nxt = __ffs(m0) - 1;
@@ -128,7 +147,7 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
   return esc;
 }
 
-template <int kCrit, bool kStochastic>
+template <int kCrit, int kAccept>
 __global__ void __launch_bounds__(kScanThreads)
 accept_scan_kernel(trispec_scan_args a) {
   pdl_launch_dependents();
@@ -136,21 +155,21 @@ accept_scan_kernel(trispec_scan_args a) {
   const int lane = threadIdx.x & 31;
   const long long b = static_cast<long long>(blockIdx.x) * (kScanThreads / 32) + (threadIdx.x >> 5);
   if (b >= a.B) return;
-  scan_sequence<kCrit, kStochastic>(a, b, lane);
+  scan_sequence<kCrit, kAccept>(a, b, lane);
 }
 
 // Up to 32 sequences (a decode batch): one block, one warp per sequence, and the ordered list of
 // escalated sequences is made by the same block from a ballot of the flags, which saves the second
 // launch of the general path.
 constexpr int kScanSmallMax = 32;
-template <int kCrit, bool kStochastic>
+template <int kCrit, int kAccept>
 __global__ void __launch_bounds__(32 * kScanSmallMax)
 accept_scan_small_kernel(trispec_scan_args a) {
   __shared__ int s_esc[kScanSmallMax];
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int esc = (warp < a.B) ? scan_sequence<kCrit, kStochastic>(a, warp, lane) : 0;
+  const int esc = (warp < a.B) ? scan_sequence<kCrit, kAccept>(a, warp, lane) : 0;
   if (lane == 0) s_esc[warp] = esc;
   __syncthreads();
   if (warp == 0 && a.esc_index) {
@@ -245,6 +264,7 @@ esc_compact_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restr
 }  // namespace trispec
 
 extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   if (!a || a->B <= 0 || a->T <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->T > 64) return TRISPEC_ERR_UNSUPPORTED;
@@ -260,20 +280,27 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
   }
   if ((a->n_escalated == nullptr) != (a->esc_index == nullptr)) return TRISPEC_ERR_INVALID_ARG;
   if ((a->q_draft == nullptr) != (a->u_accept == nullptr)) return TRISPEC_ERR_INVALID_ARG;
-  if (a->q_draft && !a->in.p_draft) return TRISPEC_ERR_INVALID_ARG;
+  // acceptance rule: the Bernoulli inputs select Eq. 6 when the rule field is left at its default
+  int rule = a->accept_rule;
+  if (rule == TRISPEC_ACCEPT_GREEDY && a->q_draft) rule = TRISPEC_ACCEPT_STOCHASTIC;
+  if (rule < TRISPEC_ACCEPT_GREEDY || rule > TRISPEC_ACCEPT_TOKEN_SPECIFIC) return TRISPEC_ERR_INVALID_ARG;
+  if (rule == TRISPEC_ACCEPT_STOCHASTIC && (!a->q_draft || !a->in.p_draft)) return TRISPEC_ERR_INVALID_ARG;
+  if (rule == TRISPEC_ACCEPT_TOKEN_SPECIFIC &&
+      (!a->in.p_draft || !a->in.p_top1 || !(a->alpha >= 0.f && a->alpha <= 1.f)))
+    return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // kernel instance for (criterion, acceptance rule); TARGET mode reads no feature: margin instance
   const int crit = (a->mode == TRISPEC_MODE_PROXY) ? a->criterion : TRISPEC_CRIT_MARGIN;
-  const int which = crit * 2 + (a->q_draft ? 1 : 0);
+  const int which = crit * 3 + rule;
   typedef void (*ScanKernel)(trispec_scan_args);
-  static const ScanKernel small_k[6] = {
-      accept_scan_small_kernel<TRISPEC_CRIT_MARGIN, false>,  accept_scan_small_kernel<TRISPEC_CRIT_MARGIN, true>,
-      accept_scan_small_kernel<TRISPEC_CRIT_TOP1, false>,    accept_scan_small_kernel<TRISPEC_CRIT_TOP1, true>,
-      accept_scan_small_kernel<TRISPEC_CRIT_ENTROPY, false>, accept_scan_small_kernel<TRISPEC_CRIT_ENTROPY, true>};
-  static const ScanKernel big_k[6] = {
-      accept_scan_kernel<TRISPEC_CRIT_MARGIN, false>,  accept_scan_kernel<TRISPEC_CRIT_MARGIN, true>,
-      accept_scan_kernel<TRISPEC_CRIT_TOP1, false>,    accept_scan_kernel<TRISPEC_CRIT_TOP1, true>,
-      accept_scan_kernel<TRISPEC_CRIT_ENTROPY, false>, accept_scan_kernel<TRISPEC_CRIT_ENTROPY, true>};
+#define TRISPEC_SCAN_ROW(K, C) K<C, TRISPEC_ACCEPT_GREEDY>, K<C, TRISPEC_ACCEPT_STOCHASTIC>, K<C, TRISPEC_ACCEPT_TOKEN_SPECIFIC>
+  static const ScanKernel small_k[9] = {TRISPEC_SCAN_ROW(accept_scan_small_kernel, TRISPEC_CRIT_MARGIN),
+                                        TRISPEC_SCAN_ROW(accept_scan_small_kernel, TRISPEC_CRIT_TOP1),
+                                        TRISPEC_SCAN_ROW(accept_scan_small_kernel, TRISPEC_CRIT_ENTROPY)};
+  static const ScanKernel big_k[9] = {TRISPEC_SCAN_ROW(accept_scan_kernel, TRISPEC_CRIT_MARGIN),
+                                      TRISPEC_SCAN_ROW(accept_scan_kernel, TRISPEC_CRIT_TOP1),
+                                      TRISPEC_SCAN_ROW(accept_scan_kernel, TRISPEC_CRIT_ENTROPY)};
+#undef TRISPEC_SCAN_ROW
   if (a->B <= kScanSmallMax) {
     TRISPEC_CUDA_OK(launch_dependent(small_k[which], 1u, static_cast<unsigned>(32 * a->B), 0, st, 1, *a));
     count_launch();

@@ -65,6 +65,7 @@ static_assert(AT_PART_ML2_OFF + AT_PART_ML2_MAX * 8 <= (AT_STAGES + 2) * AT_TILE
 struct AttnParams {
   int T, Hq, Hkv, G, NPT, n_mt, n_splits;
   int paged, max_blocks_per_seq, num_blocks;
+  int Lcap;         // capacity of a sequence's context: Lmax, or 64 x max_blocks_per_seq
   float scale_log2;
   const uint16_t* q;
   const int32_t *block_table, *ctx_len, *seq_index;
@@ -113,7 +114,13 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   const int g = idx % p.Hkv;
   const int a = idx / p.Hkv;
   const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
-  const int L = __ldg(p.ctx_len + b);
+  // a length outside [0, capacity] (a stale or corrupt entry) is clamped and flagged: the block
+  // table row and the cache are never read past their ends
+  int L = __ldg(p.ctx_len + b);
+  if (L < 0 || L > p.Lcap) {
+    if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, TRISPEC_ERR_BAD_LENGTH);
+    L = max(0, min(L, p.Lcap));
+  }
   // a pruned tree has fewer nodes: rows past them are not computed, M tiles past them do nothing
   const int nn = p.n_nodes ? max(0, min(p.T, __ldg(p.n_nodes + b))) : p.T;
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
@@ -130,7 +137,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
   const uint32_t base_u32 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base_u32 - smem_u32(smem_raw));
   const bool misaligned = base_u32 - smem_u32(smem_raw) > static_cast<uint32_t>(AT_SMEM_BYTES - AT_SMEM_USED);
-  if (misaligned && threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 7);   // shared window misaligned
+  if (misaligned && threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, TRISPEC_ERR_SMEM_ALIGN);
   // a split past the end of this sequence's context has nothing to do; in cluster mode it
   // still takes part in the merge (with weight zero), so it may not leave early
   const bool idle_cta = (split > last_split) || misaligned || (mtile * p.NPT >= nn);
@@ -193,7 +200,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         if (!p.paged || t >= t_end) return 0;
         int v = __ldg(table + t);
         if (v < 0 || v >= p.num_blocks) {
-          if (p.dev_status) atomicExch(p.dev_status, 6);   // bad block id: clamped, flagged
+          if (p.dev_status) atomicExch(p.dev_status, TRISPEC_ERR_BAD_BLOCK);   // clamped, flagged
           v = 0;
         }
         return v;
@@ -436,12 +443,14 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 #pragma unroll
       for (int cch = 0; cch < 8; ++cch) *reinterpret_cast<uint4*>(prow + ((cch ^ (row & 7)) << 4)) = pk[cch];
       l += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
-      if (nvalid < AT_BN) {
-        // keys past the end of the context: their V rows may hold anything (0 * NaN = NaN)
+      // keys past the end of the context, and tree nodes past the end of a pruned tree, have
+      // probability 0 but their V rows may hold anything (0 * NaN = NaN): zero them
+      const int vrows = tree ? ((nn < p.T) ? nn : AT_BN) : nvalid;
+      if (vrows < AT_BN) {
         mbar_wait(v_full + i % NV, (i / NV) & 1u, p.dev_status);
         uint8_t* sv = sV + (i % NV) * AT_TILE_BYTES;
-        for (int e = threadIdx.x; e < (AT_BN - nvalid) * 16; e += 128) {
-          const int r = nvalid + (e >> 4), c16 = e & 15;
+        for (int e = threadIdx.x; e < (AT_BN - vrows) * 16; e += 128) {
+          const int r = vrows + (e >> 4), c16 = e & 15;
           *reinterpret_cast<uint4*>(sv + (c16 >> 3) * AT_BOX_BYTES + r * 128 + ((c16 & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
       }
@@ -610,7 +619,7 @@ verify_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 // Merge of the KV splits: one warp per output row (sequence, node, query head).
 // ---------------------------------------------------------------------------------------
 struct AttnMergeParams {
-  int T, Hq, Hkv, G, NPT, n_mt, n_splits, n_seq;
+  int T, Hq, Hkv, G, NPT, n_mt, n_splits, n_seq, Lcap;
   const int32_t *ctx_len, *seq_index, *n_nodes;
   const float *part_o, *part_ml;
   uint16_t* o;   // bf16 [B][T][Hq][128]
@@ -633,7 +642,7 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
   const int g = hq / p.G, j = hq % p.G;
   const int mtile = node / p.NPT;
   const int row = (node % p.NPT) * p.G + j;
-  const int L = __ldg(p.ctx_len + b);
+  const int L = max(0, min(__ldg(p.ctx_len + b), p.Lcap));   // clamped as in the split kernel
   const int n_ctx_tiles = (L + AT_BN - 1) / AT_BN;
   const int tiles_per_split = max(1, (n_ctx_tiles + p.n_splits - 1) / p.n_splits);
   const int n_valid = max(0, (n_ctx_tiles + tiles_per_split - 1) / tiles_per_split - 1) + 1;
@@ -739,6 +748,7 @@ extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) {
 }
 
 extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   AttnPlan pl;
   int rc = attn_plan(a, &pl);
@@ -795,6 +805,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   p.n_splits = pl.n_splits;
   p.paged = (a->kv_layout == TRISPEC_KV_PAGED); p.max_blocks_per_seq = a->max_blocks_per_seq;
   p.num_blocks = a->num_blocks;
+  p.Lcap = p.paged ? a->max_blocks_per_seq * AT_BN : a->Lmax;
   p.scale_log2 = a->scale * kLog2e;
   p.q = static_cast<const uint16_t*>(a->q);
   p.block_table = a->block_table; p.ctx_len = a->ctx_len; p.seq_index = a->seq_index; p.mask = a->mask;
@@ -817,7 +828,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
 
   AttnMergeParams m;
   m.T = a->T; m.Hq = a->Hq; m.Hkv = a->Hkv; m.G = pl.G; m.NPT = pl.NPT; m.n_mt = pl.n_mt;
-  m.n_splits = pl.n_splits; m.n_seq = pl.n_seq;
+  m.n_splits = pl.n_splits; m.n_seq = pl.n_seq; m.Lcap = p.Lcap;
   m.ctx_len = a->ctx_len; m.seq_index = a->seq_index; m.n_nodes = a->n_nodes;
   m.part_o = p.part_o; m.part_ml = p.part_ml;
   m.o = static_cast<uint16_t*>(a->o); m.lse = a->lse;

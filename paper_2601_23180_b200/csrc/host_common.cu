@@ -10,6 +10,20 @@ namespace trispec {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+namespace {
+thread_local int tl_scope_depth = 0;
+thread_local bool tl_scope_launched = false;
+}  // namespace
+EntryScope::EntryScope() {
+  if (tl_scope_depth++ == 0) tl_scope_launched = false;
+}
+EntryScope::~EntryScope() { --tl_scope_depth; }
+bool entry_scope_next_launch_is_dependent() {
+  const bool dependent = tl_scope_depth > 0 && tl_scope_launched;
+  tl_scope_launched = true;
+  return dependent;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -117,6 +131,11 @@ extern "C" const char* trispec_status_string(int s) {
     case TRISPEC_ERR_WORKSPACE: return "workspace too small";
     case TRISPEC_ERR_CUDA: return "CUDA call failed";
     case TRISPEC_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case TRISPEC_ERR_BAD_BLOCK: return "block table entry out of range (device status)";
+    case TRISPEC_ERR_SMEM_ALIGN: return "shared-memory window misplaced (device status)";
+    case TRISPEC_ERR_NO_ROOM: return "no room in the KV cache for the committed rows (device status)";
+    case TRISPEC_ERR_BAD_LENGTH: return "context length out of range (device status)";
+    case TRISPEC_ERR_BAD_TREE: return "parent array is not a tree (device status)";
     case TRISPEC_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }

@@ -28,13 +28,31 @@ int device_sm_count();
 // Raises the dynamic shared memory limit of `func` once per device.
 int ensure_smem_limit(const void* func, int bytes, bool* done_per_device /* [64] */);
 
-// Every kernel of the verify pass is launched as a programmatic dependent of the kernel before
-// it on the stream: its CTAs may be scheduled as soon as all CTAs of that kernel have called
-// pdl_launch_dependents() (they do so at their start) and resources are free, so launch
-// latency, prologues and tails overlap. A kernel calls pdl_wait() before its first read of
-// anything an earlier kernel writes and before its first global write; the wait returns once
-// all earlier kernels on the stream have completed and their writes are visible. Because
-// every kernel waits before it completes, completion stays in stream order.
+// Programmatic dependent launch inside one call of the library. The FIRST kernel a public entry
+// point launches is an ordinary launch: it starts once everything enqueued on the stream before
+// the call has completed and its writes are visible, so every input of the call (activations,
+// the KV cache and its lengths, index arrays written by an earlier call such as the escalation
+// list, pruned-tree node counts or committed lengths) may be read by any kernel of the call at
+// any time. Every LATER kernel of the same call is launched as a programmatic dependent of the
+// kernel before it: its CTAs may be scheduled as soon as all CTAs of that kernel have called
+// pdl_launch_dependents() (they do so at their start) and resources are free, so launch latency,
+// prologues and tails inside a call overlap. Such a kernel calls pdl_wait() before its first read
+// of anything an earlier kernel OF THE SAME CALL writes and before its first global write; the
+// wait returns once all earlier kernels on the stream have completed and their writes are
+// visible. Because every kernel waits before it completes, completion stays in stream order.
+//
+// EntryScope marks the extent of one public call on the calling thread (nested entry points,
+// e.g. the fused pass calling the four steps, share the outermost scope).
+struct EntryScope {
+  EntryScope();
+  ~EntryScope();
+  EntryScope(const EntryScope&) = delete;
+  EntryScope& operator=(const EntryScope&) = delete;
+};
+// True if a kernel was already launched inside the current outermost scope (the next launch may
+// then be a programmatic dependent); records that a launch happens now.
+bool entry_scope_next_launch_is_dependent();
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
                                     cudaStream_t st, unsigned cluster_x, Args... args) {
@@ -45,9 +63,11 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, uns
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   unsigned n = 0;
-  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[n].val.programmaticStreamSerializationAllowed = 1;
-  ++n;
+  if (entry_scope_next_launch_is_dependent()) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
   if (cluster_x > 1) {
     attr[n].id = cudaLaunchAttributeClusterDimension;
     attr[n].val.clusterDim.x = cluster_x;

@@ -48,7 +48,7 @@ kv_commit_kernel(const CommitParams p) {
   const int L = __ldg(p.ctx_len + b);
   const int rows = commit_rows(p, b, L);
   if (rows < 0) {
-    if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, 9);   // no room: sequence skipped
+    if (threadIdx.x == 0 && p.dev_status) atomicExch(p.dev_status, TRISPEC_ERR_NO_ROOM);   // sequence skipped
     return;
   }
   const int row16 = p.Hkv * 16;                  // 16-byte units per row (Hkv x 128 bf16)
@@ -103,6 +103,7 @@ kv_commit_len_kernel(const CommitParams p) {
 }  // namespace trispec
 
 extern "C" int trispec_commit_kv(const trispec_commit_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   if (!a || a->B <= 0 || a->T <= 0 || a->Hkv <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->D != 128 || a->T > 64) return TRISPEC_ERR_UNSUPPORTED;

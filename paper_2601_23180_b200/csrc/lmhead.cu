@@ -717,6 +717,7 @@ extern "C" size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a) {
 }
 
 extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   int n_seq, n_mt, n_ranges;
   int rc = lm_plan(a, &n_seq, &n_mt, &n_ranges);
@@ -854,6 +855,7 @@ static int lm_noalloc_scratch(void** out) {
 }  // namespace trispec
 
 extern "C" int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   int n_seq, n_mt, n_ranges;
   int rc = lm_plan(a, &n_seq, &n_mt, &n_ranges);

@@ -86,6 +86,7 @@ prune_tree_kernel(trispec_prune_args a) {
 }  // namespace trispec
 
 extern "C" int trispec_prune_tree(const trispec_prune_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   if (!a || a->B <= 0 || a->T <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->T > 64) return TRISPEC_ERR_UNSUPPORTED;

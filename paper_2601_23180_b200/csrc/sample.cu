@@ -452,6 +452,7 @@ extern "C" size_t trispec_sample_bonus_workspace(const trispec_sample_args* a) {
 }
 
 extern "C" int trispec_sample_bonus(const trispec_sample_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   int n_mt, n_ranges;
   int rc = sample_plan(a, &n_mt, &n_ranges);

@@ -12,7 +12,7 @@ constexpr int kMaskSeqPerWarp = 2;  // sequences per warp: their loads are issue
 
 __global__ void __launch_bounds__(kMaskThreads)
 tree_mask_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask, int32_t* __restrict__ depth,
-                 long long n_seq, int T) {
+                 long long n_seq, int T, int32_t* __restrict__ status) {
   pdl_launch_dependents();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -37,6 +37,9 @@ tree_mask_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask
     int q0 = par0[u], q1 = par1[u];
     if (has0 && !(q0 >= -1 && q0 < lane && (lane != 0 || q0 == -1))) q0 = -2;
     if (has1 && !(q1 >= -1 && q1 < lane + 32)) q1 = -2;
+    // not a tree (a parent out of range, or a second root): reported through the status word
+    const bool bad = (has0 && (q0 == -2 || (lane != 0 && q0 == -1))) || (has1 && q1 < 0);
+    if (__any_sync(0xffffffffu, bad) && lane == 0 && status) atomicExch(status, TRISPEC_ERR_BAD_TREE);
     // both parents of a lane in one register (a byte each, biased by 2), so that a walk needs
     // one shuffle per level
     const int packed = (q0 + 2) | ((q1 + 2) << 8);
@@ -70,7 +73,7 @@ constexpr int kMaskRowPitch = kMaskBlockSeqs + 1;   // masks per node row
 
 __global__ void __launch_bounds__(kMaskBlockThreads)
 tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask, int32_t* __restrict__ depth,
-                       long long n_seq, int T) {
+                       long long n_seq, int T, int32_t* __restrict__ status) {
   __shared__ signed char sPar[64 * kMaskParPitch];
   __shared__ unsigned long long sMask[64 * kMaskRowPitch];
   pdl_launch_dependents();
@@ -97,19 +100,23 @@ tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict_
   __syncthreads();
   if (threadIdx.x < n_here) {
     const int t = threadIdx.x;
+    bool bad = false;
     for (int i = 0; i < T; ++i) {
       const int par = sPar[i * kMaskParPitch + t];
       unsigned long long m;
       if (par == -1) {
         m = 1ull << i;                                      // a root
+        bad |= (i != 0);                                    // a second root: not a tree
       } else if (par < 0 || par >= i) {
         m = 0ull;                                           // malformed: flagged, not followed
+        bad = true;
       } else {
         const unsigned long long pm = sMask[par * kMaskRowPitch + t];
         m = pm ? (pm | (1ull << i)) : 0ull;                 // a malformed ancestor spoils the walk
       }
       sMask[i * kMaskRowPitch + t] = m;
     }
+    if (bad && status) atomicExch(status, TRISPEC_ERR_BAD_TREE);
   }
   __syncthreads();
   uint64_t* dst = mask + s0 * T;
@@ -138,6 +145,7 @@ tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict_
 }  // namespace trispec
 
 extern "C" int trispec_build_tree_mask(const trispec_tree_args* a, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   if (!a || !a->parent || !a->mask || a->B <= 0 || a->T <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->T > 64) return TRISPEC_ERR_UNSUPPORTED;
@@ -145,14 +153,15 @@ extern "C" int trispec_build_tree_mask(const trispec_tree_args* a, void* stream)
   if (n >= 2048) {   // enough sequences to fill the chip with a thread each
     unsigned grid = static_cast<unsigned>((n + kMaskBlockSeqs - 1) / kMaskBlockSeqs);
     TRISPEC_CUDA_OK(launch_dependent(tree_mask_block_kernel, grid, kMaskBlockThreads, 0,
-                                     static_cast<cudaStream_t>(stream), 1, a->parent, a->mask, a->depth, n, a->T));
+                                     static_cast<cudaStream_t>(stream), 1, a->parent, a->mask, a->depth, n, a->T,
+                                     a->dev_status));
     count_launch();
     return TRISPEC_OK;
   }
   const int per_block = (kMaskThreads / 32) * kMaskSeqPerWarp;
   unsigned grid = static_cast<unsigned>((n + per_block - 1) / per_block);
   TRISPEC_CUDA_OK(launch_dependent(tree_mask_kernel, grid, kMaskThreads, 0, static_cast<cudaStream_t>(stream), 1,
-                                   a->parent, a->mask, a->depth, n, a->T));
+                                   a->parent, a->mask, a->depth, n, a->T, a->dev_status));
   count_launch();
   return TRISPEC_OK;
 }

@@ -6,6 +6,7 @@
 
 extern "C" int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                               const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   if (!tree || !lm || !scan) return TRISPEC_ERR_INVALID_ARG;
   int rc = trispec_build_tree_mask(tree, stream);
   if (rc != TRISPEC_OK) return rc;
@@ -53,8 +54,12 @@ static int host_pass_streams(HostPassStreams** out) {
 extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree_args* tree,
                                    const trispec_attn_args* attn, const trispec_lmhead_args* lm,
                                    const trispec_scan_args* scan, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
   if (!io || !tree || !lm || !scan) return TRISPEC_ERR_INVALID_ARG;
+  // the copies below land in the buffers the structs name: they must describe one and the same pass
+  if (tree->parent != lm->parent || tree->parent != scan->parent || lm->tok != scan->tok)
+    return TRISPEC_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t BT = static_cast<size_t>(tree->B) * tree->T;
   // A copy list is issued with neighbours merged: requests whose source AND destination follow

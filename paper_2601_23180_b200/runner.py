@@ -70,7 +70,7 @@ class VerifyPass:
         # the entropy is computed only for the routing criterion that reads it (the margin rule of Eq. 8 does not)
         self.stats = ts.alloc_stats(B, T, entropy=(criterion == ts.CRIT_ENTROPY))
         self.scan_out = ts.alloc_scan_out(B, T)
-        self.tree_args = ts.tree_args(d["parent"], self.mask, self.depth)
+        self.tree_args = ts.tree_args(d["parent"], self.mask, self.depth, dev_status=self.status)
         self.attn_args = None
         self.o = self.attn_lse = None
         if with_attention:

@@ -54,3 +54,31 @@ def test_host_side_argument_validation_without_gpu():
     l = ts.LmheadArgs()
     l.B, l.T, l.d, l.V = 1, 9, 100, 32000
     assert lib.trispec_lmhead_stats(ctypes.byref(l), None) == 2         # d % 64
+
+
+def test_status_strings_and_host_pass_struct_check_without_gpu():
+    """Every status code has its own text, and the host-buffer pass refuses argument structs that do
+    not describe one pass (different parent / token buffers) before any CUDA call."""
+    from paper_2601_23180_b200 import build
+    lib = ctypes.CDLL(build.build())
+    lib.trispec_status_string.restype = ctypes.c_char_p
+    texts = [lib.trispec_status_string(c) for c in range(0, 12)]
+    assert len(set(texts)) == 12 and b"unknown status" not in texts
+    assert lib.trispec_status_string(99) == b"unknown status"
+    from paper_2601_23180_b200 import binding as ts
+    io, t, l, s = ts.HostIO(), ts.TreeArgs(), ts.LmheadArgs(), ts.ScanArgs()
+    t.parent, l.parent, s.parent = 4096, 8192, 4096
+    assert lib.trispec_verify_host(ctypes.byref(io), ctypes.byref(t), None, ctypes.byref(l), ctypes.byref(s), None) == 1
+    l.parent = 4096
+    l.tok, s.tok = 256, 512
+    assert lib.trispec_verify_host(ctypes.byref(io), ctypes.byref(t), None, ctypes.byref(l), ctypes.byref(s), None) == 1
+    # the scan refuses an unknown acceptance rule or a slack outside [0, 1] before anything is launched
+    sc = ts.ScanArgs()
+    sc.B, sc.T = 2, 9
+    for f in ("parent", "tok", "accept_len", "bonus_tok", "path", "last_node", "escalate"):
+        setattr(sc, f, 4096)
+    sc.stats.top1_idx = sc.stats.p_top1 = sc.stats.p_top2 = sc.stats.p_draft = 4096
+    sc.accept_rule = 7
+    assert lib.trispec_accept_scan(ctypes.byref(sc), None) == 1
+    sc.accept_rule, sc.alpha = ts.ACCEPT_TOKEN_SPECIFIC, 1.5
+    assert lib.trispec_accept_scan(ctypes.byref(sc), None) == 1

@@ -3,7 +3,8 @@ benchmark times (the fused pass through `runner.VerifyPass`).
 
 The oracle cannot redo a whole pass at these sizes in reasonable time, so it recomputes
 sampled outputs one by one: a set of attention rows (sequence, node, head), the LM-head
-statistics of the first nodes of one sequence, the whole tree mask, and the acceptance scan
+statistics of three nodes in each of three sequences (all rows, and the scan decided by the oracle
+alone, for the two smallest workloads), the whole tree mask, and the acceptance scan
 of every sequence from the statistics the GPU produced (the rule is exact integer work on
 given statistics, so it must agree everywhere except where a margin sits on the threshold).
 Tolerances are those of the small-size parity tests.
@@ -19,7 +20,6 @@ from paper_2601_23180_b200 import inputs as gen
 pytestmark = pytest.mark.gpu
 
 N_ATTN_SAMPLES = 24
-N_LM_NODES = 12
 
 
 @pytest.mark.parametrize("name", gen.CONFIG_ORDER)
@@ -63,15 +63,45 @@ def test_full_size_pass_sampled_against_oracle(name):
     for b in untouched:
         assert np.isnan(got["o"][b]).all()
 
-    # ---- LM-head statistics: the first nodes of one sequence (parents precede children, so a
-    # prefix of the node list is a tree of its own)
-    b0 = seqs[len(seqs) // 2]
-    n = min(N_LM_NODES, T)
-    ref = orc.lmhead_stats(inp["h"][b0:b0 + 1, :n], inp["W"], inp["parent"][b0:b0 + 1, :n],
-                           inp["tok"][b0:b0 + 1, :n], cfg.logit_scale)
-    sub = {k: v[b0:b0 + 1, :n] for k, v in got["stats"].items()}
-    n_tie = H.check_stats(sub, ref, [0], n)
-    assert n_tie <= 1
+    # ---- LM-head statistics: the root, an inner node and the last node of the first, the middle and
+    # the last verified sequence, so that the first and last rows of an M tile and both CTAs of a
+    # pair are compared. The oracle gets each node as the second row of a two-row chain whose first
+    # row is the node's parent (the drafted-token probability is read in the parent's row).
+    W64 = orc.bf16_to_f64(inp["W"])
+    lm_seqs = sorted({seqs[0], seqs[len(seqs) // 2], seqs[-1]})
+    lm_nodes = sorted({0, min(12, T - 1), T - 1})
+    for b0 in lm_seqs:
+        for node in lm_nodes:
+            par = int(inp["parent"][b0, node])
+            rows = [node] if par < 0 else [par, node]
+            sub_parent = np.array([[-1, 0][:len(rows)]], dtype=np.int32)
+            ref = orc.lmhead_stats(inp["h"][b0:b0 + 1, rows], inp["W"], sub_parent, inp["tok"][b0:b0 + 1, rows],
+                                   cfg.logit_scale, W64=W64)
+            j = len(rows) - 1
+            sub = {k: v[b0:b0 + 1, node:node + 1] for k, v in got["stats"].items()}
+            one = {k: v[:, j:j + 1] for k, v in ref.items()}
+            n_tie = H.check_stats(sub, one, [0], 1)
+            assert n_tie <= 1
+
+    # ---- the two smallest workloads: the oracle's whole LM head, and the scan decided by the oracle alone
+    if name in ("tiny_chain", "proxy_tree"):
+        ref_st = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale, seqs=seqs, W64=W64)
+        H.check_stats(got["stats"], ref_st, seqs, T)
+        ref_only = orc.accept_scan(ref_st["p_top1"], ref_st["p_top2"], ref_st["top1_idx"], inp["parent"], inp["tok"],
+                                   cfg.lam, mode=cfg.mode)
+        gap = ref_st["top1_val"] - ref_st["top2_val"]
+        near_tie = gap < 1e-3 * np.maximum(1.0, np.abs(ref_st["top1_val"]))
+        n_cmp = 0
+        for b in seqs:
+            visited = [0] + [int(x) for x in ref_only["path"][b] if x >= 0]
+            if ref_only["near_thr"][b] > 0 or got["scan"]["near_thr"][b] > 0 or near_tie[b, visited].any():
+                continue
+            for k in ("accept_len", "escalate", "bonus_tok", "last_node"):
+                assert got["scan"][k][b] == ref_only[k][b], (k, b)
+            assert np.array_equal(got["scan"]["path"][b], ref_only["path"][b])
+            n_cmp += 1
+        assert n_cmp >= len(seqs) - max(1, len(seqs) // 4)
+    del W64
 
     # ---- acceptance scan: every sequence, from the GPU's own statistics
     st = got["stats"]

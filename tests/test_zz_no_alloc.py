@@ -5,7 +5,7 @@ memory pool already owns all free device memory: there a cudaMalloc fails, or st
 stream while it runs, so the loop has no way to obtain the workspace that
 `trispec_lmhead_stats` asks for. The variant keeps its partial statistics in a fixed 1 MiB
 array inside the library instead. This file checks, through the C ABI, that it returns what
-the workspace entry point returns, on two calls in a row with different inputs (the array
+the workspace entry point returns and what the CPU oracle computes, on two calls in a row with different inputs (the array
 is shared and keeps the previous call's contents, which must not leak into the next result),
 and that a problem too large for the array is refused before anything is launched.
 
@@ -14,6 +14,7 @@ The file is named so that pytest collects it after every other test file.
 import numpy as np
 import pytest
 
+from oracle import trispec_oracle as orc
 from paper_2601_23180_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
@@ -67,6 +68,11 @@ def test_noalloc_entry_matches_workspace_entry_twice_in_a_row():
         ref = _run(ts, torch, dev, cfg, noalloc=False)
         got = _run(ts, torch, dev, cfg, noalloc=True)
         _same(got, ref, seqs, cfg.T)
+        # and against the CPU oracle, with the tolerances of the LM-head parity tests: agreement of the
+        # two entry points alone would only show that they share their kernels
+        want = orc.lmhead_stats(inp["h"], inp["W"], inp["parent"], inp["tok"], cfg.logit_scale, seqs=seqs)
+        n_tie = H.check_stats(got, want, seqs, cfg.T)
+        assert n_tie <= 0.02 * len(seqs) * cfg.T + 2
 
 
 def test_noalloc_entry_refuses_what_does_not_fit():
