@@ -28,9 +28,15 @@ if ROOT not in sys.path:
 
 METRIC = "verified_draft_tokens_per_s"
 UNIT = "draft tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum (bytes) of one lmhead_gemm_kernel launch on the bench
-# workload, from the ncu capture summarised in profiles/lmhead_gemm_kernel_proxy_tree.md.
-LMHEAD_GEMM_DRAM_TRAFFIC = {"proxy_tree": 630.4e6}
+NOMINAL = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}     # data-sheet figures, for context beside the measured peaks
+
+
+def dram_traffic(kernel: str, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel` on `workload`, from the
+    tracked record of the last profiler capture, or None when there is no capture or when the kernel's
+    sources have changed since it was taken (the record carries their digest)."""
+    from paper_2601_23180_b200 import profile_traffic as pt
+    return pt.lookup(kernel, workload)
 
 
 def _peaks():
@@ -194,10 +200,12 @@ def run_reference(args, cfg, rank):
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg_tokens(cfg) / value,
+        # every step times a bounded sample of the pass and scales it to the whole pass: ms_per_step is
+        # what one whole pass of the oracle would take, not a time this run spent
+        "extrapolated": True, "seconds_measured": time.perf_counter() - t_start,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "draft_tokens": cfg.k, "context": cfg.L, "Hq": cfg.Hq,
-                   "Hkv": cfg.Hkv, "hidden": cfg.d, "vocab": cfg.V},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "config": config_dict(cfg),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle (numpy/BLAS)", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -409,6 +417,7 @@ def run_only(args, cfg):
         flops = 4.0 * rows * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
         roof = _roof(peaks, flops, byts, ms)
         roof["kernel"] = "verify_attn_split_kernel"
+        roof["traffic"] = dram_traffic("verify_attn_split_kernel", cfg.name)
     else:
         inp = gen.make_inputs(cfg, with_attention=False)
         pas = runner.VerifyPass(cfg, inp, with_attention=False)
@@ -417,7 +426,7 @@ def run_only(args, cfg):
         ms = timed(lambda: ts.trispec_lmhead_stats(pas.lm_args), lm_bytes)
         roof = _roof(peaks, 2.0 * M * cfg.d * cfg.V, lm_bytes, ms)
         roof["kernel"] = "lmhead_gemm_kernel (+ finalize)"
-        roof["traffic"] = LMHEAD_GEMM_DRAM_TRAFFIC.get(cfg.name)
+        roof["traffic"] = dram_traffic("lmhead_gemm_kernel", cfg.name)
     assert int(pas.status.item()) == 0, "a device-side wait timed out"
     out.update({"value": n_seq * cfg.k / (ms * 1e-3), "ms_per_step": ms, "dtype": "bf16", "roofline": roof})
     print(json.dumps(out), flush=True)
@@ -452,15 +461,178 @@ def cfg_tokens(cfg):
     return n * cfg.k
 
 
+def config_dict(cfg):
+    """The workload as both arms of the benchmark print it (same keys, same values)."""
+    n_seq = cfg.B if cfg.n_active is None else cfg.n_active
+    return {"workload": cfg.name, "B": cfg.B, "active_sequences": n_seq, "draft_tokens": cfg.k,
+            "tree_nodes": cfg.T, "context": cfg.L, "context_min": cfg.L if cfg.L_min is None else cfg.L_min,
+            "Hq": cfg.Hq, "Hkv": cfg.Hkv, "head_dim": cfg.D, "hidden": cfg.d, "vocab": cfg.V,
+            "kv": "paged" if cfg.paged else "contiguous", "mode": "target" if cfg.mode else "proxy",
+            "l2": "inputs larger than L2 (LM-head weights + KV cache are streamed every pass)",
+            "parallelism": "independent replicas, one batch per GPU"}
+
+
+# ---------------------------------------------------------------------------------------------
+# One workload measured through the fused call
+# ---------------------------------------------------------------------------------------------
+def _roofline(kind, peaks, flops, byts, ms, loop_ms, kernel, workload, timed):
+    """Roofline record of one entry point: the bound is the larger of the two lower-bound times at the
+    measured peaks. `frac` is against the measured peak (the sustained bf16 figure when the timed loop
+    ran long enough for the power cap to bite, else the burst figure); the burst and the data-sheet
+    fractions stand beside it."""
+    sustained = kind == "lmhead" and peaks.get("bf16_tflops_sustained") and loop_ms >= 200.0
+    tc_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    tflops, gbs = flops / (ms * 1e-3) / 1e12, byts / (ms * 1e-3) / 1e9
+    if flops / (tc_peak * 1e12) >= byts / (peaks["hbm_gbs"] * 1e9):
+        r = {"kernel": kernel, "bound": "tensor", "achieved": tflops, "peak": tc_peak, "unit": "TFLOP/s",
+             "frac": tflops / tc_peak, "work_per_launch": flops,
+             "peak_source": f"{peaks['source']} {'sustained' if sustained else 'burst'} bf16 GEMM",
+             "frac_of_burst_peak": tflops / peaks["bf16_tflops"], "frac_of_nominal": tflops / NOMINAL["bf16_tflops"]}
+    else:
+        r = {"kernel": kernel, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+             "frac": gbs / peaks["hbm_gbs"], "work_per_launch": byts,
+             "peak_source": f"{peaks['source']} copy bandwidth", "frac_of_nominal": gbs / NOMINAL["hbm_gbs"]}
+    r.update({"traffic": dram_traffic(kernel, workload), "ms_per_launch": ms, "timed": timed})
+    return r
+
+
+def measure_workload(cfg, inp, steps, warmup, peaks, world=1, dist=None, clock_index=0, sample_clocks=True):
+    """Times one workload on the current device: K passes back to back (the metric), single-pass
+    latency, the LM head and the attention in situ, and the pass through the host-buffer entry point.
+    Returns a dict; `total_ms` and `e2e_ms` are this rank's (the caller takes the maximum over ranks)."""
+    import numpy as np
+    import torch
+    from paper_2601_23180_b200 import binding as ts
+    from paper_2601_23180_b200 import runner
+    pas = runner.VerifyPass(cfg, inp)
+    pas.prepare_host(inp)
+    stream = torch.cuda.current_stream()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        pas.run()
+    sync_all()
+    assert int(pas.status.item()) == 0, "a device-side wait timed out"
+
+    # ---- device-resident timing: K passes, CUDA events on the launching stream
+    sampler = ClockSampler(clock_index)
+    if sample_clocks:
+        sampler.start()
+    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = ts.launch_count()
+    sync_all()
+    t_host0 = time.perf_counter()
+    e_start.record(stream)
+    for _ in range(steps):
+        pas.run()
+    e_end.record(stream)
+    host_us_per_call = (time.perf_counter() - t_host0) / steps * 1e6   # launch cost, GPU running behind
+    sync_all()
+    launches = ts.launch_count() - n0
+    total_ms = e_start.elapsed_time(e_end)      # K passes back to back, one bracket
+    # latency of a single pass (each bracketed by its own events; clocks recover between them)
+    n_lat = min(steps, 100)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
+    for s_, e_ in ev:
+        s_.record(stream)
+        pas.run()
+        e_.record(stream)
+    torch.cuda.synchronize()
+    pass_latency_ms = statistics.median(s_.elapsed_time(e_) for s_, e_ in ev)
+
+    # ---- per-step breakdown, measured in situ with the launch queue kept full:
+    #   lmhead    = K back-to-back calls of trispec_lmhead_stats (W, 0.6 GB or more, evicts itself from L2)
+    #   attention = event-bracketed attention calls, each preceded by an LM-head call (W streaming
+    #               flushes the KV cache from L2, as in the real pass); the marginal cost
+    #               (K full passes) - (K passes without attention) is reported beside it
+    def timed_loop(fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    def bracketed(fn, before):
+        """Mean device time of `fn` alone, each call preceded (untimed) by `before`, which streams the
+        LM-head weights through L2 exactly as the full pass does, so the timed call sees the cache
+        state it has inside a pass."""
+        n = min(steps, 200)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for s_, e_ in evs:
+            before()
+            s_.record(stream)
+            fn()
+            e_.record(stream)
+        torch.cuda.synchronize()
+        return sum(s_.elapsed_time(e_) for s_, e_ in evs) / n
+
+    lm_call = lambda: ts.trispec_lmhead_stats(pas.lm_args)
+    attn_call = lambda: ts.trispec_verify_attn(pas.attn_args)
+    ms_lmhead = timed_loop(lm_call)
+    ms_full = timed_loop(pas.run)
+    ms_no_attn = timed_loop(lambda: ts.trispec_verify(pas.tree_args, None, pas.lm_args, pas.scan_args))
+    ms_attn = bracketed(attn_call, lm_call)
+    ms_lmhead_single = bracketed(lm_call, attn_call)
+    part_ms = {"lmhead": ms_lmhead, "lmhead_single_call": ms_lmhead_single, "attention": ms_attn,
+               "attention_marginal_in_pass": ms_full - ms_no_attn,
+               "tree_mask_and_scan": max(ms_no_attn - ms_lmhead, 0.0), "full_pass_back_to_back": ms_full}
+
+    # ---- end to end through the host-buffer entry point: H2D inputs + pass + D2H results per step
+    for _ in range(3):
+        pas.run_host()
+    sync_all()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        pas.run_host()
+        torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    clocks = sampler.stop() if sample_clocks else None
+    assert int(pas.status.item()) == 0, "a device-side wait timed out"
+
+    n_seq = cfg.B if cfg.n_active is None else cfg.n_active
+    M = n_seq * cfg.T
+    lm_flops = 2.0 * M * cfg.d * cfg.V
+    lm_bytes = 2.0 * cfg.V * cfg.d + 2.0 * M * cfg.d + 40.0 * M
+    lm_kernel = "lmhead_rows_kernel" if n_seq == 1 else "lmhead_gemm_kernel"
+    lm_roof = _roofline("lmhead", peaks, lm_flops, lm_bytes, ms_lmhead, ms_lmhead * steps, lm_kernel, cfg.name,
+                        "trispec_lmhead_stats back to back (GEMM + finalize kernel; CUDA events on the stream)")
+    Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
+    attn_bytes = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 2 * 2 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
+    attn_flops = 4.0 * cfg.T * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
+    attn_roof = _roofline("attention", peaks, attn_flops, attn_bytes, ms_attn, 0.0, "verify_attn_split_kernel",
+                          cfg.name, "trispec_verify_attn bracketed by CUDA events right after an LM-head call "
+                          "(the cache state it meets inside a pass)")
+    out = {"total_ms": total_ms, "e2e_ms": e2e_ms, "launches": launches, "host_us_per_call": host_us_per_call,
+           "pass_latency_ms_median": pass_latency_ms, "kernels_ms": part_ms, "clocks": clocks,
+           "roofline": lm_roof, "attention_roofline": attn_roof, "h2d_bytes": pas.h2d_bytes,
+           "d2h_bytes": pas.d2h_bytes}
+    del pas
+    torch.cuda.empty_cache()
+    return out
+
+
 # ---------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="proxy_tree")
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="long_paged",
+                    help="the workload of the headline figures (default: the largest single-GPU configuration)")
     ap.add_argument("--impl", default="trispec", choices=["trispec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the per_workload block (the other four configurations)")
     ap.add_argument("--only", default=None, choices=["attention", "lmhead", "scan", "prune", "commit", "sample"],
                     help="time one entry point alone (L2 flushed before each call) instead of the pass")
     ap.add_argument("--tree-nodes", type=int, default=None,
@@ -488,7 +660,6 @@ def main():
             run_only(args, cfg)
         return
 
-    import numpy as np
     import torch
     import torch.distributed as dist
     if not torch.cuda.is_available():
@@ -501,106 +672,15 @@ def main():
         tbuild.build()
     if world > 1:
         dist.barrier()
-    from paper_2601_23180_b200 import binding as ts
-    from paper_2601_23180_b200 import runner
+    peaks = _peaks()
 
-    # every rank verifies its own batch of the same shape (seed offset by rank)
+    # every rank verifies its own batch of the same shape (seed offset by rank); the inputs are
+    # generated once, before anything is timed
     rcfg = rank_config(cfg, rank)
     inp = gen.make_inputs(rcfg)
-    pas = runner.VerifyPass(rcfg, inp)
-    pas.prepare_host(inp)
-    stream = torch.cuda.current_stream()
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
-        pas.run()
-    sync_all()
-    assert int(pas.status.item()) == 0, "a device-side wait timed out"
-
-    # ---- device-resident timing: K passes, CUDA events on the launching stream
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n0 = ts.launch_count()
-    sync_all()
-    t_host0 = time.perf_counter()
-    e_start.record(stream)
-    for _ in range(args.steps):
-        pas.run()
-    e_end.record(stream)
-    host_us_per_call = (time.perf_counter() - t_host0) / args.steps * 1e6   # launch cost, GPU running behind
-    sync_all()
-    launches = ts.launch_count() - n0
-    total_ms = e_start.elapsed_time(e_end)      # K passes back to back, one bracket
-    # latency of a single pass (each bracketed by its own events; clocks recover between them)
-    n_lat = min(args.steps, 100)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
-    for s_, e_ in ev:
-        s_.record(stream)
-        pas.run()
-        e_.record(stream)
-    torch.cuda.synchronize()
-    pass_latency_ms = statistics.median(s_.elapsed_time(e_) for s_, e_ in ev)
-
-    # ---- per-step breakdown, measured in situ with the launch queue kept full:
-    #   lmhead    = K back-to-back calls of trispec_lmhead_stats (W, 0.6 GB, evicts itself from L2)
-    #   attention = event-bracketed attention calls, each preceded by an LM-head call (W streaming
-    #               flushes the KV cache from L2, as in the real pass); the marginal cost
-    #               (K full passes) - (K passes without attention) is reported beside it
-    def timed_loop(fn):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for _ in range(3):
-            fn()
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(args.steps):
-            fn()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / args.steps
-
-    def bracketed(fn, before):
-        """Mean device time of `fn` alone, each call preceded (untimed) by `before`, which
-        streams the 0.6 GB of LM-head weights through L2 exactly as the full pass does, so the
-        timed call sees the cache state it has inside a pass."""
-        n = min(args.steps, 200)
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
-        for s_, e_ in evs:
-            before()
-            s_.record(stream)
-            fn()
-            e_.record(stream)
-        torch.cuda.synchronize()
-        return sum(s_.elapsed_time(e_) for s_, e_ in evs) / n
-
-    lm_call = lambda: ts.trispec_lmhead_stats(pas.lm_args)
-    ms_lmhead = timed_loop(lm_call)
-    ms_full = timed_loop(pas.run)
-    ms_no_attn = timed_loop(lambda: ts.trispec_verify(pas.tree_args, None, pas.lm_args, pas.scan_args))
-    ms_attn = bracketed(lambda: ts.trispec_verify_attn(pas.attn_args), lm_call)
-    ms_lmhead_single = bracketed(lm_call, lambda: ts.trispec_verify_attn(pas.attn_args))
-    part_ms = {"lmhead": ms_lmhead, "lmhead_single_call": ms_lmhead_single, "attention": ms_attn,
-               "attention_marginal_in_pass": ms_full - ms_no_attn,
-               "tree_mask_and_scan": max(ms_no_attn - ms_lmhead, 0.0), "full_pass_back_to_back": ms_full}
-
-    # ---- end to end through the host-buffer entry point: H2D inputs + pass + D2H results per step
-    for _ in range(3):
-        pas.run_host()
-    sync_all()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        pas.run_host()
-        torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    clocks = sampler.stop() if rank == 0 else None
-
-    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_s * 1e3], world, device="cuda")
+    m = measure_workload(rcfg, inp, args.steps, args.warmup, peaks, world=world, dist=dist, clock_index=local_rank,
+                         sample_clocks=(rank == 0))
+    total_ms, e2e_ms = max_over_ranks([m["total_ms"], m["e2e_ms"]], world, device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -608,54 +688,47 @@ def main():
 
     tokens = cfg_tokens(cfg) * world
     ms_per_step = total_ms / args.steps
-    value = aggregate_throughput(cfg, world, ms_per_step)
-    peaks = _peaks()
-    n_seq = cfg.B if cfg.n_active is None else cfg.n_active
-    M = n_seq * cfg.T
-    lm_flops = 2.0 * M * cfg.d * cfg.V
-    lm_bytes = 2.0 * cfg.V * cfg.d + 2.0 * M * cfg.d + 40.0 * M
-    lm_tflops = lm_flops / (part_ms["lmhead"] * 1e-3) / 1e12
-    lm_gbs = lm_bytes / (part_ms["lmhead"] * 1e-3) / 1e9
-    # the back-to-back loop is a sustained run when it lasts long enough for the power cap to bite
-    sustained = peaks.get("bf16_tflops_sustained") and part_ms["lmhead"] * args.steps >= 200.0
-    tc_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-    lm_tensor_bound = lm_flops / (tc_peak * 1e12) >= lm_bytes / (peaks["hbm_gbs"] * 1e9)
-    if lm_tensor_bound:
-        roof = {"kernel": "lmhead_gemm_kernel", "bound": "tensor", "achieved": lm_tflops, "peak": tc_peak,
-                "unit": "TFLOP/s", "frac": lm_tflops / tc_peak,
-                "peak_source": f"{peaks['source']} {'sustained' if sustained else 'burst'} bf16 GEMM",
-                "frac_of_burst_peak": lm_tflops / peaks["bf16_tflops"],
-                "work_per_launch": lm_flops}
-    else:
-        roof = {"kernel": "lmhead_gemm_kernel", "bound": "hbm", "achieved": lm_gbs, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": lm_gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['source']} copy bandwidth",
-                "work_per_launch": lm_bytes}
-    roof.update({"traffic": LMHEAD_GEMM_DRAM_TRAFFIC.get(cfg.name), "ms_per_launch": part_ms["lmhead"],
-                 "timed": "trispec_lmhead_stats back to back (GEMM + finalize kernel; CUDA events on the stream)"})
-    Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
-    attn_bytes = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 2 * 2 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
-    attn_gbs = attn_bytes / (part_ms["attention"] * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "active_sequences": n_seq, "draft_tokens": cfg.k,
-                   "tree_nodes": cfg.T, "context": cfg.L, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "head_dim": cfg.D,
-                   "hidden": cfg.d, "vocab": cfg.V, "kv": "paged" if cfg.paged else "contiguous",
-                   "l2": "inputs larger than L2 (LM-head weights + KV cache are streamed every pass)",
-                   "parallelism": "independent replicas, one batch per GPU"},
+        "metric": METRIC, "value": aggregate_throughput(cfg, world, ms_per_step), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": config_dict(cfg),
         "e2e": {"value": tokens / (e2e_ms * 1e-3 / args.steps), "unit": UNIT,
-                "h2d_bytes_per_step": pas.h2d_bytes, "d2h_bytes_per_step": pas.d2h_bytes},
-        "gpu_launches": launches, "host_us_per_call": host_us_per_call, "pass_latency_ms_median": pass_latency_ms,
-        "clocks": clocks,
-        "roofline": roof,
-        "kernels_ms": part_ms,
-        "attention_roofline": {"bound": "hbm", "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": attn_gbs / peaks["hbm_gbs"], "bytes_per_launch": attn_bytes},
+                "h2d_bytes_per_step": m["h2d_bytes"], "d2h_bytes_per_step": m["d2h_bytes"]},
+        "gpu_launches": m["launches"], "host_us_per_call": m["host_us_per_call"],
+        "pass_latency_ms_median": m["pass_latency_ms_median"], "clocks": m["clocks"],
+        "roofline": m["roofline"], "kernels_ms": m["kernels_ms"], "attention_roofline": m["attention_roofline"],
     }
     if not args.no_cpu_baseline and world == 1:
         v, desc, threads = oracle_timed(cfg, inp, budget_s=20.0)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle (numpy/BLAS)",
+                                "sample": desc}
+    del inp
+
+    # ---- the other configurations, same measurements with fewer steps (one GPU only: with N > 1 all
+    # GPUs would be held meanwhile)
+    if world == 1 and not args.no_per_workload and args.batch is None:
+        per = {}
+        n_steps = min(args.steps, 200)
+        for name in gen.CONFIG_ORDER:
+            if name == cfg.name:
+                mm, k_steps = m, args.steps
+            else:
+                wcfg = gen.CONFIGS[name]
+                winp = gen.make_inputs(wcfg)
+                mm, k_steps = measure_workload(wcfg, winp, n_steps, args.warmup, peaks, clock_index=local_rank), n_steps
+                del winp
+            wc = gen.CONFIGS[name]
+            ms = mm["total_ms"] / k_steps
+            per[name] = {"config": config_dict(wc), "steps": k_steps, "pass_ms_back_to_back": ms,
+                         "pass_latency_ms_median": mm["pass_latency_ms_median"],
+                         "value": cfg_tokens(wc) / (ms * 1e-3),
+                         "e2e_value": cfg_tokens(wc) / (mm["e2e_ms"] * 1e-3 / k_steps),
+                         "lmhead_roofline": mm["roofline"], "attention_roofline": mm["attention_roofline"],
+                         "kernels_ms": mm["kernels_ms"], "gpu_launches": mm["launches"],
+                         "sm_mhz": None if mm["clocks"] is None else mm["clocks"]["sm_mhz"],
+                         "clock_reasons": None if mm["clocks"] is None else mm["clocks"]["reasons"]}
+        line["per_workload"] = per
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
