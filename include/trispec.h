@@ -201,9 +201,9 @@ int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream);
  *     the library image (every GPU that loads the library holds that much until the process
  *     exits). `workspace` and `workspace_bytes` of the argument struct are ignored; inputs
  *     and outputs are still the caller's. No device or host memory is allocated or freed.
- *       - Limit: trispec_lmhead_stats_workspace(a) <= TRISPEC_NOALLOC_SCRATCH_BYTES (1 MiB:
- *         up to 512 active sequences); beyond that the call returns TRISPEC_ERR_TOO_LARGE
- *         and launches nothing.
+ *       - Limit: up to 512 active sequences (the partial statistics, planned for this entry
+ *         point so that they fit where they can, must not exceed TRISPEC_NOALLOC_SCRATCH_BYTES =
+ *         1 MiB); beyond that the call returns TRISPEC_ERR_TOO_LARGE and launches nothing.
  *       - The first call on each device looks up the device address of the array (one
  *         runtime call, with that device current); make that first call outside any stream
  *         capture. Later calls on the device reuse the address.

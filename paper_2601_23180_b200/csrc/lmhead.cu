@@ -58,10 +58,12 @@ struct LmParams {
   int T, d, V;
   int n_seq;      // active sequences
   int n_mt;       // M tiles of 4 sequence slots = ceil(n_seq / 4)
-  int n_ranges;   // vocabulary ranges
+  int n_ranges;   // vocabulary ranges of the main part: pair c < n_mt * n_ranges works on M tile c % n_mt, range c / n_mt
+  int n_tail;     // pairs beyond those: each sweeps ALL M tiles over its slice of the vocabulary's tail
+  int main_units; // 32-column units [0, main_units) belong to the main part, the rest to the tail
   float c;        // logit_scale * log2(e)
   const int32_t* seq_index;
-  LmPartial* partial;  // [n_ranges][n_mt * 256]
+  LmPartial* partial;  // [n_ranges + n_tail][n_mt * 256]
   int32_t* dev_status;
 };
 
@@ -71,21 +73,45 @@ struct LmParams {
 // and the MMA time does not shrink in proportion - so the rest is not spread over the tiles.)
 struct TileIter {
   int u0, units, n_tiles;
-  __device__ TileIter(int V, int n_ranges, int r) {
-    // Every range gets V32 / n_ranges units of 32 columns. What is left over goes to the first ranges in
-    // chunks that cost as few extra tiles as possible: a tile costs a whole k-loop whatever its width, so
-    // a chunk first fills up a range's last, partial tile (no extra tile), and where the ranges consist of
-    // whole tiles it is a whole tile (few ranges run one tile longer, instead of many).
-    const int V32 = (V + 31) >> 5;
-    const int base = V32 / n_ranges, rem = V32 - base * n_ranges;
+  // part r of n_parts of the 32-column units [first, first + count)
+  __device__ TileIter(int first, int count, int n_parts, int r) {
+    // Every part gets count / n_parts units. What is left over goes to the first parts in chunks that
+    // cost as few extra tiles as possible: a tile costs a whole k-loop whatever its width, so a chunk
+    // first fills up a part's last, partial tile (no extra tile), and where the parts consist of whole
+    // tiles it is a whole tile (few parts run one tile longer, instead of many).
+    const int base = count / n_parts, rem = count - base * n_parts;
     const int chunk = 8 - (base & 7);               // 1..8
-    u0 = r * base + min(rem, r * chunk);
+    u0 = first + r * base + min(rem, r * chunk);
     units = base + min(chunk, max(0, rem - r * chunk));
     n_tiles = (units + 7) >> 3;
   }
   __device__ void tile(int t, int& n0, int& nw) const {
     n0 = (u0 + 8 * t) << 5;
     nw = min(8, units - 8 * t) << 5;
+  }
+};
+
+// What a CTA pair works on. A main pair computes one M tile over one vocabulary range (one sweep). When
+// the M tiles do not divide the pairs of the chip, the pairs left over take the tail of the vocabulary:
+// each of them sweeps all M tiles, one after the other, over its own slice of that tail, which is
+// short enough to stay in L2 between the sweeps; the main ranges shrink accordingly, so that every
+// pair of the chip runs about the same number of tiles.
+struct PairWork {
+  int n_sweeps, mt0, part;      // M tile of sweep s = mt0 + s; `part` = row block of the partial array
+  TileIter tiles;
+  __device__ PairWork(const LmParams& p, int pair)
+      : n_sweeps(1), mt0(0), part(0), tiles(0, 0, 1, 0) {
+    const int V32 = (p.V + 31) >> 5;
+    const int n_main = p.n_mt * p.n_ranges;
+    if (pair < n_main) {
+      mt0 = pair % p.n_mt;
+      part = pair / p.n_mt;
+      tiles = TileIter(0, p.main_units, p.n_ranges, part);
+    } else {
+      n_sweeps = p.n_mt;
+      part = p.n_ranges + (pair - n_main);
+      tiles = TileIter(p.main_units, V32 - p.main_units, p.n_tail, pair - n_main);
+    }
   }
 };
 
@@ -109,9 +135,8 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();        // 0 = leader
   const int pair = blockIdx.x >> 1;
-  const int mt = pair % p.n_mt;
-  const int range = pair / p.n_mt;
-  const TileIter tiles(p.V, p.n_ranges, range);
+  const PairWork work(p, pair);
+  const TileIter& tiles = work.tiles;
   const int n_kb = p.d / LM_BK;
 
   if (threadIdx.x == 0) {
@@ -135,14 +160,15 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
       // sequence slots of this CTA; a slot past the last active sequence re-reads the M tile's
       // first sequence (its rows are computed and never looked at), which keeps the byte count
       // of a stage the same in both CTAs
-      const int a_first = 4 * mt;
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int sweep = 0; sweep < work.n_sweeps; ++sweep) {
+      const int a_first = 4 * (work.mt0 + sweep);
       int a0 = a_first + 2 * static_cast<int>(rank), a1 = a0 + 1;
       if (a0 >= p.n_seq) a0 = a_first;
       if (a1 >= p.n_seq) a1 = a_first;
       const int s0 = p.seq_index ? __ldg(p.seq_index + a0) : a0;
       const int s1 = p.seq_index ? __ldg(p.seq_index + a1) : a1;
-      int stage = 0;
-      uint32_t phase = 0;
       for (int t = 0; t < tiles.n_tiles; ++t) {
         int n0, nw;
         tiles.tile(t, n0, nw);
@@ -163,17 +189,20 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
           if (++stage == LM_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      }   // sweeps
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA)
     if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      for (int t = 0; t < tiles.n_tiles; ++t) {
+      const int n_all = work.n_sweeps * tiles.n_tiles;      // the accumulator buffers alternate over all sweeps
+      for (int tt = 0; tt < n_all; ++tt) {
+        const int t = tt % tiles.n_tiles;
         int n0, nw;
         tiles.tile(t, n0, nw);
-        const int buf = t & 1;
-        mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
+        const int buf = tt & 1;
+        mbar_wait(tmem_empty + buf, ((tt >> 1) & 1u) ^ 1u, p.dev_status);
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * LM_BN);
         const uint32_t idesc = idesc_bf16(2 * LM_BM, nw, false, false);
@@ -198,15 +227,17 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
   } else {
     // ------------------------------------------------------------------ epilogue (warps 0-3)
     const int row = warp * 32 + lane;  // TMEM lane == row of this CTA's half of the M tile
-    float m = -INFINITY, s = 0.f, tz = 0.f, v1 = -INFINITY, v2 = -INFINITY;
-    int i1 = -1, i2 = -1;
     const float c = p.c;
     const uint32_t tmem_empty_leader = cluster_map(smem_u32(tmem_empty), 0);
+    for (int sweep = 0; sweep < work.n_sweeps; ++sweep) {
+    float m = -INFINITY, s = 0.f, tz = 0.f, v1 = -INFINITY, v2 = -INFINITY;
+    int i1 = -1, i2 = -1;
     for (int t = 0; t < tiles.n_tiles; ++t) {
       int n0, nw;
       tiles.tile(t, n0, nw);
-      const int buf = t & 1;
-      mbar_wait(tmem_full + buf, (t >> 1) & 1u, p.dev_status);
+      const int tt = sweep * tiles.n_tiles + t;
+      const int buf = tt & 1;
+      mbar_wait(tmem_full + buf, (tt >> 1) & 1u, p.dev_status);
       tc_fence_after();
       const int ncols = min(nw, p.V - n0);  // valid columns of this tile
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(warp * 32) << 16) + static_cast<uint32_t>(buf * LM_BN);
@@ -287,10 +318,11 @@ lmhead_gemm_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(tmem_empty_leader + static_cast<uint32_t>(buf) * 8u);
     }
-    pdl_wait();   // the partials of the previous pass may still be read until earlier kernels are done
+    if (sweep == 0) pdl_wait();   // the partials of the previous pass may still be read until earlier kernels are done
     LmPartial out;
     out.m = m; out.s = s; out.v1 = v1; out.v2 = v2; out.i1 = i1; out.i2 = i2; out.t = tz; out.pad = 0;
-    p.partial[static_cast<size_t>(range) * (p.n_mt * 2 * LM_BM) + (mt * 2 + rank) * LM_BM + row] = out;
+    p.partial[static_cast<size_t>(work.part) * (p.n_mt * 2 * LM_BM) + ((work.mt0 + sweep) * 2 + rank) * LM_BM + row] = out;
+    }   // sweeps
   }
 
   pdl_wait();
@@ -685,24 +717,64 @@ lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
 // per SM, LW_ROWS partial rows per range.
 static bool lm_rows_path(int n_seq) { return n_seq == 1; }
 
-static int lm_plan(const trispec_lmhead_args* a, int* n_seq, int* n_mt, int* n_ranges) {
+struct LmPlan {
+  int n_seq, n_mt;
+  int n_ranges;    // pair kernel: vocabulary ranges of the main part; single-sequence kernel: ranges (= CTAs)
+  int n_tail;      // pair kernel: pairs that sweep all M tiles over a slice of the vocabulary's tail
+  int main_units;  // 32-column units of the main part
+  size_t partial_rows() const { return static_cast<size_t>(n_ranges + n_tail) * n_mt * 2 * LM_BM; }
+};
+
+// `max_ws` bounds the partial array (the no-allocation entry point has a fixed one): tail pairs, which
+// cost n_mt x 256 partial rows each, are given up until it fits.
+static int lm_plan(const trispec_lmhead_args* a, LmPlan* pl, size_t max_ws = ~static_cast<size_t>(0)) {
   if (!a || a->B <= 0 || a->T <= 0 || a->d <= 0 || a->V <= 0) return TRISPEC_ERR_INVALID_ARG;
   if (a->T > 64 || (a->d % LM_BK) != 0 || a->V < 2) return TRISPEC_ERR_UNSUPPORTED;
-  *n_seq = a->seq_index ? a->B_active : a->B;
-  if (*n_seq <= 0 || *n_seq > a->B) return TRISPEC_ERR_INVALID_ARG;
-  if (lm_rows_path(*n_seq)) {
-    *n_mt = 1;
+  pl->n_seq = a->seq_index ? a->B_active : a->B;
+  if (pl->n_seq <= 0 || pl->n_seq > a->B) return TRISPEC_ERR_INVALID_ARG;
+  pl->n_tail = 0;
+  pl->main_units = (a->V + 31) / 32;
+  if (lm_rows_path(pl->n_seq)) {
+    pl->n_mt = 1;
     const int V16 = (a->V + 15) / 16;
-    *n_ranges = device_sm_count() < V16 ? device_sm_count() : V16;
+    pl->n_ranges = device_sm_count() < V16 ? device_sm_count() : V16;
     return TRISPEC_OK;
   }
-  *n_mt = (*n_seq + 3) / 4;
+  pl->n_mt = (pl->n_seq + 3) / 4;
   const int pairs = device_sm_count() / 2;       // one CTA pair per two SMs
-  int r = pairs / *n_mt;
+  int r = pairs / pl->n_mt;
   if (r < 1) r = 1;
   const int V32 = (a->V + 31) / 32;
   if (r > V32) r = V32;
-  *n_ranges = r;
+  pl->n_ranges = r;
+  // Pairs that the M tiles leave over (74 = 16 x 4 + 10 for 64 sequences) take the tail of the vocabulary,
+  // every one of them for all M tiles in turn. Balance in whole tiles (a tile costs a k-loop whatever its
+  // width): a main pair runs ceil(main_units / r / 8) tiles, a tail pair n_mt x ceil(slice / 8).
+  int tail = pairs - pl->n_mt * r;
+  if (pl->n_mt < 2 || tail < 1 || pl->n_mt * r > pairs) tail = 0;
+  while (tail > 0 && static_cast<size_t>(r + tail) * pl->n_mt * 2 * LM_BM * sizeof(LmPartial) > max_ws) --tail;
+  if (tail > 0) {
+    int best_slice = 0, best_cost = (V32 / r + 7) / 8 + 1;    // without a tail: the longest main range
+    {
+      const int base = V32 / r, rem = V32 - base * r;
+      best_cost = (base + (rem ? ((8 - (base & 7)) < rem ? (8 - (base & 7)) : rem) : 0) + 7) / 8;
+    }
+    const int ideal = static_cast<int>((static_cast<long long>(V32) * tail) / (static_cast<long long>(pl->n_mt) * r + tail) / tail);
+    for (int slice = (ideal / 8 > 1 ? ideal / 8 - 1 : 1) * 8; slice <= (ideal / 8 + 2) * 8; slice += 8) {
+      const int main_u = V32 - slice * tail;
+      if (main_u < r) break;
+      const int base = main_u / r, rem = main_u - base * r;
+      const int chunk = 8 - (base & 7);
+      const int longest = base + (rem ? (chunk < rem ? chunk : rem) : 0);
+      const int main_tiles = (longest + 7) / 8, tail_tiles = pl->n_mt * (slice / 8);
+      const int cost = main_tiles > tail_tiles ? main_tiles : tail_tiles;
+      if (cost < best_cost) { best_cost = cost; best_slice = slice; }
+    }
+    if (best_slice > 0) {
+      pl->n_tail = tail;
+      pl->main_units = V32 - best_slice * tail;
+    }
+  }
   return TRISPEC_OK;
 }
 
@@ -710,18 +782,28 @@ static int lm_plan(const trispec_lmhead_args* a, int* n_seq, int* n_mt, int* n_r
 
 extern "C" size_t trispec_lmhead_stats_workspace(const trispec_lmhead_args* a) {
   using namespace trispec;
-  int n_seq, n_mt, n_ranges;
-  if (lm_plan(a, &n_seq, &n_mt, &n_ranges) != TRISPEC_OK) return 0;
-  if (lm_rows_path(n_seq)) return static_cast<size_t>(n_ranges) * LW_ROWS * sizeof(LmPartial);
-  return static_cast<size_t>(n_ranges) * n_mt * 2 * LM_BM * sizeof(LmPartial);
+  LmPlan pl;
+  if (lm_plan(a, &pl) != TRISPEC_OK) return 0;
+  if (lm_rows_path(pl.n_seq)) return static_cast<size_t>(pl.n_ranges) * LW_ROWS * sizeof(LmPartial);
+  return pl.partial_rows() * sizeof(LmPartial);
+}
+
+namespace trispec {
+static int lmhead_stats_planned(const trispec_lmhead_args* a, const LmPlan& pl, size_t ws_needed, void* stream);
 }
 
 extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) {
   trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
-  int n_seq, n_mt, n_ranges;
-  int rc = lm_plan(a, &n_seq, &n_mt, &n_ranges);
+  LmPlan pl;
+  int rc = lm_plan(a, &pl);
   if (rc != TRISPEC_OK) return rc;
+  return lmhead_stats_planned(a, pl, trispec_lmhead_stats_workspace(a), stream);
+}
+
+static int trispec::lmhead_stats_planned(const trispec_lmhead_args* a, const LmPlan& pl, size_t ws_needed, void* stream) {
+  const int n_seq = pl.n_seq, n_mt = pl.n_mt, n_ranges = pl.n_ranges;
+  int rc = TRISPEC_OK;
   if (!a->h || !a->W || !a->parent || !a->tok || !a->workspace) return TRISPEC_ERR_INVALID_ARG;
   if (!aligned16(a->h) || !aligned16(a->W) || (reinterpret_cast<uintptr_t>(a->workspace) & 255u))
     return TRISPEC_ERR_INVALID_ARG;
@@ -730,7 +812,7 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   if (!o.max || !o.lse || !o.top1_val || !o.top2_val || !o.p_top1 || !o.p_top2 || !o.top1_idx || !o.top2_idx ||
       !o.draft_logit || !o.p_draft)
     return TRISPEC_ERR_INVALID_ARG;
-  if (a->workspace_bytes < trispec_lmhead_stats_workspace(a)) return TRISPEC_ERR_WORKSPACE;
+  if (a->workspace_bytes < ws_needed) return TRISPEC_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
   CUtensorMap tm_h, tm_w;
@@ -749,7 +831,7 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   // the entropy sum costs two more instructions per logit: only computed when it is asked for
   const bool want_entropy = a->out.entropy != nullptr;
   LmFinalizeParams f;
-  f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges;
+  f.T = a->T; f.d = a->d; f.V = a->V; f.n_mt = n_mt; f.n_ranges = n_ranges + pl.n_tail;
   f.scale = a->logit_scale; f.c = a->logit_scale * kLog2e;
   f.seq_index = a->seq_index;
   f.partial = static_cast<LmPartial*>(a->workspace);
@@ -761,6 +843,7 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
     LmRowsParams sp;
     sp.base.T = a->T; sp.base.d = a->d; sp.base.V = a->V;
     sp.base.n_seq = 1; sp.base.n_mt = 1; sp.base.n_ranges = n_ranges;
+    sp.base.n_tail = 0; sp.base.main_units = pl.main_units;
     sp.base.c = f.c;
     sp.base.seq_index = a->seq_index;
     sp.base.partial = static_cast<LmPartial*>(a->workspace);
@@ -805,15 +888,16 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   LmParams p;
   p.T = a->T; p.d = a->d; p.V = a->V;
   p.n_seq = n_seq; p.n_mt = n_mt; p.n_ranges = n_ranges;
+  p.n_tail = pl.n_tail; p.main_units = pl.main_units;
   p.c = a->logit_scale * kLog2e;
   p.seq_index = a->seq_index;
   p.partial = static_cast<LmPartial*>(a->workspace);
   p.dev_status = a->dev_status;
   if (want_entropy) {
-    TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel<true>, static_cast<unsigned>(2 * n_mt * n_ranges), LM_THREADS,
+    TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel<true>, static_cast<unsigned>(2 * (n_mt * n_ranges + pl.n_tail)), LM_THREADS,
                                      LM_SMEM_BYTES, st, 2, tm_h, tm_w, p));
   } else {
-    TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel<false>, static_cast<unsigned>(2 * n_mt * n_ranges), LM_THREADS,
+    TRISPEC_CUDA_OK(launch_dependent(lmhead_gemm_kernel<false>, static_cast<unsigned>(2 * (n_mt * n_ranges + pl.n_tail)), LM_THREADS,
                                      LM_SMEM_BYTES, st, 2, tm_h, tm_w, p));
   }
   count_launch();
@@ -857,15 +941,18 @@ static int lm_noalloc_scratch(void** out) {
 extern "C" int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream) {
   trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;
-  int n_seq, n_mt, n_ranges;
-  int rc = lm_plan(a, &n_seq, &n_mt, &n_ranges);
+  // planned so that the partial array fits the built-in scratch (fewer tail pairs where they would not)
+  LmPlan pl;
+  int rc = lm_plan(a, &pl, TRISPEC_NOALLOC_SCRATCH_BYTES);
   if (rc != TRISPEC_OK) return rc;
-  if (trispec_lmhead_stats_workspace(a) > TRISPEC_NOALLOC_SCRATCH_BYTES) return TRISPEC_ERR_TOO_LARGE;
+  const size_t need = lm_rows_path(pl.n_seq) ? static_cast<size_t>(pl.n_ranges) * LW_ROWS * sizeof(LmPartial)
+                                             : pl.partial_rows() * sizeof(LmPartial);
+  if (need > TRISPEC_NOALLOC_SCRATCH_BYTES) return TRISPEC_ERR_TOO_LARGE;
   void* scratch = nullptr;
   rc = lm_noalloc_scratch(&scratch);
   if (rc != TRISPEC_OK) return rc;
   trispec_lmhead_args b = *a;     // same call, with the built-in array as its workspace
   b.workspace = scratch;
   b.workspace_bytes = TRISPEC_NOALLOC_SCRATCH_BYTES;
-  return trispec_lmhead_stats(&b, stream);
+  return lmhead_stats_planned(&b, pl, need, stream);
 }

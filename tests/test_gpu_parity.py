@@ -131,6 +131,10 @@ LM_CASES = [
     ("proxy_tree", dict(B=5, V=151936 // 8, d=192, logit_scale=3.6 / (0.02 * math.sqrt(192)))),
     ("target_escalated", dict(B=7, n_active=3, V=9000, d=320, logit_scale=3.6 / (0.02 * math.sqrt(320)))),
     ("llama_tree", dict(B=2, V=128256 // 4, d=1024, logit_scale=3.6 / (0.02 * 32.0))),
+    # M tiles that do not divide the chip's CTA pairs: the pairs left over sweep all M tiles over a tail of the vocabulary
+    ("proxy_tree", dict(B=20, V=40011, d=256)),                                  # 5 M tiles: 14 ranges + 4 tail pairs
+    ("llama_tree", dict(B=31, V=21000, d=128)),                                  # 8 M tiles (the last one ragged): 9 + 2
+    ("target_escalated", dict(B=40, n_active=37, V=3000, d=64)),                 # 10 M tiles picked by seq_index: 7 + 4
     # one active sequence: the kernel with W on the M side and the tree's nodes as columns
     ("proxy_tree", dict(B=1, V=40011, d=512)),                                   # 61 nodes: two column chunks
     ("llama_tree", dict(B=1, V=9000, d=256)),                                    # 49 nodes

@@ -41,7 +41,11 @@ def test_lmhead_workspace_shows_the_kernel_choice():
         return a
     # batches: CTA pairs, 74 // n_mt vocabulary ranges x n_mt M tiles x 256 rows x 32 bytes
     assert ts.trispec_lmhead_stats_workspace(args(8, 61, 2048, 151936)) == 37 * 2 * 256 * 32
-    assert ts.trispec_lmhead_stats_workspace(args(64, 61, 2048, 151936)) == 4 * 16 * 256 * 32
+    # 16 M tiles leave 10 of the 74 pairs over: they become tail pairs (one more block of partial rows each)
+    assert ts.trispec_lmhead_stats_workspace(args(64, 61, 2048, 151936)) == (4 + 10) * 16 * 256 * 32
+    assert ts.trispec_lmhead_stats_workspace(args(32, 61, 2048, 151936)) == (9 + 2) * 8 * 256 * 32
+    # no tail where it would not shorten the longest pair (llama_tree: 28 tiles either way)
+    assert ts.trispec_lmhead_stats_workspace(args(16, 49, 4096, 128256)) == 18 * 4 * 256 * 32
     # one active sequence: one range per SM x 64 rows x 32 bytes
     assert ts.trispec_lmhead_stats_workspace(args(1, 9, 2048, 32000)) == 148 * 64 * 32
     assert ts.trispec_lmhead_stats_workspace(args(8, 61, 5120, 151936, n_active=1)) == 148 * 64 * 32

@@ -5,7 +5,7 @@ memory pool already owns all free device memory: there a cudaMalloc fails, or st
 stream while it runs, so the loop has no way to obtain the workspace that
 `trispec_lmhead_stats` asks for. The variant keeps its partial statistics in a fixed 1 MiB
 array inside the library instead. This file checks, through the C ABI, that it returns what
-the workspace entry point returns and what the CPU oracle computes, on two calls in a row with different inputs (the array
+the workspace entry point returns and what the CPU oracle computes, on calls in a row with different inputs (the array
 is shared and keeps the previous call's contents, which must not leak into the next result),
 and that a problem too large for the array is refused before anything is launched.
 
@@ -27,7 +27,6 @@ def _run(ts, torch, dev, cfg, noalloc: bool):
     a = ts.lmhead_args(dev["h"], dev["W"], dev["parent"], dev["tok"], cfg.logit_scale, st,
                        seq_index=dev.get("seq_index"), dev_status=status)
     if noalloc:
-        assert ts.trispec_lmhead_stats_workspace(a) <= ts.NOALLOC_SCRATCH_BYTES
         ts.trispec_lmhead_stats_noalloc(a)                 # no workspace in the arguments
     else:
         ws = ts.alloc_workspace(ts.trispec_lmhead_stats_workspace(a))
@@ -60,6 +59,9 @@ def test_noalloc_entry_matches_workspace_entry_twice_in_a_row():
         # second call: other shapes, a sequence subset and another seed, so that anything left
         # in the shared array by the first call would show
         gen.small_variant(gen.CONFIGS["target_escalated"], B=6, n_active=3, L=64, V=9000, d=320, Hq=32, seed=7),
+        # 64 sequences: the workspace entry point would plan more partial rows than the built-in array
+        # holds (pairs that sweep every M tile); this entry point plans fewer of them and must still agree
+        gen.small_variant(gen.CONFIGS["proxy_tree"], B=64, L=64, V=6000, d=64, logit_scale=3.6 / (0.02 * 8.0), seed=9),
     ]
     for cfg in cases:
         inp = gen.make_inputs(cfg)
