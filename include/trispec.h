@@ -244,7 +244,8 @@ int trispec_lmhead_stats_noalloc(const trispec_lmhead_args* a, void* stream);
  *      being the margin, p_top1 or the entropy as `criterion` selects;
  *      n_escalated int32 [1]; esc_index int32 [B] ascending ids of escalated sequences,
  *      -1 padded. near_thr, n_escalated and esc_index may be NULL (n_escalated and esc_index
- *      only together).
+ *      only together). compact_scratch (optional) only changes how fast esc_index is built for
+ *      very large batches, never its contents.
  * ------------------------------------------------------------------------------------- */
 typedef struct {
   int B, T;
@@ -260,6 +261,8 @@ typedef struct {
   float alpha;                      /* slack of the token-specific rule; ignored by the other rules */
   int32_t *accept_len, *bonus_tok, *path, *last_node, *near_thr, *n_escalated, *esc_index;
   uint8_t* escalate;
+  int32_t* compact_scratch;         /* optional, int32 [ceil(B / 65536)], contents undefined: lets batches above
+                                       65536 sequences build esc_index with one block per 65536 flags */
 } trispec_scan_args;
 int trispec_accept_scan(const trispec_scan_args* a, void* stream);
 

@@ -59,7 +59,7 @@ class ScanArgs(C.Structure):
                 ("stats", Stats), ("active", _vp), ("start_node", _vp), ("q_draft", _vp), ("u_accept", _vp),
                 ("accept_rule", _i), ("alpha", _f), ("accept_len", _vp),
                 ("bonus_tok", _vp), ("path", _vp), ("last_node", _vp), ("near_thr", _vp),
-                ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp)]
+                ("n_escalated", _vp), ("esc_index", _vp), ("escalate", _vp), ("compact_scratch", _vp)]
 
 
 class PruneArgs(C.Structure):
@@ -244,7 +244,8 @@ def scan_args(stats, parent, tok, lam, mode, out: Dict[str, torch.Tensor], activ
     a.active, a.start_node = _p(active), _p(start_node)
     a.q_draft, a.u_accept = _p(q_draft), _p(u_accept)
     a.accept_rule, a.alpha = int(accept_rule), float(alpha)
-    for k in ("accept_len", "bonus_tok", "path", "last_node", "near_thr", "n_escalated", "esc_index", "escalate"):
+    for k in ("accept_len", "bonus_tok", "path", "last_node", "near_thr", "n_escalated", "esc_index", "escalate",
+              "compact_scratch"):
         setattr(a, k, _p(out.get(k)))
     return _hold(a, stats, parent, tok, out, active, start_node, q_draft, u_accept)
 
@@ -291,6 +292,8 @@ def alloc_scan_out(B: int, T: int, device="cuda") -> Dict[str, torch.Tensor]:
     i32 = dict(dtype=torch.int32, device=device)
     out.update({"near_thr": torch.full((B,), -7, **i32), "n_escalated": torch.full((1,), -7, **i32),
                 "esc_index": torch.full((B,), -7, **i32)})
+    if B > 65536:     # scratch that lets the escalation list be built by one block per 65536 sequences
+        out["compact_scratch"] = torch.full(((B + 65535) // 65536,), -7, **i32)
     return out
 
 

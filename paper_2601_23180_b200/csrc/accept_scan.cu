@@ -6,7 +6,7 @@
 // of all nodes becomes two ballots, and the walk then runs on registers: the current node's
 // top-1 comes from a warp shuffle, the child match is a warp ballot. The accepted path is
 // collected in registers and stored as one row. The ordered list of escalated sequence ids is
-// made by the same block when the batch has at most 32 sequences, by a second kernel otherwise.
+// made by the same block when the batch has at most 32 sequences, by further kernels otherwise.
 #include "host_common.h"
 
 namespace trispec {
@@ -182,49 +182,102 @@ accept_scan_small_kernel(trispec_scan_args a) {
   }
 }
 
-// Ordered compaction of the escalated sequence ids by one block. Per round a warp owns 2048
-// consecutive flags: lane l reads the 4-byte words l, l + 32, ... of them (coalesced), the
-// block orders the warp totals with one barrier (double-buffered; the running total is carried
-// in registers), and each word column is scattered with a warp scan, so that a warp writes
-// consecutive entries of esc_index. Entries past the last escalated sequence were set to -1 by
-// the scan kernel. 65536 flags per round.
+// Ordered compaction of the escalated sequence ids. A block owns 65536 consecutive flags; inside it a
+// warp owns 2048 of them: lane l reads the 4-byte words l, l + 32, ... (coalesced), the block orders
+// the warp totals with one barrier, and each word column is scattered with a warp scan, so that a warp
+// writes consecutive entries of esc_index. Entries past the last escalated sequence were set to -1 by
+// the scan kernel. Batches of more than 65536 sequences take one block per 65536 flags in two
+// launches: the first leaves every block's count in a scratch array, the second starts each block at
+// the sum of the counts before it (a caller without scratch gets one block that walks all rounds).
 constexpr int kCompactThreads = 1024;
 constexpr int kCompactWords = 16;                       // 4-byte words per lane and round
 constexpr int kCompactPerWarp = 32 * kCompactWords * 4;  // flags per warp and round
+constexpr long long kCompactPerBlock = static_cast<long long>(kCompactThreads / 32) * kCompactPerWarp;   // 65536
+
+// flags of this warp's region as one bit per byte (0x01 per non-zero flag), and their count
+__device__ __forceinline__ int compact_load(const uint8_t* __restrict__ escalate, long long B, long long region,
+                                            bool word_ok, int lane, uint32_t (&w)[kCompactWords]) {
+  if (word_ok && region + kCompactPerWarp <= B) {
+    // whole region in range: sixteen independent coalesced loads in flight
+#pragma unroll
+    for (int j = 0; j < kCompactWords; ++j)
+      w[j] = __ldg(reinterpret_cast<const uint32_t*>(escalate + region) + j * 32 + lane);
+  } else {
+#pragma unroll
+    for (int j = 0; j < kCompactWords; ++j) {
+      const long long first = region + (j * 32 + lane) * 4;
+      uint32_t x = 0;
+      for (int k = 0; k < 4; ++k)
+        if (first + k < B) x |= static_cast<uint32_t>(escalate[first + k]) << (8 * k);
+      w[j] = x;
+    }
+  }
+  int cnt = 0;
+#pragma unroll
+  for (int j = 0; j < kCompactWords; ++j) {
+    w[j] = __vcmpne4(w[j], 0u) & 0x01010101u;        // one bit per non-zero flag byte
+    cnt += __popc(w[j]);
+  }
+  return cnt;
+}
+
+// first launch of the two-launch form: block_count[blk] = escalated sequences among the block's flags
 __global__ void __launch_bounds__(kCompactThreads)
-esc_compact_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restrict__ esc_index,
-                   int32_t* __restrict__ n_escalated) {
-  __shared__ int warp_total[2][32];
+esc_count_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restrict__ block_count) {
+  __shared__ int warp_total[32];
   pdl_launch_dependents();
   pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool word_ok = (reinterpret_cast<uintptr_t>(escalate) & 3u) == 0;
-  int running = 0;      // escalated sequences in earlier rounds (same value in every thread)
+  const long long region = blockIdx.x * kCompactPerBlock + static_cast<long long>(warp) * kCompactPerWarp;
+  uint32_t w[kCompactWords];
+  int cnt = compact_load(escalate, B, region, word_ok, lane, w);
+  for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) warp_total[warp] = cnt;
+  __syncthreads();
+  if (warp == 0) {
+    int t = warp_total[lane];
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (lane == 0) block_count[blockIdx.x] = t;
+  }
+}
+
+// One block per 65536 flags when block_count is given (gridDim.x blocks, each starting at the sum of
+// the counts of the blocks before it), else a single block that walks all rounds itself.
+__global__ void __launch_bounds__(kCompactThreads)
+esc_compact_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restrict__ esc_index,
+                   int32_t* __restrict__ n_escalated, const int32_t* __restrict__ block_count) {
+  __shared__ int warp_total[2][32];
+  __shared__ int s_start;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool word_ok = (reinterpret_cast<uintptr_t>(escalate) & 3u) == 0;
+  int running = 0;      // escalated sequences before the current round (same value in every thread)
+  long long start = 0, end = B;
+  if (block_count) {
+    // sum of the counts of the earlier blocks
+    int part = 0;
+    for (int j = tid; j < static_cast<int>(blockIdx.x); j += kCompactThreads) part += __ldg(block_count + j);
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    if (lane == 0) warp_total[0][warp] = part;
+    __syncthreads();
+    if (warp == 0) {
+      int t = warp_total[0][lane];
+      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+      if (lane == 0) s_start = t;
+    }
+    __syncthreads();
+    running = s_start;
+    start = blockIdx.x * kCompactPerBlock;
+    end = min(static_cast<long long>(B), start + kCompactPerBlock);
+    __syncthreads();                                   // warp_total is reused below
+  }
   int round = 0;
-  for (long long start = 0; start < B; start += static_cast<long long>(kCompactThreads / 32) * kCompactPerWarp, ++round) {
+  for (; start < end; start += kCompactPerBlock, ++round) {
     const long long region = start + static_cast<long long>(warp) * kCompactPerWarp;
     uint32_t w[kCompactWords];
-    int cnt = 0;
-    if (word_ok && region + kCompactPerWarp <= B) {
-      // whole region in range: sixteen independent coalesced loads in flight
-#pragma unroll
-      for (int j = 0; j < kCompactWords; ++j)
-        w[j] = __ldg(reinterpret_cast<const uint32_t*>(escalate + region) + j * 32 + lane);
-    } else {
-#pragma unroll
-      for (int j = 0; j < kCompactWords; ++j) {
-        const long long first = region + (j * 32 + lane) * 4;
-        uint32_t x = 0;
-        for (int k = 0; k < 4; ++k)
-          if (first + k < B) x |= static_cast<uint32_t>(escalate[first + k]) << (8 * k);
-        w[j] = x;
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < kCompactWords; ++j) {
-      w[j] = __vcmpne4(w[j], 0u) & 0x01010101u;        // one bit per non-zero flag byte
-      cnt += __popc(w[j]);
-    }
+    int cnt = compact_load(escalate, B, region, word_ok, lane, w);
     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);   // warp total
     if (lane == 0) warp_total[round & 1][warp] = cnt;
     __syncthreads();
@@ -258,7 +311,7 @@ esc_compact_kernel(const uint8_t* __restrict__ escalate, int B, int32_t* __restr
     }
   }
   // entries past the last escalated sequence already hold -1 (written by the scan kernel)
-  if (tid == 0) *n_escalated = running;
+  if (tid == 0 && (!block_count || blockIdx.x == gridDim.x - 1)) *n_escalated = running;
 }
 
 }  // namespace trispec
@@ -311,9 +364,21 @@ extern "C" int trispec_accept_scan(const trispec_scan_args* a, void* stream) {
   TRISPEC_CUDA_OK(launch_dependent(big_k[which], grid, kScanThreads, 0, st, 1, *a));
   count_launch();
   if (a->esc_index) {
-    TRISPEC_CUDA_OK(launch_dependent(esc_compact_kernel, 1, kCompactThreads, 0, st, 1,
-                                     static_cast<const uint8_t*>(a->escalate), a->B, a->esc_index, a->n_escalated));
-    count_launch();
+    const unsigned n_blk = static_cast<unsigned>((static_cast<long long>(a->B) + kCompactPerBlock - 1) / kCompactPerBlock);
+    if (a->compact_scratch && n_blk > 1) {
+      TRISPEC_CUDA_OK(launch_dependent(esc_count_kernel, n_blk, kCompactThreads, 0, st, 1,
+                                       static_cast<const uint8_t*>(a->escalate), a->B, a->compact_scratch));
+      count_launch();
+      TRISPEC_CUDA_OK(launch_dependent(esc_compact_kernel, n_blk, kCompactThreads, 0, st, 1,
+                                       static_cast<const uint8_t*>(a->escalate), a->B, a->esc_index, a->n_escalated,
+                                       static_cast<const int32_t*>(a->compact_scratch)));
+      count_launch();
+    } else {
+      TRISPEC_CUDA_OK(launch_dependent(esc_compact_kernel, 1, kCompactThreads, 0, st, 1,
+                                       static_cast<const uint8_t*>(a->escalate), a->B, a->esc_index, a->n_escalated,
+                                       static_cast<const int32_t*>(nullptr)));
+      count_launch();
+    }
   }
   return TRISPEC_OK;
 }

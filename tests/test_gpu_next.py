@@ -512,3 +512,53 @@ def test_host_pass_with_separately_allocated_host_buffers():
     assert int(pas.status.item()) == 0
     for k in ("accept_len", "bonus_tok", "last_node", "path", "escalate"):
         assert torch.equal(host[k], want[k].cpu()), k
+
+
+def test_escalation_list_of_a_very_large_batch():
+    """More than 65536 sequences: with the optional scratch the ordered list of escalated ids is built by
+    one block per 65536 flags (two launches), without it by one block; both must give the ascending ids
+    of the sequences the scan flagged, -1 beyond them, and the scan itself must match the oracle."""
+    import torch
+    import tests.gpu_helpers as H
+    from paper_2601_23180_b200 import binding as ts
+    cfg, parent64, tok64 = _trees("proxy_tree", 64, seed=21)
+    B, T = 3 * 65536 + 4321, cfg.T                      # four blocks, the last one ragged
+    reps = (B + 63) // 64
+    parent, tok = np.tile(parent64, (reps, 1))[:B], np.tile(tok64, (reps, 1))[:B]
+    g = np.random.default_rng(12)
+    first_child = np.full((64, T), -1)
+    for b in range(64):
+        for c in range(T - 1, 0, -1):
+            first_child[b, parent64[b, c]] = c
+    fc = np.tile(first_child, (reps, 1))[:B]
+    top1 = np.where(fc >= 0, np.take_along_axis(tok, np.maximum(fc, 0), axis=1), 7).astype(np.int64)
+    p1 = g.uniform(0.52, 1.0, size=(B, T)).astype(np.float32)
+    p1[g.uniform(size=(B, T)) < 0.1] = 0.3              # about a tenth of the nodes is untrusted
+    p1[1000:70000] = 0.9                                # a long stretch without any escalation
+    p2 = np.zeros((B, T), dtype=np.float32)
+    st = {"p_top1": torch.from_numpy(p1).cuda(), "p_top2": torch.from_numpy(p2).cuda(),
+          "top1_idx": H.i32_dev(top1)}
+    pd, td = H.i32_dev(parent), H.i32_dev(tok)
+    results = []
+    for with_scratch in (True, False):
+        out = ts.alloc_scan_out(B, T)
+        assert "compact_scratch" in out
+        if not with_scratch:
+            del out["compact_scratch"]
+        n0 = ts.launch_count()
+        ts.trispec_accept_scan(ts.scan_args(st, pd, td, 0.5, gen.MODE_PROXY, out))
+        torch.cuda.synchronize()
+        assert ts.launch_count() - n0 == (3 if with_scratch else 2)
+        got = {k: v.cpu().numpy() for k, v in out.items()}
+        esc = np.nonzero(got["escalate"])[0]
+        assert 1000 < len(esc) < B - 1000 and not ((esc >= 1000) & (esc < 70000)).any()
+        assert got["n_escalated"][0] == len(esc)
+        assert np.array_equal(got["esc_index"][:len(esc)], esc) and (got["esc_index"][len(esc):] == -1).all()
+        results.append(got)
+    for k in ("accept_len", "escalate", "bonus_tok", "last_node", "esc_index"):
+        assert np.array_equal(results[0][k], results[1][k]), k
+    # the walk itself against the oracle, on a sample that spans the block boundaries
+    pick = np.concatenate([np.arange(0, 40), np.arange(65536 - 20, 65536 + 20), np.arange(B - 40, B)])
+    ref = orc.accept_scan(p1[pick].astype(np.float64), p2[pick].astype(np.float64), top1[pick], parent[pick], tok[pick], 0.5)
+    for k in ("accept_len", "escalate", "bonus_tok", "last_node"):
+        assert np.array_equal(results[0][k][pick], ref[k]), k
