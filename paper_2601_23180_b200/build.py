@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libtrispec.so")
 STAMP = os.path.join(PKG, "csrc", ".build_stamp")
-SOURCES = ["host_common.cu", "tree_mask.cu", "accept_scan.cu", "lmhead.cu", "attn.cu", "verify.cu", "prune.cu",
+SOURCES = ["host_common.cu", "tree_mask.cu", "accept_scan.cu", "lmhead.cu", "attn.cu", "attn_pieces.cu", "verify.cu", "prune.cu",
            "kv_commit.cu", "sample.cu"]
 
 NVCC_FLAGS = [

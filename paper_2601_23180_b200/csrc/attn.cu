@@ -31,70 +31,11 @@
 // two P buffers (short loops: tile i waits for P V of tile i - 2 only).
 // A sequence may carry fewer than T tree nodes (a pruned tree): rows past its count are not
 // computed and M tiles past it do nothing.
-#include <math.h>
+#include <stdlib.h>
 
-#include "host_common.h"
-#include "sm100.cuh"
+#include "attn_common.cuh"
 
 namespace trispec {
-
-constexpr int AT_BM = 128;      // rows per M tile
-constexpr int AT_BN = 64;       // keys per tile (= paged block size)
-constexpr int AT_D = 128;
-constexpr int AT_STAGES = 3;        // K ring; the V ring has 3 slots with one P buffer, 2 with two
-constexpr int AT_BOX_BYTES = 64 * 64 * 2;               // 64 rows x 64 elements
-constexpr int AT_KV_STAGE_BYTES = 4 * AT_BOX_BYTES;     // one K slot + one V slot = 32 KB
-constexpr int AT_TILE_BYTES = 2 * AT_BOX_BYTES;         // a K tile or a V tile: 64 keys x 128 dims bf16 = 16 KB
-constexpr int AT_P_BYTES = AT_BM * AT_BN * 2;           // 16 KB
-constexpr int AT_THREADS = 192;
-constexpr int AT_SMEM_USED = AT_STAGES * AT_KV_STAGE_BYTES + AT_P_BYTES + 256;
-// two CTAs per SM: 2 x (dynamic + 1 KB reserved) must fit 228 KB, which leaves 768 bytes of alignment slack
-constexpr int AT_SMEM_BYTES = AT_SMEM_USED + 768;
-constexpr int AT_TMEM_COLS = 256;                        // Q [0,64) S [64,128) O [128,256)
-constexpr int AT_TM_Q = 0, AT_TM_S = 64, AT_TM_O = 128;
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;                // log2 units
-constexpr int AT_PART_PITCH = AT_D * 2 + 16;             // bytes per row of the in-smem partial (bf16, bank spread)
-constexpr int AT_PART_ML_OFF = AT_BM * AT_PART_PITCH;    // (m, l) pairs follow the partial rows
-constexpr int AT_PART_ML2_OFF = AT_PART_ML_OFF + AT_BM * 8;   // gathered (m, l) of every split for this CTA's rows
-constexpr int AT_PART_ML2_MAX = AT_BM + 2 * 8;                // n_splits x rows per CTA, rows rounded up to even
-static_assert(AT_PART_ML2_OFF + AT_PART_ML2_MAX * 8 <= (AT_STAGES + 2) * AT_TILE_BYTES,
-              "partial must fit in the K ring plus the shorter V ring");
-
-struct AttnParams {
-  int T, Hq, Hkv, G, NPT, n_mt, n_splits;
-  int paged, max_blocks_per_seq, num_blocks;
-  int Lcap;         // capacity of a sequence's context: Lmax, or 64 x max_blocks_per_seq
-  float scale_log2;
-  const uint16_t* q;
-  const int32_t *block_table, *ctx_len, *seq_index;
-  const int32_t* n_nodes;   // tree nodes per sequence (a pruned tree), or null = T
-  const uint64_t* mask;
-  float* part_o;    // [items][128][128]   (workspace mode only)
-  float* part_ml;   // [items][128][2]
-  uint16_t* o;      // bf16 [B][T][Hq][128]  (cluster mode writes the result itself)
-  float* lse;       // [B][Hq][T] or null
-  int32_t* dev_status;
-};
-
-__device__ __forceinline__ uint4 ld_cluster_u4(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared::cluster.v4.b32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
-  float2 v;
-  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
-  return v;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
 
 // NP = number of P buffers. With one, the softmax of tile i waits for O += P V of tile i - 1 before
 // it may overwrite P; with two (and a V ring of two slots instead of three, same shared memory) it
@@ -675,8 +616,20 @@ verify_attn_merge_kernel(const AttnMergeParams p) {
 struct AttnPlan {
   int n_seq, G, NPT, n_mt, tiles_max, n_splits;
   bool cluster;      // splits merged inside a thread-block cluster (no workspace)
+  bool pieces;       // persistent CTAs over balanced pieces of the work (attn_pieces.cu)
+  int n_cta;         // CTAs of the persistent launch
   size_t items;
 };
+
+// TRISPEC_ATTN_PLAN = "pieces" or "splits" overrides the planner's choice between the persistent kernel
+// and the split kernels where both apply (a tuning and testing aid; read at every call).
+static int attn_plan_override() {
+  const char* e = getenv("TRISPEC_ATTN_PLAN");
+  if (!e) return 0;
+  if (e[0] == 'p') return 1;
+  if (e[0] == 's') return 2;
+  return 0;
+}
 
 static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   if (!a || a->B <= 0 || a->T <= 0 || a->Hq <= 0 || a->Hkv <= 0) return TRISPEC_ERR_INVALID_ARG;
@@ -705,7 +658,7 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   // five workloads: more than about 1.25 waves of CTAs with at least 32 tiles each run best (the fixed
   // costs of a CTA - pipeline fill, Q load, merge - hide behind other CTAs); when tiles are too few
   // for that, one wave filled as far as possible; very few (sequence, head) pairs are cut further.
-  const long long slots = static_cast<long long>(device_sm_count()) * 2;   // two CTAs per SM
+  const long long slots = static_cast<long long>(device_sm_count()) * 2;   // two CTAs per SM (split kernels)
   const int tiles = pl->tiles_max;
   int best_s = 0;
   for (int sp = 1; sp <= 8 && !best_s; ++sp)
@@ -734,6 +687,27 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   }
   pl->items = static_cast<size_t>(fixed) * pl->n_splits;
   if (pl->items > 0x7fffffffull) return TRISPEC_ERR_UNSUPPORTED;
+  // The persistent kernel: every CTA slot of the chip gets the same number of tile steps whatever the
+  // shape. It pays where the split plan cannot fill the slots evenly: fewer CTAs than slots, a last
+  // wave that is mostly empty, or clusters that cannot be placed everywhere.
+  pl->pieces = false;
+  pl->n_cta = 0;
+  if (pl->n_seq <= AT_PIECES_MAX_SEQ) {
+    // groups of n_mt neighbouring CTAs (one per M tile) share a range of the (sequence, head, tile) steps
+    const long long steps_max = static_cast<long long>(pl->n_seq) * a->Hkv * (tiles + 1);   // upper bound of the work
+    long long n_grp = steps_max / 4;                                  // at least four steps per CTA on average
+    if (n_grp > slots / pl->n_mt) n_grp = slots / pl->n_mt;
+    if (n_grp < 1) n_grp = 1;
+    pl->n_cta = static_cast<int>(n_grp) * pl->n_mt;
+    const long long ctas = static_cast<long long>(pl->items);
+    const long long waves = (ctas + slots - 1) / slots;
+    const bool uneven = ctas * 100 < waves * slots * 93;              // the split plan leaves 7 % of the slots idle or more
+    // The partials' trip through the workspace and the merge launch cost 15-20 us whatever the size:
+    // worth it from a few hundred tile steps per CTA on (long_paged: 555 steps, 1.09 -> 0.98 ms; at 110
+    // steps, llama_tree, the split plan is still ahead, 165 against 180 us).
+    const int ov = attn_plan_override();
+    pl->pieces = ov == 1 || (ov == 0 && uneven && steps_max >= 256 * n_grp);
+  }
   return TRISPEC_OK;
 }
 
@@ -743,6 +717,7 @@ extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) {
   using namespace trispec;
   AttnPlan pl;
   if (attn_plan(a, &pl) != TRISPEC_OK) return 0;
+  if (pl.pieces) return attn_pieces_workspace(pl.n_cta);
   if (pl.cluster) return 0;
   return pl.items * AT_BM * (AT_D + 2) * sizeof(float);
 }
@@ -754,7 +729,7 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   int rc = attn_plan(a, &pl);
   if (rc != TRISPEC_OK) return rc;
   if (!a->q || !a->k_tree || !a->v_tree || !a->ctx_len || !a->mask || !a->o) return TRISPEC_ERR_INVALID_ARG;
-  if (!pl.cluster && !a->workspace) return TRISPEC_ERR_INVALID_ARG;
+  if ((pl.pieces || !pl.cluster) && !a->workspace) return TRISPEC_ERR_INVALID_ARG;
   if (pl.tiles_max > 0 && (!a->k_cache || !a->v_cache)) return TRISPEC_ERR_INVALID_ARG;
   if (a->kv_layout == TRISPEC_KV_PAGED && !a->block_table) return TRISPEC_ERR_INVALID_ARG;
   if (!aligned16(a->q) || !aligned16(a->k_tree) || !aligned16(a->v_tree) || !aligned16(a->k_cache) ||
@@ -793,7 +768,8 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   // tile, and never reaches the HBM-bound steady state); one P buffer and the deeper V ring for long
   // tile loops. Measured: proxy_tree (16 tiles per CTA) 45.1 -> 43.2 us with two; long_paged
   // (128-512) 1005 -> 1023 us, target_escalated (64) 150 -> 154 us, llama_tree (129) unchanged.
-  const bool two_p = pl.tiles_max / pl.n_splits <= 32;
+  const bool two_p = pl.pieces ? (static_cast<long long>(pl.n_seq) * a->Hkv * pl.n_mt * (pl.tiles_max + 1) / pl.n_cta <= 32)
+                               : (pl.tiles_max / pl.n_splits <= 32);
   typedef void (*AttnKernel)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, AttnParams);
   const AttnKernel kernel = pl.cluster ? (two_p ? verify_attn_split_kernel<true, 2> : verify_attn_split_kernel<true, 1>)
                                        : (two_p ? verify_attn_split_kernel<false, 2> : verify_attn_split_kernel<false, 1>);
@@ -815,6 +791,12 @@ extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   p.o = static_cast<uint16_t*>(a->o);
   p.lse = a->lse;
   p.dev_status = a->dev_status;
+  p.n_seq = pl.n_seq;
+  p.n_cta = pl.n_cta;
+  if (pl.pieces) {
+    const CUtensorMap maps[4] = {tm_k, tm_v, tm_kt, tm_vt};
+    return attn_launch_pieces(p, maps, two_p, a->workspace, st);
+  }
   if (pl.cluster) {
     TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(pl.items), AT_THREADS,
                                      AT_SMEM_BYTES, st, static_cast<unsigned>(pl.n_splits), tm_k, tm_v, tm_kt, tm_vt,

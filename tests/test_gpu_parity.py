@@ -237,6 +237,21 @@ def test_attention_against_oracle(H, name, over, ctx):
             assert np.isnan(o[b]).all()                       # untouched
 
 
+PIECES_CASES = [c for c in ATTN_CASES if c[0] != "tiny_chain" or c[1]] + [
+    ("long_paged", dict(B=9, L=3000, L_min=200), None),                        # ragged lengths: pieces of very different items
+    ("target_escalated", dict(B=5, n_active=3, L=1500), None),                 # 4 M tiles: groups of four CTAs share K/V
+    ("proxy_tree", dict(B=130, L=64), None),                                   # more than 128 sequences: falls back to the split plan
+]
+
+
+@pytest.mark.parametrize("name,over,ctx", PIECES_CASES)
+def test_attention_persistent_kernel_against_oracle(H, monkeypatch, name, over, ctx):
+    """The persistent kernel (balanced pieces, partials merged by a second kernel), forced through the
+    planner's override, on the cases of the split kernels and a few of its own."""
+    monkeypatch.setenv("TRISPEC_ATTN_PLAN", "pieces")
+    test_attention_against_oracle(H, name, over, ctx)
+
+
 def test_attention_argument_errors(H):
     import torch
     from paper_2601_23180_b200 import binding as ts

@@ -30,6 +30,12 @@ def test_attention_workspace_follows_the_split_plan():
     # one sequence with a very long context: more than 8 splits, workspace as well
     long1 = gen.small_variant(gen.CONFIGS["proxy_tree"], B=1, L=65536, Hq=4, Hkv=2)
     assert ts.trispec_verify_attn_workspace(_attn_args(long1)) > 0
+    # long_paged: 512 (sequence, head) items of up to 513 steps would fill two waves of 296 slots to 86 %:
+    # the persistent kernel takes it, two partial slots for each of its 296 CTAs
+    cfg = gen.CONFIGS["long_paged"]
+    a = _attn_args(cfg)
+    a.kv_layout, a.block_size, a.max_blocks_per_seq, a.num_blocks = ts.KV_PAGED, 64, cfg.L // 64, 1000
+    assert ts.trispec_verify_attn_workspace(a) == 2 * 296 * 128 * (128 + 2) * 4
 
 
 def test_lmhead_workspace_shows_the_kernel_choice():
