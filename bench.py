@@ -328,7 +328,7 @@ def run_only(args, cfg):
             "roofline": {"kernel": "accept_scan_kernel", "bound": "hbm", "achieved": scan_bytes / ms_scan / 1e6,
                          "peak": hb, "unit": "GB/s", "frac": scan_bytes / ms_scan / 1e6 / hb,
                          "work_per_launch": scan_bytes, "ms_per_launch": ms_scan, "traffic": None},
-            "scan_with_compaction": {"kernel": "accept_scan_kernel + esc_compact_kernel (one block)", "ms": ms_both,
+            "scan_with_compaction": {"kernel": "accept_scan_kernel + esc_count_kernel + esc_compact_kernel (one block per 65536 flags)", "ms": ms_both,
                                      "achieved": (scan_bytes + compact_bytes) / ms_both / 1e6, "unit": "GB/s",
                                      "frac": (scan_bytes + compact_bytes) / ms_both / 1e6 / hb},
             "tree_mask_roofline": {"kernel": "tree_mask_block_kernel", "bound": "hbm", "achieved": mask_bytes / ms_mask / 1e6,
@@ -416,8 +416,9 @@ def run_only(args, cfg):
         ms = timed(lambda: ts.trispec_verify_attn(pas.attn_args), byts)
         flops = 4.0 * rows * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
         roof = _roof(peaks, flops, byts, ms)
-        roof["kernel"] = "verify_attn_split_kernel"
-        roof["traffic"] = dram_traffic("verify_attn_split_kernel", cfg.name)
+        roof["kernel"] = ("verify_attn_pieces_kernel" if ts.trispec_verify_attn_plan(pas.attn_args) == "pieces"
+                          else "verify_attn_split_kernel")
+        roof["traffic"] = dram_traffic(roof["kernel"], cfg.name)
     else:
         inp = gen.make_inputs(cfg, with_attention=False)
         pas = runner.VerifyPass(cfg, inp, with_attention=False)
@@ -609,7 +610,9 @@ def measure_workload(cfg, inp, steps, warmup, peaks, world=1, dist=None, clock_i
     Lsum = float(np.asarray(inp["ctx_len"])[pas.seqs].sum())
     attn_bytes = (Lsum + n_seq * cfg.T) * cfg.Hkv * cfg.D * 2 * 2 + 2 * n_seq * cfg.T * cfg.Hq * cfg.D * 2
     attn_flops = 4.0 * cfg.T * cfg.Hq * cfg.D * (Lsum + n_seq * cfg.T)
-    attn_roof = _roofline("attention", peaks, attn_flops, attn_bytes, ms_attn, 0.0, "verify_attn_split_kernel",
+    attn_kernel = "verify_attn_pieces_kernel" if ts.trispec_verify_attn_plan(pas.attn_args) == "pieces" \
+        else "verify_attn_split_kernel"
+    attn_roof = _roofline("attention", peaks, attn_flops, attn_bytes, ms_attn, 0.0, attn_kernel,
                           cfg.name, "trispec_verify_attn bracketed by CUDA events right after an LM-head call "
                           "(the cache state it meets inside a pass)")
     out = {"total_ms": total_ms, "e2e_ms": e2e_ms, "launches": launches, "host_us_per_call": host_us_per_call,

@@ -155,6 +155,12 @@ typedef struct {
 } trispec_attn_args;
 size_t trispec_verify_attn_workspace(const trispec_attn_args* a);
 int trispec_verify_attn(const trispec_attn_args* a, void* stream);
+/* Which kernels a call with these arguments would take (a diagnostic; host only, nothing is launched):
+ * "cluster" = key/value splits merged on chip, "splits" = splits merged through the workspace,
+ * "pieces" = persistent CTAs over balanced pieces of the work (long or ragged contexts), "none" =
+ * arguments refused. The environment variable TRISPEC_ATTN_PLAN = pieces | splits overrides the choice
+ * between the last one and the first two where both apply. */
+const char* trispec_verify_attn_plan(const trispec_attn_args* a);
 
 /* ---------------------------------------------------------------------------------------
  * 3. LM-head softmax statistics (distributions p_i in R^V of Eq. 5; top_1, top_2 of Eq. 8).

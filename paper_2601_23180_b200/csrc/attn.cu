@@ -722,6 +722,13 @@ extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) {
   return pl.items * AT_BM * (AT_D + 2) * sizeof(float);
 }
 
+extern "C" const char* trispec_verify_attn_plan(const trispec_attn_args* a) {
+  using namespace trispec;
+  AttnPlan pl;
+  if (attn_plan(a, &pl) != TRISPEC_OK) return "none";
+  return pl.pieces ? "pieces" : (pl.cluster ? "cluster" : "splits");
+}
+
 extern "C" int trispec_verify_attn(const trispec_attn_args* a, void* stream) {
   trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
   using namespace trispec;

@@ -13,7 +13,7 @@
 // piece while the softmax threads finish the current one. A piece that covers a whole
 // (sequence, head, M tile) is normalised and stored directly; any other piece leaves an fp32 partial
 // (O, m, l) in the caller's workspace (a CTA has at most two of those, its first and its last piece),
-// and a second kernel merges the partials of every row. No CTA waits for another one.
+// and a second kernel merges the partials of the items that were cut. No CTA waits for another one.
 //
 // Nothing here depends on how the tile counts divide the chip: there is no wave of CTAs that ends
 // early or late, and every SM hosts the same two CTAs from start to end. The price is the partials'
@@ -589,22 +589,24 @@ verify_attn_pieces_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid
 }
 
 // ---------------------------------------------------------------------------------------
-// Merge of the partials: one warp per output row (sequence, node, query head). The warp rebuilds
-// the partition (before it waits for the first kernel), finds the groups that shared the row's
-// (sequence, head) and folds their partials in one pass, four partials' loads in flight at a time;
-// a row whose (sequence, head) was a single piece has been written by the first kernel.
+// Merge of the partials: four blocks per (sequence, KV head, M tile), each with sixteen warps that take
+// a quarter of the item's rows in turn. Every warp rebuilds the partition (before it waits for the first kernel) and
+// finds the groups that shared the item; an item that was a single piece has been written by the
+// first kernel and costs its block nothing more. A row's partials are folded in one pass, four
+// partials' loads in flight at a time.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+constexpr int AP_MERGE_THREADS = 512;
+constexpr int AP_MERGE_BLOCKS = 4;              // blocks per item, 32 rows each
+
+__global__ void __launch_bounds__(AP_MERGE_THREADS)
 verify_attn_pieces_merge_kernel(const AttnParams p) {
   pdl_launch_dependents();
-  const int lane = threadIdx.x & 31;
-  const long long wi = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
-  const long long total = static_cast<long long>(p.n_seq) * p.T * p.Hq;
-  if (wi >= total) return;                       // whole warps leave: the collectives below stay complete
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int item = blockIdx.x / AP_MERGE_BLOCKS, quarter = blockIdx.x % AP_MERGE_BLOCKS;
+  const int mtile = item % p.n_mt;
+  const int g = (item / p.n_mt) % p.Hkv;
+  const int a = item / (p.n_mt * p.Hkv);
   const WorkMap wm = load_work_map(p, lane, false);
-  const int hq = static_cast<int>(wi % p.Hq);
-  const int node = static_cast<int>((wi / p.Hq) % p.T);
-  const int a = static_cast<int>(wi / (static_cast<long long>(p.Hq) * p.T));
   // the sequence's entry of the map lives in lane a % 32, slot a / 32
   int L = 0, nn = 0, pre = 0;
 #pragma unroll
@@ -613,58 +615,61 @@ verify_attn_pieces_merge_kernel(const AttnParams p) {
     const int pj = __shfl_sync(0xffffffffu, wm.pre[j], a & 31);
     if (j == (a >> 5)) { L = Lj; nn = nj; pre = pj; }
   }
-  if (node >= nn) return;                        // not a node of this (pruned) tree
-  const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
-  const int g = hq / p.G, jq = hq % p.G;
-  const int mtile = node / p.NPT;
-  const int row = (node % p.NPT) * p.G + jq;
+  if (mtile * p.NPT >= nn) return;               // no node of this (pruned) tree in the M tile
   const int n_it = (L + AT_BN - 1) / AT_BN + 1;
   const long long W = wm.total;
   const int n_grp = p.n_cta / p.n_mt;
   const long long x = pre + static_cast<long long>(g) * n_it;                 // first global step of the (sequence, head)
   const int r_first = cta_of_step(W, n_grp, x), r_last = cta_of_step(W, n_grp, x + n_it - 1);
   if (r_first == r_last) return;                 // one piece: stored by the first kernel
+  const int b = p.seq_index ? __ldg(p.seq_index + a) : a;
   pdl_wait();                                    // the partials come from the kernel before
-  float M = -INFINITY, Lsum = 0.f;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int r0 = r_first; r0 <= r_last; r0 += 4) {
-    float2 ml[4];
-    float4 v[4];
+  const int n_rows = min(min(AT_BM, p.NPT * p.G), (quarter + 1) * (AT_BM / AP_MERGE_BLOCKS));
+  for (int row = quarter * (AT_BM / AP_MERGE_BLOCKS) + warp; row < n_rows; row += AP_MERGE_THREADS / 32) {
+    const int node = mtile * p.NPT + row / p.G;
+    if (node >= nn) break;                       // rows are in node order
+    const int hq = g * p.G + row % p.G;
+    float M = -INFINITY, Lsum = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int r0 = r_first; r0 <= r_last; r0 += 4) {
+      float2 ml[4];
+      float4 v[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      ml[k] = make_float2(-INFINITY, 0.f);
-      v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      const int r = r0 + k;
-      if (r <= r_last) {
-        // slot 2c for the piece a CTA starts with (the item began before the group's range), else 2c + 1
-        const size_t c = static_cast<size_t>(r) * p.n_mt + mtile;
-        const size_t slot = 2 * c + (cta_first_step(W, n_grp, r) >= x ? 0 : 1);
-        ml[k] = __ldg(reinterpret_cast<const float2*>(p.part_ml + (slot * AT_BM + row) * 2));
-        v[k] = __ldg(reinterpret_cast<const float4*>(p.part_o + (slot * AT_BM + row) * AT_D) + lane);
+      for (int k = 0; k < 4; ++k) {
+        ml[k] = make_float2(-INFINITY, 0.f);
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int r = r0 + k;
+        if (r <= r_last) {
+          // slot 2c for the piece a CTA starts with (the item began before the group's range), else 2c + 1
+          const size_t c = static_cast<size_t>(r) * p.n_mt + mtile;
+          const size_t slot = 2 * c + (cta_first_step(W, n_grp, r) >= x ? 0 : 1);
+          ml[k] = __ldg(reinterpret_cast<const float2*>(p.part_ml + (slot * AT_BM + row) * 2));
+          v[k] = __ldg(reinterpret_cast<const float4*>(p.part_o + (slot * AT_BM + row) * AT_D) + lane);
+        }
+      }
+      float Mn = M;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) Mn = fmaxf(Mn, ml[k].x);
+      const float keep = (M == -INFINITY) ? 0.f : ex2f(M - Mn);
+      Lsum *= keep;
+      acc.x *= keep; acc.y *= keep; acc.z *= keep; acc.w *= keep;
+      M = Mn;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float wgt = (ml[k].x == -INFINITY) ? 0.f : ex2f(ml[k].x - M);
+        Lsum += ml[k].y * wgt;
+        acc.x = fmaf(v[k].x, wgt, acc.x); acc.y = fmaf(v[k].y, wgt, acc.y);
+        acc.z = fmaf(v[k].z, wgt, acc.z); acc.w = fmaf(v[k].w, wgt, acc.w);
       }
     }
-    float Mn = M;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) Mn = fmaxf(Mn, ml[k].x);
-    const float keep = (M == -INFINITY) ? 0.f : ex2f(M - Mn);
-    Lsum *= keep;
-    acc.x *= keep; acc.y *= keep; acc.z *= keep; acc.w *= keep;
-    M = Mn;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float wgt = (ml[k].x == -INFINITY) ? 0.f : ex2f(ml[k].x - M);
-      Lsum += ml[k].y * wgt;
-      acc.x = fmaf(v[k].x, wgt, acc.x); acc.y = fmaf(v[k].y, wgt, acc.y);
-      acc.z = fmaf(v[k].z, wgt, acc.z); acc.w = fmaf(v[k].w, wgt, acc.w);
-    }
+    const float inv = (Lsum > 0.f) ? 1.f / Lsum : 0.f;
+    uint2 out;
+    out.x = pack_bf16(acc.x * inv, acc.y * inv);
+    out.y = pack_bf16(acc.z * inv, acc.w * inv);
+    uint16_t* orow = p.o + ((static_cast<size_t>(b) * p.T + node) * p.Hq + hq) * AT_D;
+    *reinterpret_cast<uint2*>(orow + lane * 4) = out;
+    if (p.lse && lane == 0) p.lse[(static_cast<size_t>(b) * p.Hq + hq) * p.T + node] = (M + log2f(Lsum)) * kLn2;
   }
-  const float inv = (Lsum > 0.f) ? 1.f / Lsum : 0.f;
-  uint2 out;
-  out.x = pack_bf16(acc.x * inv, acc.y * inv);
-  out.y = pack_bf16(acc.z * inv, acc.w * inv);
-  uint16_t* orow = p.o + ((static_cast<size_t>(b) * p.T + node) * p.Hq + hq) * AT_D;
-  *reinterpret_cast<uint2*>(orow + lane * 4) = out;
-  if (p.lse && lane == 0) p.lse[(static_cast<size_t>(b) * p.Hq + hq) * p.T + node] = (M + log2f(Lsum)) * kLn2;
 }
 
 size_t attn_pieces_workspace(int n_cta) {
@@ -683,9 +688,9 @@ int attn_launch_pieces(AttnParams p, const CUtensorMap* maps, bool two_p, void* 
   TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(p.n_cta), AT_THREADS, AT_SMEM_BYTES, st, 1, maps[0],
                                    maps[1], maps[2], maps[3], p));
   count_launch();
-  const long long rows = static_cast<long long>(p.n_seq) * p.T * p.Hq;
-  TRISPEC_CUDA_OK(launch_dependent(verify_attn_pieces_merge_kernel, static_cast<unsigned>((rows + 7) / 8), 256, 0, st,
-                                   1, p));
+  const long long items = static_cast<long long>(p.n_seq) * p.Hkv * p.n_mt;
+  TRISPEC_CUDA_OK(launch_dependent(verify_attn_pieces_merge_kernel, static_cast<unsigned>(items * AP_MERGE_BLOCKS), AP_MERGE_THREADS, 0,
+                                   st, 1, p));
   count_launch();
   return TRISPEC_OK;
 }

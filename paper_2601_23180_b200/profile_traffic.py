@@ -31,7 +31,8 @@ _COMMON = ["csrc/sm100.cuh", "csrc/host_common.h"]
 SOURCES = {
     "lmhead_gemm_kernel": ["csrc/lmhead.cu"] + _COMMON,
     "lmhead_rows_kernel": ["csrc/lmhead.cu"] + _COMMON,
-    "verify_attn_split_kernel": ["csrc/attn.cu"] + _COMMON,
+    "verify_attn_split_kernel": ["csrc/attn.cu", "csrc/attn_common.cuh"] + _COMMON,
+    "verify_attn_pieces_kernel": ["csrc/attn_pieces.cu", "csrc/attn_common.cuh"] + _COMMON,
     "accept_scan_kernel": ["csrc/accept_scan.cu", "csrc/host_common.h"],
     "tree_mask_block_kernel": ["csrc/tree_mask.cu", "csrc/host_common.h"],
 }

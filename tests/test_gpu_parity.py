@@ -394,3 +394,34 @@ def test_fused_pass_at_size_limits(H, name, over):
     ref = orc.verify(inp, 1.0 / math.sqrt(cfg.D), cfg.logit_scale, cfg.lam, mode=cfg.mode)
     _check_pass(H, cfg, inp, got, ref, list(range(cfg.B)))
     assert got["mask"].view(np.uint64).max() == ref["mask"].max()
+
+
+@pytest.mark.parametrize("plan", ["splits", "pieces"])
+def test_attention_with_one_dominant_split_and_large_values(H, monkeypatch, plan):
+    """Eight KV splits of one sequence, one of which holds every key that matters (scores about 20
+    above the rest) while the values are eight times larger than usual: the splits' partials differ by
+    e^20 in weight, which is where a partial kept in low precision, or merged with the wrong reference
+    maximum, would show. The outputs reach several units here, where half a bf16 step of the result alone is
+    1.6e-2: the bound is the usual 2e-2 plus one bf16 step (2^-8 relative) of the reference value."""
+    monkeypatch.setenv("TRISPEC_ATTN_PLAN", plan)
+    cfg = gen.small_variant(gen.CONFIGS["proxy_tree"], B=1, L=2048, seed=23)
+    inp = gen.make_inputs(cfg, with_lm_head=False)
+    q = gen.bf16_bits_to_f32(inp["q"])
+    k = gen.bf16_bits_to_f32(inp["k_cache"])
+    q[..., 0] = 8.0                                           # every query row looks along dimension 0
+    k[0, 768:1024, :, 0] = 28.25                              # keys of tiles 12-15 (split 3 of 8): +20 after scaling
+    inp["q"], inp["k_cache"] = gen.f32_to_bf16_bits(q), gen.f32_to_bf16_bits(k)
+    for name in ("v_cache", "v_tree"):
+        inp[name] = gen.f32_to_bf16_bits(gen.bf16_bits_to_f32(inp[name]) * 8.0)
+    dev = H.to_device(inp)
+    mask_dev, _ = H.run_tree_mask(dev["parent"])
+    o, lse = H.run_attn(dev, cfg, mask_dev)
+    ref_mask, _ = orc.build_tree_mask(inp["parent"])
+    ref_o, ref_lse = orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], ref_mask, inp["k_cache"], inp["v_cache"],
+                                     inp["ctx_len"], 1.0 / math.sqrt(cfg.D))
+    assert np.abs(ref_lse).min() > 18.0                       # the dominant split decides every row
+    assert 0.3 < np.abs(ref_o).max() < 8.0
+    assert (np.abs(o - ref_o) <= 2e-2 + np.abs(ref_o) / 256.0).all()
+    small = np.abs(ref_o) < 1.0
+    assert small.mean() > 0.3 and np.abs(o - ref_o)[small].max() <= 2e-2
+    assert np.abs(lse - ref_lse).max() <= 1e-3 * np.abs(ref_lse).max()

@@ -36,6 +36,9 @@ def test_attention_workspace_follows_the_split_plan():
     a = _attn_args(cfg)
     a.kv_layout, a.block_size, a.max_blocks_per_seq, a.num_blocks = ts.KV_PAGED, 64, cfg.L // 64, 1000
     assert ts.trispec_verify_attn_workspace(a) == 2 * 296 * 128 * (128 + 2) * 4
+    assert ts.trispec_verify_attn_plan(a) == "pieces"
+    assert ts.trispec_verify_attn_plan(_attn_args(gen.CONFIGS["proxy_tree"])) == "cluster"
+    assert ts.trispec_verify_attn_plan(_attn_args(gen.CONFIGS["target_escalated"], n_active=3)) == "splits"
 
 
 def test_lmhead_workspace_shows_the_kernel_choice():
