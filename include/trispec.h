@@ -336,8 +336,10 @@ int trispec_commit_kv(const trispec_commit_args* a, void* stream);
  *    Gumbel-max identity: argmax_v (z_v + G_v), G_v independent standard Gumbel variates
  *    (ties -> lowest index). The noise is counter-based and reproducible: word (v mod 4) of
  *    Philox-4x32-10 with counter (v div 4, b, step low, step high) and key (seed low, seed high)
- *    gives u = ((word >> 9) + 0.5) / 2^23 and G = -ln(-ln u). One more pass over W, no logits
- *    in global memory.
+ *    gives u = ((word >> 9) + 0.5) / 2^23 and G = -ln(-ln u). (The upper 23 bits of the word: u is
+ *    then exact in single precision and never 0 or 1. It bounds the variate to [-2.812, 16.636]:
+ *    an entry more than 19.45 below the largest logit, probability under 4e-9, is never drawn.)
+ *    One more pass over W, no logits in global memory.
  *      h [B*T][d], W [V][d] bf16 as in trispec_lmhead_stats; last_node [B] int32.
  *      bonus_tok [B] int32, in/out: entries equal to -2 are replaced by the sampled token;
  *        other entries are left alone. sample_value (optional f32 [B]): the winning z_v + G_v.
