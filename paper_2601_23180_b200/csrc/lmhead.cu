@@ -488,8 +488,17 @@ lmhead_finalize_kernel(const LmFinalizeParams p, int n_seq) {
 // One sequence (batch-1 decoding, the paper's own setting): operands swapped. With at most 64
 // rows the GEMM is bound by streaming W, and the pair kernel above spends half of its ring
 // on H tiles. Here W is the M-side operand (128 vocabulary entries per MMA), the sequence's
-// rows are the N side (16-64 columns), one CTA per SM, and a stage is 16 KB of W plus 2-8 KB of
-// H: up to 12 stages, almost all of them W. TMEM lane = vocabulary entry, column = tree node.
+// rows are the N side (16-64 columns), one CTA per SM, and a stage is KPS k-blocks of 16 KB of W plus
+// 2-8 KB of H each, almost all of it W. TMEM lane = vocabulary entry, column = tree node.
+// A CTA's vocabulary range is a multiple of 16 entries but rarely of 128: its last tile is fetched with
+// a second, lower box (only the rows the range owns; the MMA still spans 128 lanes, the lanes past
+// the range read stale shared memory and are ignored), so the chip streams W once, not the 5-18 %
+// more that whole tiles would cost on a launch that is bound by exactly this stream.
+// With KPS = 4 (any vocabulary that is a multiple of 8) W is read through a 4-D view
+// [V/8][d/64][8 rows][64 elements], whose box puts the k-blocks of one group of 8 rows next to each
+// other in the request stream; the stage then holds [16 row groups][KPS k-blocks][8 rows][128 B], and
+// the MMA descriptor of k-block j starts j KB in with KPS KB between row groups. KPS = 1 is the
+// plain 2-D view, the same layout with one k-block.
 // Epilogue: per tile a warp reduces 32 columns at once over its 32 vocabulary entries with
 // transposing shuffle butterflies (top-2 with indices, then the sums of exponentials), after which
 // lane l holds column l's result and folds it into the running statistics it keeps for that column.
@@ -502,14 +511,15 @@ struct LmRowsParams {
   LmParams base;
   int N;            // node columns: T rounded up to 16
   int stages, stage_bytes;
+  int tail_rows;    // height of the second W box (a multiple of 16 below 128), 0 = no second box
 };
 
 struct LmColStats { float m, s, t, v1, v2; int i1, i2; };
 
-template <bool kEntropy>
+template <bool kEntropy, int KPS>
 __global__ void __launch_bounds__(LW_THREADS, 1)
-lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-                   const LmRowsParams sp) {
+lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_wt,
+                   const __grid_constant__ CUtensorMap tmap_h, const LmRowsParams sp) {
   pdl_launch_dependents();
   const LmParams& p = sp.base;
   extern __shared__ uint8_t smem_raw[];
@@ -541,7 +551,7 @@ lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     tmem_alloc(tmem_slot, 128);                   // two accumulators of at most 64 columns
     tmem_relinquish();
   }
-  if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_h); prefetch_tmap(&tmap_w); }
+  if (warp == 4 && lane == 0) { prefetch_tmap(&tmap_h); prefetch_tmap(&tmap_w); prefetch_tmap(&tmap_wt); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -551,15 +561,23 @@ lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     if (lane == 0) {   // ---------------------------------------------------------- TMA producer
       int stage = 0;
       uint32_t phase = 0;
-      const uint32_t tx = static_cast<uint32_t>(LW_A_BYTES + sp.N * LW_BK * 2);
       const int seq = p.seq_index ? __ldg(p.seq_index) : 0;     // the one active sequence
+      const int h_bytes = sp.N * LW_BK * 2;
       for (int t = 0; t < n_tiles; ++t) {
-        for (int kb = 0; kb < n_kb; ++kb) {
+        const int row0 = v_begin + t * LW_BM;
+        // a box always delivers its full size (rows past V, k-blocks past d: zero fill)
+        const bool low = sp.tail_rows > 0 && v_end - row0 <= sp.tail_rows;
+        const CUtensorMap* tw = low ? &tmap_wt : &tmap_w;
+        const int w_bytes = KPS * (low ? sp.tail_rows : LW_BM) * LW_BK * 2;
+        for (int kb = 0; kb < n_kb; kb += KPS) {
+          const int kc = min(KPS, n_kb - kb);
           mbar_wait(empty_bar + stage, phase ^ 1u, p.dev_status);
           uint8_t* sa = smem + stage * sp.stage_bytes;
-          mbar_expect_tx(full_bar + stage, tx);
-          tma_load_2d(sa, &tmap_w, full_bar + stage, kb * LW_BK, v_begin + t * LW_BM);   // rows past V: zero fill
-          tma_load_3d(sa + LW_A_BYTES, &tmap_h, full_bar + stage, kb * LW_BK, 0, seq);     // nodes past T: zero fill
+          mbar_expect_tx(full_bar + stage, static_cast<uint32_t>(w_bytes + kc * h_bytes));
+          if (KPS == 1) tma_load_2d(sa, tw, full_bar + stage, kb * LW_BK, row0);
+          else tma_load_4d(sa, tw, full_bar + stage, 0, 0, kb, row0 >> 3);
+          for (int j = 0; j < kc; ++j)                                                     // nodes past T: zero fill
+            tma_load_3d(sa + KPS * LW_A_BYTES + j * h_bytes, &tmap_h, full_bar + stage, (kb + j) * LW_BK, 0, seq);
           if (++stage == sp.stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -574,14 +592,17 @@ lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         mbar_wait(tmem_empty + buf, ((t >> 1) & 1u) ^ 1u, p.dev_status);
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * 64);
-        for (int kb = 0; kb < n_kb; ++kb) {
+        for (int kb = 0; kb < n_kb; kb += KPS) {
+          const int kc = min(KPS, n_kb - kb);
           mbar_wait(full_bar + stage, phase, p.dev_status);
           tc_fence_after();
           const uint32_t sa = base_u32 + stage * sp.stage_bytes;
-          const uint64_t adesc = smem_desc_sw128(sa, 1024, 16);
-          const uint64_t bdesc = smem_desc_sw128(sa + LW_A_BYTES, 1024, 16);
+          for (int j = 0; j < kc; ++j) {
+            const uint64_t adesc = smem_desc_sw128(sa + j * 1024, KPS * 1024, 16);
+            const uint64_t bdesc = smem_desc_sw128(sa + KPS * LW_A_BYTES + j * (sp.N * LW_BK * 2), 1024, 16);
 #pragma unroll
-          for (int k = 0; k < LW_BK / 16; ++k) tc_mma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < LW_BK / 16; ++k) tc_mma_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | j | k) != 0);
+          }
           tc_commit(empty_bar + stage);
           if (++stage == sp.stages) { stage = 0; phase ^= 1u; }
         }
@@ -849,16 +870,35 @@ static int trispec::lmhead_stats_planned(const trispec_lmhead_args* a, const LmP
     sp.base.partial = static_cast<LmPartial*>(a->workspace);
     sp.base.dev_status = a->dev_status;
     sp.N = ((a->T + 15) / 16) * 16;
-    sp.stage_bytes = LW_A_BYTES + sp.N * LW_BK * 2;
+    const int kps = (a->V % 8) == 0 ? 4 : 1;
+    sp.stage_bytes = kps * (LW_A_BYTES + sp.N * LW_BK * 2);
     sp.stages = (216 * 1024) / sp.stage_bytes;
     if (sp.stages > LW_MAX_STAGES) sp.stages = LW_MAX_STAGES;
     const int smem_bytes = sp.stages * sp.stage_bytes + 1024 + 8192;
-    CUtensorMap tm_w128, tm_hn;
+    // the longer of the two range lengths (they differ by 16 rows) decides the height of the second box
     {
-      const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
-      const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
-      const uint32_t box[2] = {LW_BK, LW_BM};
-      if (!cached_tmap_bf16(&tm_w128, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+      const int V16 = (a->V + 15) / 16;
+      const int r_big = ((V16 + n_ranges - 1) / n_ranges) * 16;
+      const int last = r_big - LW_BM * ((r_big + LW_BM - 1) / LW_BM - 1);
+      sp.tail_rows = last < LW_BM ? last : 0;
+    }
+    CUtensorMap tm_w128, tm_wt, tm_hn;
+    for (int m = 0; m < 2; ++m) {
+      const uint32_t rows = m == 0 ? LW_BM : static_cast<uint32_t>(sp.tail_rows);
+      CUtensorMap* tm = m == 0 ? &tm_w128 : &tm_wt;
+      if (rows == 0) { tm_wt = tm_w128; break; }
+      if (kps == 1) {
+        const uint64_t dims[2] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->V)};
+        const uint64_t strides[1] = {static_cast<uint64_t>(a->d) * 2};
+        const uint32_t box[2] = {LW_BK, rows};
+        if (!cached_tmap_bf16(tm, a->W, 2, dims, strides, box)) return TRISPEC_ERR_CUDA;
+      } else {
+        // [V/8 groups][d/64 k-blocks][8 rows][64 elements]: the k-block index moves 128 B, the row 2 d B
+        const uint64_t dims[4] = {LW_BK, 8, static_cast<uint64_t>(a->d / LW_BK), static_cast<uint64_t>(a->V / 8)};
+        const uint64_t strides[3] = {static_cast<uint64_t>(a->d) * 2, LW_BK * 2, static_cast<uint64_t>(a->d) * 16};
+        const uint32_t box[4] = {LW_BK, 8, static_cast<uint32_t>(kps), rows / 8};
+        if (!cached_tmap_bf16(tm, a->W, 4, dims, strides, box)) return TRISPEC_ERR_CUDA;
+      }
     }
     {
       const uint64_t dims[3] = {static_cast<uint64_t>(a->d), static_cast<uint64_t>(a->T), static_cast<uint64_t>(a->B)};
@@ -866,13 +906,16 @@ static int trispec::lmhead_stats_planned(const trispec_lmhead_args* a, const LmP
       const uint32_t box[3] = {LW_BK, static_cast<uint32_t>(sp.N), 1};
       if (!cached_tmap_bf16(&tm_hn, a->h, 3, dims, strides, box)) return TRISPEC_ERR_CUDA;
     }
-    typedef void (*RowsKernel)(CUtensorMap, CUtensorMap, LmRowsParams);
-    const RowsKernel kernel = want_entropy ? lmhead_rows_kernel<true> : lmhead_rows_kernel<false>;
-    static bool smem_set_rows[2][64] = {};
-    rc = ensure_smem_limit(reinterpret_cast<const void*>(kernel), 227 * 1024, smem_set_rows[want_entropy ? 1 : 0]);
+    typedef void (*RowsKernel)(CUtensorMap, CUtensorMap, CUtensorMap, LmRowsParams);
+    static const RowsKernel table[2][2] = {{lmhead_rows_kernel<false, 1>, lmhead_rows_kernel<false, 4>},
+                                           {lmhead_rows_kernel<true, 1>, lmhead_rows_kernel<true, 4>}};
+    const int wide = kps > 1 ? 1 : 0;
+    const RowsKernel kernel = table[want_entropy ? 1 : 0][wide];
+    static bool smem_set_rows[4][64] = {};
+    rc = ensure_smem_limit(reinterpret_cast<const void*>(kernel), 227 * 1024, smem_set_rows[(want_entropy ? 2 : 0) + wide]);
     if (rc != TRISPEC_OK) return rc;
     TRISPEC_CUDA_OK(launch_dependent(kernel, static_cast<unsigned>(n_ranges), LW_THREADS,
-                                     static_cast<size_t>(smem_bytes), st, 1, tm_w128, tm_hn, sp));
+                                     static_cast<size_t>(smem_bytes), st, 1, tm_w128, tm_wt, tm_hn, sp));
     count_launch();
     f.stride = LW_ROWS;
     TRISPEC_CUDA_OK(launch_dependent(lmhead_finalize_kernel, static_cast<unsigned>((a->T + 7) / 8),

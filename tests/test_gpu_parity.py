@@ -141,6 +141,8 @@ LM_CASES = [
     ("target_escalated", dict(B=4, n_active=1, V=7000, d=320)),                  # the one sequence is picked by seq_index
     ("tiny_chain", dict(k=15, V=3000, d=128)),                                   # 16 nodes: exactly one 16-column block
     ("tiny_chain", dict(k=31, V=200, d=64)),                                     # 32 nodes, fewer vocabulary units than SMs
+    ("proxy_tree", dict(B=1, V=151936 // 8, d=192)),                             # ranges of 128 + 16 rows: the low second box
+    ("llama_tree", dict(B=1, V=128256 // 8 + 4, d=256)),                         # vocabulary not a multiple of 8: the 2-D view of W
 ]
 
 
