@@ -362,8 +362,10 @@ size_t trispec_sample_bonus_workspace(const trispec_sample_args* a);
 int trispec_sample_bonus(const trispec_sample_args* a, void* stream);
 
 /* ---------------------------------------------------------------------------------------
- * Fused pass: the four calls above in order on `stream` (one verification round of
- * Algorithm 1 for one verifier). `attn` may be NULL to skip attention.
+ * Fused pass: the four calls above on `stream` (one verification round of Algorithm 1 for
+ * one verifier): tree mask first, acceptance scan last; the attention and the LM-head
+ * statistics, which do not read each other's results, in the order the library finds faster
+ * for the shape. `attn` may be NULL to skip attention.
  * ------------------------------------------------------------------------------------- */
 int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                    const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream);

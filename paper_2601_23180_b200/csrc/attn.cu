@@ -711,6 +711,12 @@ static int attn_plan(const trispec_attn_args* a, AttnPlan* pl) {
   return TRISPEC_OK;
 }
 
+int attn_planned_ctas(const trispec_attn_args* a) {
+  AttnPlan pl;
+  if (attn_plan(a, &pl) != TRISPEC_OK) return 0;
+  return pl.pieces ? pl.n_cta : static_cast<int>(pl.items);
+}
+
 }  // namespace trispec
 
 extern "C" size_t trispec_verify_attn_workspace(const trispec_attn_args* a) {

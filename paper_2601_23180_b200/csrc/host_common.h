@@ -85,6 +85,9 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
+// CTAs the attention launch for these arguments will use (0 if the arguments are not accepted)
+int attn_planned_ctas(const trispec_attn_args* a);
+
 #define TRISPEC_CUDA_OK(expr)                        \
   do {                                               \
     cudaError_t _e = (expr);                         \
