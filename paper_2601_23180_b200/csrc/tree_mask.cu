@@ -66,16 +66,34 @@ tree_mask_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask
 // about ten instructions per node for one thread, against a whole warp climbing level by level
 // above (which is the better shape for a decode batch, where sequences are few). A block takes 64
 // sequences: all 256 threads load their parents (16-byte loads) into shared memory, 64 threads walk,
-// all 256 threads write masks and depths back, coalesced.
+// all 256 threads write masks and depths back, coalesced. The (sequence, node) pair of a flat element
+// index is carried along incrementally (no division by the run-time T in the copy loops), and the
+// masks sit in shared memory sequence-major with an odd pitch: the walkers (one sequence per lane)
+// and the copy-out (consecutive elements per lane) both touch distinct banks.
 constexpr int kMaskBlockSeqs = 64, kMaskBlockThreads = 256;
 constexpr int kMaskParPitch = kMaskBlockSeqs + 4;   // bytes per node row of the parent table (bank spread)
-constexpr int kMaskRowPitch = kMaskBlockSeqs + 1;   // masks per node row
+constexpr int kMaskSeqPitch = 65;                   // masks per sequence row (T <= 64, odd)
+
+// element index e = seq * T + node, advanced by `step` elements
+struct MaskElem {
+  int seq, node;
+  __device__ __forceinline__ void advance(int dseq, int dnode, int T) {
+    seq += dseq;
+    node += dnode;
+    if (node >= T) { node -= T; ++seq; }
+  }
+  __device__ __forceinline__ MaskElem next(int T) const {
+    MaskElem r = *this;
+    if (++r.node == T) { r.node = 0; ++r.seq; }
+    return r;
+  }
+};
 
 __global__ void __launch_bounds__(kMaskBlockThreads)
 tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask, int32_t* __restrict__ depth,
                        long long n_seq, int T, int32_t* __restrict__ status) {
   __shared__ signed char sPar[64 * kMaskParPitch];
-  __shared__ unsigned long long sMask[64 * kMaskRowPitch];
+  __shared__ unsigned long long sMask[kMaskBlockSeqs * kMaskSeqPitch];
   pdl_launch_dependents();
   pdl_wait();
   const long long s0 = static_cast<long long>(blockIdx.x) * kMaskBlockSeqs;
@@ -83,23 +101,33 @@ tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict_
   const int n_elem = n_here * T;
   const int32_t* src = parent + s0 * T;
   // parents -> shared memory as bytes ([node][sequence]); anything outside [-1, 62] becomes -2
-  auto put = [&](int e, int v) {
-    const int seq = e / T, node = e - seq * T;
-    sPar[node * kMaskParPitch + seq] = static_cast<signed char>((v >= -1 && v < 63) ? v : -2);
+  auto put = [&](const MaskElem& e, int v) {
+    sPar[e.node * kMaskParPitch + e.seq] = static_cast<signed char>((v >= -1 && v < 63) ? v : -2);
   };
   if ((n_elem & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
     const int4* src4 = reinterpret_cast<const int4*>(src);
+    const int first = 4 * threadIdx.x, step = 4 * kMaskBlockThreads;
+    MaskElem e0 = {first / T, first % T};
+    const int dseq = step / T, dnode = step % T;
 #pragma unroll 2
     for (int q = threadIdx.x; q < (n_elem >> 2); q += kMaskBlockThreads) {
       const int4 v = __ldg(src4 + q);
-      put(4 * q, v.x); put(4 * q + 1, v.y); put(4 * q + 2, v.z); put(4 * q + 3, v.w);
+      const MaskElem e1 = e0.next(T), e2 = e1.next(T), e3 = e2.next(T);
+      put(e0, v.x); put(e1, v.y); put(e2, v.z); put(e3, v.w);
+      e0.advance(dseq, dnode, T);
     }
   } else {
-    for (int e = threadIdx.x; e < n_elem; e += kMaskBlockThreads) put(e, __ldg(src + e));
+    MaskElem e0 = {static_cast<int>(threadIdx.x) / T, static_cast<int>(threadIdx.x) % T};
+    const int dseq = kMaskBlockThreads / T, dnode = kMaskBlockThreads % T;
+    for (int e = threadIdx.x; e < n_elem; e += kMaskBlockThreads) {
+      put(e0, __ldg(src + e));
+      e0.advance(dseq, dnode, T);
+    }
   }
   __syncthreads();
   if (threadIdx.x < n_here) {
     const int t = threadIdx.x;
+    unsigned long long* row = sMask + t * kMaskSeqPitch;
     bool bad = false;
     for (int i = 0; i < T; ++i) {
       const int par = sPar[i * kMaskParPitch + t];
@@ -111,33 +139,37 @@ tree_mask_block_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict_
         m = 0ull;                                           // malformed: flagged, not followed
         bad = true;
       } else {
-        const unsigned long long pm = sMask[par * kMaskRowPitch + t];
+        const unsigned long long pm = row[par];
         m = pm ? (pm | (1ull << i)) : 0ull;                 // a malformed ancestor spoils the walk
       }
-      sMask[i * kMaskRowPitch + t] = m;
+      row[i] = m;
     }
     if (bad && status) atomicExch(status, TRISPEC_ERR_BAD_TREE);
   }
   __syncthreads();
   uint64_t* dst = mask + s0 * T;
   int32_t* ddst = depth ? depth + s0 * T : nullptr;
-  auto get = [&](int e) -> unsigned long long {
-    const int seq = e / T, node = e - seq * T;
-    return sMask[node * kMaskRowPitch + seq];
-  };
+  auto get = [&](const MaskElem& e) -> unsigned long long { return sMask[e.seq * kMaskSeqPitch + e.node]; };
   if ((n_elem & 1) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0 &&
       (!ddst || (reinterpret_cast<uintptr_t>(ddst) & 7u) == 0)) {
+    const int first = 2 * threadIdx.x, step = 2 * kMaskBlockThreads;
+    MaskElem e0 = {first / T, first % T};
+    const int dseq = step / T, dnode = step % T;
 #pragma unroll 2
     for (int q = threadIdx.x; q < (n_elem >> 1); q += kMaskBlockThreads) {   // two masks = 16 bytes per store
-      const unsigned long long m0 = get(2 * q), m1 = get(2 * q + 1);
+      const unsigned long long m0 = get(e0), m1 = get(e0.next(T));
       reinterpret_cast<ulonglong2*>(dst)[q] = make_ulonglong2(m0, m1);
       if (ddst) reinterpret_cast<int2*>(ddst)[q] = make_int2(__popcll(m0) - 1, __popcll(m1) - 1);
+      e0.advance(dseq, dnode, T);
     }
   } else {
+    MaskElem e0 = {static_cast<int>(threadIdx.x) / T, static_cast<int>(threadIdx.x) % T};
+    const int dseq = kMaskBlockThreads / T, dnode = kMaskBlockThreads % T;
     for (int e = threadIdx.x; e < n_elem; e += kMaskBlockThreads) {
-      const unsigned long long m = get(e);
+      const unsigned long long m = get(e0);
       dst[e] = m;
       if (ddst) ddst[e] = __popcll(m) - 1;
+      e0.advance(dseq, dnode, T);
     }
   }
 }

@@ -474,6 +474,14 @@ def test_tree_mask_large_batch_matches_oracle():
                 assert mask[b, i] == 0 and depth[b, i] == -1
             else:
                 assert mask[b, i] == ref_mask[idx[b], i] and depth[b, i] == ref_depth[idx[b], i]
+    # other node counts (49: copy loops that wrap a sequence boundary at odd offsets; 9: several sequences per step)
+    for name, nb in (("llama_tree", 2048 + 5), ("tiny_chain", 4096 + 2)):
+        c2 = gen.CONFIGS[name]
+        d2 = np.stack([gen.make_tree(dataclasses.replace(c2, seed=c2.seed + s), 0) for s in range(100)])
+        i2 = (np.arange(nb) * 7) % len(d2)
+        m2, dp2 = H.run_tree_mask(H.i32_dev(d2[i2].copy()))
+        rm2, rd2 = orc.build_tree_mask(d2)
+        assert np.array_equal(m2.cpu().numpy().view(np.uint64), rm2[i2]) and np.array_equal(dp2.cpu().numpy(), rd2[i2])
     chain = np.tile(np.arange(-1, 63, dtype=np.int32), (2048, 1))
     m, d = H.run_tree_mask(H.i32_dev(chain))
     cm, cd = orc.build_tree_mask(chain[:1])
