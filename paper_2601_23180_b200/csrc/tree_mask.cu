@@ -71,7 +71,8 @@ tree_mask_kernel(const int32_t* __restrict__ parent, uint64_t* __restrict__ mask
 // masks sit in shared memory sequence-major with an odd pitch: the walkers (one sequence per lane)
 // and the copy-out (consecutive elements per lane) both touch distinct banks.
 constexpr int kMaskBlockSeqs = 64, kMaskBlockThreads = 256;
-constexpr int kMaskParPitch = kMaskBlockSeqs + 4;   // bytes per node row of the parent table (bank spread)
+constexpr int kMaskParPitch = kMaskBlockSeqs + 1;   // bytes per node row of the parent table: a lane's four
+                                                    // consecutive nodes, and its neighbours' (4 nodes on), hit distinct banks
 constexpr int kMaskSeqPitch = 65;                   // masks per sequence row (T <= 64, odd)
 
 // element index e = seq * T + node, advanced by `step` elements
