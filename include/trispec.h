@@ -365,7 +365,13 @@ int trispec_sample_bonus(const trispec_sample_args* a, void* stream);
  * Fused pass: the four calls above on `stream` (one verification round of Algorithm 1 for
  * one verifier): tree mask first, acceptance scan last; the attention and the LM-head
  * statistics, which do not read each other's results, in the order the library finds faster
- * for the shape. `attn` may be NULL to skip attention.
+ * for the shape. `attn` may be NULL to skip attention. For one active sequence and a short
+ * context the library runs mask + attention on an internal second stream beside the LM head and
+ * the scan, and `stream` waits for that stream before the call returns its place in the queue:
+ * what the caller sees is unchanged (everything the call enqueues has completed before anything
+ * enqueued on `stream` afterwards starts), but no output buffer of the call may overlap an input
+ * of another step of the same call (the one case the library checks and serialises itself:
+ * scan->esc_index == attn->seq_index).
  * ------------------------------------------------------------------------------------- */
 int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                    const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream);

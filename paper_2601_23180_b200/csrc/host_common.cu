@@ -18,6 +18,7 @@ EntryScope::EntryScope() {
   if (tl_scope_depth++ == 0) tl_scope_launched = false;
 }
 EntryScope::~EntryScope() { --tl_scope_depth; }
+void entry_scope_next_launch_ordinary() { tl_scope_launched = false; }
 bool entry_scope_next_launch_is_dependent() {
   const bool dependent = tl_scope_depth > 0 && tl_scope_launched;
   tl_scope_launched = true;

@@ -52,6 +52,12 @@ struct EntryScope {
 // True if a kernel was already launched inside the current outermost scope (the next launch may
 // then be a programmatic dependent); records that a launch happens now.
 bool entry_scope_next_launch_is_dependent();
+// The next launch inside the current scope is an ordinary one again (after work was moved to or joined from
+// another stream, where "the kernel before it" is not the kernel enqueued last).
+void entry_scope_next_launch_ordinary();
+// SMs the single-sequence LM head leaves free on its next launch from this thread (0 = none); consumed by
+// that launch. The fused pass sets it when a small attention runs beside the LM head on a second stream.
+void lm_reserve_sms_once(int n);
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,

@@ -737,6 +737,8 @@ lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
 // One active sequence takes the W-on-M kernel (lmhead_rows_kernel): one CTA and one vocabulary range
 // per SM, LW_ROWS partial rows per range.
 static bool lm_rows_path(int n_seq) { return n_seq == 1; }
+static thread_local int tl_lm_reserved_sms = 0;
+void lm_reserve_sms_once(int n) { tl_lm_reserved_sms = n > 0 ? n : 0; }
 
 struct LmPlan {
   int n_seq, n_mt;
@@ -758,7 +760,9 @@ static int lm_plan(const trispec_lmhead_args* a, LmPlan* pl, size_t max_ws = ~st
   if (lm_rows_path(pl->n_seq)) {
     pl->n_mt = 1;
     const int V16 = (a->V + 15) / 16;
-    pl->n_ranges = device_sm_count() < V16 ? device_sm_count() : V16;
+    int sms = device_sm_count() - tl_lm_reserved_sms;
+    if (sms < 1) sms = 1;
+    pl->n_ranges = sms < V16 ? sms : V16;
     return TRISPEC_OK;
   }
   pl->n_mt = (pl->n_seq + 3) / 4;
@@ -818,8 +822,10 @@ extern "C" int trispec_lmhead_stats(const trispec_lmhead_args* a, void* stream) 
   using namespace trispec;
   LmPlan pl;
   int rc = lm_plan(a, &pl);
+  const size_t ws_needed = trispec_lmhead_stats_workspace(a);
+  tl_lm_reserved_sms = 0;            // a reservation holds for one call
   if (rc != TRISPEC_OK) return rc;
-  return lmhead_stats_planned(a, pl, trispec_lmhead_stats_workspace(a), stream);
+  return lmhead_stats_planned(a, pl, ws_needed, stream);
 }
 
 static int trispec::lmhead_stats_planned(const trispec_lmhead_args* a, const LmPlan& pl, size_t ws_needed, void* stream) {

@@ -4,34 +4,6 @@
 
 #include "host_common.h"
 
-extern "C" int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
-                              const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream) {
-  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
-  if (!tree || !lm || !scan) return TRISPEC_ERR_INVALID_ARG;
-  int rc = trispec_build_tree_mask(tree, stream);
-  if (rc != TRISPEC_OK) return rc;
-  // The attention and the LM head do not depend on each other, so their order is free. A kernel launched as
-  // a programmatic dependent gets its launch latency and prologue hidden, but its loads make almost no
-  // progress while the kernel before it still runs (measured: the stages of the single-sequence LM head
-  // arrive within a microsecond of the attention's end, whenever it started). For one active sequence the
-  // LM head is a pure stream of W: behind an attention that fills a good part of the chip it loses more
-  // than the hidden latency (one sequence of 4096 context tokens: 166 us against 156 us the other way
-  // round), behind a small one (16 CTAs, 14 us) it still gains (59 against 63 us).
-  const int lm_seqs = lm->seq_index ? lm->B_active : lm->B;
-  const bool lm_first = attn && lm_seqs == 1 && trispec::attn_planned_ctas(attn) > trispec::device_sm_count() / 4;
-  if (attn && !lm_first) {
-    rc = trispec_verify_attn(attn, stream);
-    if (rc != TRISPEC_OK) return rc;
-  }
-  rc = trispec_lmhead_stats(lm, stream);
-  if (rc != TRISPEC_OK) return rc;
-  if (lm_first) {
-    rc = trispec_verify_attn(attn, stream);
-    if (rc != TRISPEC_OK) return rc;
-  }
-  return trispec_accept_scan(scan, stream);
-}
-
 namespace trispec {
 // Side stream and events of trispec_verify_host, one set per device, created on first use.
 struct HostPassStreams {
@@ -58,6 +30,68 @@ static int host_pass_streams(HostPassStreams** out) {
   return TRISPEC_OK;
 }
 }  // namespace trispec
+
+extern "C" int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
+                              const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream) {
+  trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
+  if (!tree || !lm || !scan) return TRISPEC_ERR_INVALID_ARG;
+  // The attention and the LM head do not depend on each other, so their order is free. A kernel launched as
+  // a programmatic dependent gets its launch latency and prologue hidden, but its loads make almost no
+  // progress while the kernel before it still runs (measured: the stages of the single-sequence LM head
+  // arrive within a microsecond of the attention's end, whenever it started). For one active sequence the
+  // LM head is a pure stream of W: behind an attention that fills a good part of the chip it loses more
+  // than the hidden latency (one sequence of 4096 context tokens: 166 us against 156 us the other way
+  // round), so there the LM head goes first.
+  const int lm_seqs = lm->seq_index ? lm->B_active : lm->B;
+  const int attn_ctas = attn ? trispec::attn_planned_ctas(attn) : 0;
+  const bool lm_first = attn && lm_seqs == 1 && attn_ctas > trispec::device_sm_count() / 4;
+  int rc;
+  // One active sequence and a small attention (a short context: a few CTAs for 10-20 us, all latency): the
+  // two run side by side. Mask and attention go to a second stream behind an event recorded on `stream` at the
+  // start of the call; the LM head, whose grid is one persistent CTA per SM, leaves them one SM per attention
+  // CTA and starts at once, the scan follows it, and `stream` then waits for the second stream: everything
+  // the call enqueues is complete before anything enqueued on `stream` after it.
+  // (not when the scan's escalation list is written over the index list the attention reads: in stream
+  // order the scan comes last, side by side it would not)
+  const bool in_place_list = attn && attn->seq_index && scan->esc_index == attn->seq_index;
+  if (attn && lm_seqs == 1 && attn_ctas > 0 && attn_ctas * 8 <= trispec::device_sm_count() && !in_place_list) {
+    using namespace trispec;
+    HostPassStreams* hs = nullptr;
+    rc = host_pass_streams(&hs);
+    if (rc != TRISPEC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::unique_lock<std::mutex> enqueue_lock(hs->enqueue);
+    TRISPEC_CUDA_OK(cudaEventRecord(hs->fork, st));
+    TRISPEC_CUDA_OK(cudaStreamWaitEvent(hs->copy, hs->fork, 0));
+    rc = trispec_build_tree_mask(tree, hs->copy);          // ordinary launch: first kernel of the call
+    if (rc != TRISPEC_OK) return rc;
+    rc = trispec_verify_attn(attn, hs->copy);              // dependent of the mask kernel
+    if (rc != TRISPEC_OK) return rc;
+    TRISPEC_CUDA_OK(cudaEventRecord(hs->copied, hs->copy));
+    entry_scope_next_launch_ordinary();                    // first kernel on `stream`
+    lm_reserve_sms_once(attn_ctas);
+    rc = trispec_lmhead_stats(lm, stream);
+    lm_reserve_sms_once(0);
+    if (rc != TRISPEC_OK) return rc;
+    rc = trispec_accept_scan(scan, stream);                // dependent of the LM head's last kernel
+    if (rc != TRISPEC_OK) return rc;
+    TRISPEC_CUDA_OK(cudaStreamWaitEvent(st, hs->copied, 0));
+    return TRISPEC_OK;
+  }
+  rc = trispec_build_tree_mask(tree, stream);
+  if (rc != TRISPEC_OK) return rc;
+  if (attn && !lm_first) {
+    rc = trispec_verify_attn(attn, stream);
+    if (rc != TRISPEC_OK) return rc;
+  }
+  rc = trispec_lmhead_stats(lm, stream);
+  if (rc != TRISPEC_OK) return rc;
+  if (lm_first) {
+    rc = trispec_verify_attn(attn, stream);
+    if (rc != TRISPEC_OK) return rc;
+  }
+  return trispec_accept_scan(scan, stream);
+}
 
 // The host-buffer form of the pass. The LM head needs only h (and the tree), the attention
 // needs q and the tree keys/values: the latter are copied on a side stream while the LM-head

@@ -267,3 +267,50 @@ def test_host_pass_rejects_argument_structs_of_different_passes():
     pas.run_host()
     torch.cuda.synchronize()
     assert int(pas.status.item()) == 0
+
+
+def test_single_sequence_pass_with_its_attention_on_the_second_stream_stays_one_ordered_unit():
+    """One active sequence with a short context: the fused pass runs mask + attention on the library's
+    second stream beside the LM head. Inputs written on the caller's stream just before the call must be
+    seen by both sides, and work enqueued on that stream right after the call must see every output."""
+    import torch
+    from paper_2601_23180_b200 import binding as ts, runner
+    cfg = gen.small_variant(gen.CONFIGS["tiny_chain"], V=4096, d=256, L=700, seed=31,
+                            logit_scale=3.6 / (0.02 * math.sqrt(256)))
+    inp = gen.make_inputs(cfg)
+    pas = runner.VerifyPass(cfg, inp)
+    assert ts.trispec_verify_attn_plan(pas.attn_args) in ("cluster", "splits")
+    # reference: the four steps one after the other, synchronised
+    ts.trispec_build_tree_mask(pas.tree_args)
+    ts.trispec_verify_attn(pas.attn_args)
+    ts.trispec_lmhead_stats(pas.lm_args)
+    ts.trispec_accept_scan(pas.scan_args)
+    torch.cuda.synchronize()
+    want = {"o": pas.o.clone(), "mask": pas.mask.clone(), "top1": pas.stats["top1_idx"].clone(),
+            "lse": pas.stats["lse"].clone(), "acc": pas.scan_out["accept_len"].clone(),
+            "path": pas.scan_out["path"].clone()}
+    ref_o, _ = orc.verify_attn(inp["q"], inp["k_tree"], inp["v_tree"], orc.build_tree_mask(inp["parent"])[0],
+                               inp["k_cache"], inp["v_cache"], inp["ctx_len"], 1.0 / math.sqrt(cfg.D))
+    assert np.abs(want["o"].float().cpu().numpy() - ref_o).max() <= 2e-2
+    q_good, h_good, parent_good = pas.dev["q"].clone(), pas.dev["h"].clone(), pas.dev["parent"].clone()
+    side = torch.cuda.Stream()
+    for rep in range(20):
+        with torch.cuda.stream(side):
+            # spoil the inputs and the outputs, then restore the inputs on the same stream right before the call
+            pas.dev["q"].zero_(); pas.dev["h"].zero_(); pas.dev["parent"].fill_(-1)
+            pas.o.fill_(float("nan")); pas.mask.zero_(); pas.stats["top1_idx"].fill_(-7)
+            pas.scan_out["accept_len"].fill_(-9)
+            big = torch.empty(64 << 20, dtype=torch.uint8, device="cuda"); big.zero_()   # keeps the stream busy
+            pas.dev["q"].copy_(q_good); pas.dev["h"].copy_(h_good); pas.dev["parent"].copy_(parent_good)
+            pas.run(side)
+            got = {"o": pas.o.clone(), "mask": pas.mask.clone(), "top1": pas.stats["top1_idx"].clone(),
+                   "lse": pas.stats["lse"].clone(), "acc": pas.scan_out["accept_len"].clone(),
+                   "path": pas.scan_out["path"].clone()}
+        side.synchronize()
+        for k in want:
+            a, b = got[k], want[k]
+            if a.dtype.is_floating_point:
+                assert torch.equal(torch.nan_to_num(a.float(), nan=-1.0), torch.nan_to_num(b.float(), nan=-1.0)), (k, rep)
+            else:
+                assert torch.equal(a, b), (k, rep)
+    assert int(pas.status.item()) == 0
