@@ -8,7 +8,7 @@ namespace trispec {
 // Side stream and events of trispec_verify_host, one set per device, created on first use.
 struct HostPassStreams {
   cudaStream_t copy = nullptr;
-  cudaEvent_t fork = nullptr, copied = nullptr;
+  cudaEvent_t fork = nullptr, copied = nullptr, inputs = nullptr;
   bool ready = false;
   std::mutex enqueue;   // the stream and the events are shared by every caller on this device
 };
@@ -24,6 +24,7 @@ static int host_pass_streams(HostPassStreams** out) {
     if (cudaStreamCreateWithFlags(&h.copy, cudaStreamNonBlocking) != cudaSuccess) return TRISPEC_ERR_CUDA;
     if (cudaEventCreateWithFlags(&h.fork, cudaEventDisableTiming) != cudaSuccess) return TRISPEC_ERR_CUDA;
     if (cudaEventCreateWithFlags(&h.copied, cudaEventDisableTiming) != cudaSuccess) return TRISPEC_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&h.inputs, cudaEventDisableTiming) != cudaSuccess) return TRISPEC_ERR_CUDA;
     h.ready = true;
   }
   *out = &h;
@@ -151,25 +152,50 @@ extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree
                      {const_cast<void*>(lm->h), io->h, BT * static_cast<size_t>(lm->d) * 2}};
     TRISPEC_CUDA_OK(copy_list(in, 3, cudaMemcpyHostToDevice, st));
   }
+  const int lm_seqs = lm->seq_index ? lm->B_active : lm->B;
+  const int attn_ctas = attn ? attn_planned_ctas(attn) : 0;
+  const bool side_by_side = attn && lm_seqs == 1 && attn_ctas > 0 && attn_ctas * 8 <= device_sm_count() &&
+                            !(attn->seq_index && scan->esc_index == attn->seq_index);
+  if (side_by_side) TRISPEC_CUDA_OK(cudaEventRecord(hs->inputs, st));
   if (attn) {
     TRISPEC_CUDA_OK(cudaStreamWaitEvent(hs->copy, hs->fork, 0));
     CopyReq in[3] = {{const_cast<void*>(attn->q), io->q, BT * static_cast<size_t>(attn->Hq) * attn->D * 2},
                      {const_cast<void*>(attn->k_tree), io->k_tree, BT * static_cast<size_t>(attn->Hkv) * attn->D * 2},
                      {const_cast<void*>(attn->v_tree), io->v_tree, BT * static_cast<size_t>(attn->Hkv) * attn->D * 2}};
     TRISPEC_CUDA_OK(copy_list(in, 3, cudaMemcpyHostToDevice, hs->copy));
-    TRISPEC_CUDA_OK(cudaEventRecord(hs->copied, hs->copy));
+    if (!side_by_side) TRISPEC_CUDA_OK(cudaEventRecord(hs->copied, hs->copy));
   }
-  int rc = trispec_build_tree_mask(tree, stream);
-  if (rc != TRISPEC_OK) return rc;
-  rc = trispec_lmhead_stats(lm, stream);
-  if (rc != TRISPEC_OK) return rc;
-  if (attn) {
+  int rc;
+  if (side_by_side) {
+    // one active sequence, short context (as in trispec_verify): mask and attention follow their inputs on
+    // the second stream, the LM head and the scan run on `stream`, which then waits for the second stream
+    TRISPEC_CUDA_OK(cudaStreamWaitEvent(hs->copy, hs->inputs, 0));   // the tree's parents have arrived
+    rc = trispec_build_tree_mask(tree, hs->copy);
+    if (rc != TRISPEC_OK) return rc;
+    rc = trispec_verify_attn(attn, hs->copy);
+    if (rc != TRISPEC_OK) return rc;
+    TRISPEC_CUDA_OK(cudaEventRecord(hs->copied, hs->copy));
+    entry_scope_next_launch_ordinary();                              // first kernel on `stream`
+    lm_reserve_sms_once(attn_ctas);
+    rc = trispec_lmhead_stats(lm, stream);
+    lm_reserve_sms_once(0);
+    if (rc != TRISPEC_OK) return rc;
+    rc = trispec_accept_scan(scan, stream);
+    if (rc != TRISPEC_OK) return rc;
     TRISPEC_CUDA_OK(cudaStreamWaitEvent(st, hs->copied, 0));
-    rc = trispec_verify_attn(attn, stream);
+  } else {
+    rc = trispec_build_tree_mask(tree, stream);
+    if (rc != TRISPEC_OK) return rc;
+    rc = trispec_lmhead_stats(lm, stream);
+    if (rc != TRISPEC_OK) return rc;
+    if (attn) {
+      TRISPEC_CUDA_OK(cudaStreamWaitEvent(st, hs->copied, 0));
+      rc = trispec_verify_attn(attn, stream);
+      if (rc != TRISPEC_OK) return rc;
+    }
+    rc = trispec_accept_scan(scan, stream);
     if (rc != TRISPEC_OK) return rc;
   }
-  rc = trispec_accept_scan(scan, stream);
-  if (rc != TRISPEC_OK) return rc;
   const size_t B = static_cast<size_t>(scan->B);
   CopyReq out[5] = {{io->accept_len, scan->accept_len, B * 4},
                     {io->bonus_tok, scan->bonus_tok, B * 4},

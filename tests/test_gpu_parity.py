@@ -318,6 +318,10 @@ PASS_CASES = [
     ("target_escalated", dict(B=5, n_active=2, L=300, V=6000, d=320, Hq=32, rho=0.3)),
     ("llama_tree", dict(B=3, L=260, V=9000, d=128, rho=0.3)),
     ("long_paged", dict(B=6, L=900, L_min=100, V=5000, d=192, rho=0.3)),
+    # one active sequence: a short context (mask + attention beside the LM head on the library's second
+    # stream; the sequence picked through seq_index) and a long one (LM head first, then the attention)
+    ("target_escalated", dict(B=4, n_active=1, L=300, V=6000, d=320, Hq=32, rho=0.3)),
+    ("proxy_tree", dict(B=1, L=4096, V=20000, d=256, rho=0.3)),
 ]
 
 
