@@ -375,6 +375,12 @@ int trispec_sample_bonus(const trispec_sample_args* a, void* stream);
  * ------------------------------------------------------------------------------------- */
 int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                    const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream);
+/* How a pass with these arguments arranges its attention and its LM head (a diagnostic; host only,
+ * nothing is launched; `attn` and `scan` may be NULL): "attention_first", "lm_first" (one active
+ * sequence behind a chip-filling attention) or "side_by_side" (one active sequence, short context:
+ * the second-stream form described above); "none" without `lm`. */
+const char* trispec_verify_plan(const trispec_attn_args* attn, const trispec_lmhead_args* lm,
+                                const trispec_scan_args* scan);
 
 /* ---------------------------------------------------------------------------------------
  * The same pass for callers whose per-round data lives in HOST memory (one verification

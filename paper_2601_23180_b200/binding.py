@@ -93,6 +93,8 @@ _lib.trispec_build_tree_mask.argtypes = [C.POINTER(TreeArgs), _vp]
 _lib.trispec_verify_attn_workspace.restype = _sz
 _lib.trispec_verify_attn_workspace.argtypes = [C.POINTER(AttnArgs)]
 _lib.trispec_verify_attn.argtypes = [C.POINTER(AttnArgs), _vp]
+_lib.trispec_verify_plan.restype = C.c_char_p
+_lib.trispec_verify_plan.argtypes = [C.POINTER(AttnArgs), C.POINTER(LmheadArgs), C.POINTER(ScanArgs)]
 _lib.trispec_verify_attn_plan.restype = C.c_char_p
 _lib.trispec_verify_attn_plan.argtypes = [C.POINTER(AttnArgs)]
 _lib.trispec_lmhead_stats_workspace.restype = _sz
@@ -111,7 +113,7 @@ _lib.trispec_verify.argtypes = [C.POINTER(TreeArgs), C.POINTER(AttnArgs), C.POIN
 _lib.trispec_verify_host.argtypes = [C.POINTER(HostIO), C.POINTER(TreeArgs), C.POINTER(AttnArgs),
                                      C.POINTER(LmheadArgs), C.POINTER(ScanArgs), _vp]
 
-EXPORTS = ["trispec_verify_host", "trispec_verify_attn_plan", "trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
+EXPORTS = ["trispec_verify_host", "trispec_verify_plan", "trispec_verify_attn_plan", "trispec_status_string", "trispec_launch_count", "trispec_build_tree_mask",
            "trispec_verify_attn_workspace", "trispec_verify_attn", "trispec_lmhead_stats_workspace",
            "trispec_lmhead_stats", "trispec_lmhead_stats_noalloc", "trispec_accept_scan", "trispec_verify",
            "trispec_prune_tree", "trispec_commit_kv", "trispec_sample_bonus_workspace", "trispec_sample_bonus"]
@@ -350,6 +352,11 @@ def trispec_verify_attn_workspace(args: AttnArgs) -> int:
 
 def trispec_verify_attn_plan(args: AttnArgs) -> str:
     return _lib.trispec_verify_attn_plan(C.byref(args)).decode()
+
+
+def trispec_verify_plan(attn: Optional[AttnArgs], lm: LmheadArgs, scan: Optional[ScanArgs] = None) -> str:
+    return _lib.trispec_verify_plan(C.byref(attn) if attn is not None else None, C.byref(lm),
+                                    C.byref(scan) if scan is not None else None).decode()
 
 
 def trispec_verify_attn(args: AttnArgs, stream=None):

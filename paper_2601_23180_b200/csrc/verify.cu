@@ -32,6 +32,34 @@ static int host_pass_streams(HostPassStreams** out) {
 }
 }  // namespace trispec
 
+namespace trispec {
+// How a pass arranges its attention and its LM head (they do not depend on each other).
+enum PassForm { PASS_ATTENTION_FIRST = 0, PASS_LM_FIRST = 1, PASS_SIDE_BY_SIDE = 2 };
+static PassForm pass_form(const trispec_attn_args* attn, const trispec_lmhead_args* lm, const trispec_scan_args* scan,
+                          int* attn_ctas_out) {
+  const int lm_seqs = lm->seq_index ? lm->B_active : lm->B;
+  const int attn_ctas = attn ? attn_planned_ctas(attn) : 0;
+  if (attn_ctas_out) *attn_ctas_out = attn_ctas;
+  if (!attn || lm_seqs != 1 || attn_ctas <= 0) return PASS_ATTENTION_FIRST;
+  // not side by side when the scan's escalation list is written over the index list the attention reads:
+  // in stream order the scan comes last, side by side it would not
+  const bool in_place_list = attn->seq_index && scan && scan->esc_index == attn->seq_index;
+  if (attn_ctas * 8 <= device_sm_count() && !in_place_list) return PASS_SIDE_BY_SIDE;
+  if (attn_ctas * 4 > device_sm_count()) return PASS_LM_FIRST;
+  return PASS_ATTENTION_FIRST;
+}
+}  // namespace trispec
+
+extern "C" const char* trispec_verify_plan(const trispec_attn_args* attn, const trispec_lmhead_args* lm,
+                                           const trispec_scan_args* scan) {
+  if (!lm) return "none";
+  switch (trispec::pass_form(attn, lm, scan, nullptr)) {
+    case trispec::PASS_LM_FIRST: return "lm_first";
+    case trispec::PASS_SIDE_BY_SIDE: return "side_by_side";
+    default: return "attention_first";
+  }
+}
+
 extern "C" int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                               const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream) {
   trispec::EntryScope entry_scope;   // the first kernel launched below is an ordinary launch
@@ -43,19 +71,16 @@ extern "C" int trispec_verify(const trispec_tree_args* tree, const trispec_attn_
   // LM head is a pure stream of W: behind an attention that fills a good part of the chip it loses more
   // than the hidden latency (one sequence of 4096 context tokens: 166 us against 156 us the other way
   // round), so there the LM head goes first.
-  const int lm_seqs = lm->seq_index ? lm->B_active : lm->B;
-  const int attn_ctas = attn ? trispec::attn_planned_ctas(attn) : 0;
-  const bool lm_first = attn && lm_seqs == 1 && attn_ctas > trispec::device_sm_count() / 4;
+  int attn_ctas = 0;
+  const trispec::PassForm form = trispec::pass_form(attn, lm, scan, &attn_ctas);
+  const bool lm_first = form == trispec::PASS_LM_FIRST;
   int rc;
   // One active sequence and a small attention (a short context: a few CTAs for 10-20 us, all latency): the
   // two run side by side. Mask and attention go to a second stream behind an event recorded on `stream` at the
   // start of the call; the LM head, whose grid is one persistent CTA per SM, leaves them one SM per attention
   // CTA and starts at once, the scan follows it, and `stream` then waits for the second stream: everything
   // the call enqueues is complete before anything enqueued on `stream` after it.
-  // (not when the scan's escalation list is written over the index list the attention reads: in stream
-  // order the scan comes last, side by side it would not)
-  const bool in_place_list = attn && attn->seq_index && scan->esc_index == attn->seq_index;
-  if (attn && lm_seqs == 1 && attn_ctas > 0 && attn_ctas * 8 <= trispec::device_sm_count() && !in_place_list) {
+  if (form == trispec::PASS_SIDE_BY_SIDE) {
     using namespace trispec;
     HostPassStreams* hs = nullptr;
     rc = host_pass_streams(&hs);
@@ -152,10 +177,8 @@ extern "C" int trispec_verify_host(const trispec_host_io* io, const trispec_tree
                      {const_cast<void*>(lm->h), io->h, BT * static_cast<size_t>(lm->d) * 2}};
     TRISPEC_CUDA_OK(copy_list(in, 3, cudaMemcpyHostToDevice, st));
   }
-  const int lm_seqs = lm->seq_index ? lm->B_active : lm->B;
-  const int attn_ctas = attn ? attn_planned_ctas(attn) : 0;
-  const bool side_by_side = attn && lm_seqs == 1 && attn_ctas > 0 && attn_ctas * 8 <= device_sm_count() &&
-                            !(attn->seq_index && scan->esc_index == attn->seq_index);
+  int attn_ctas = 0;
+  const bool side_by_side = pass_form(attn, lm, scan, &attn_ctas) == PASS_SIDE_BY_SIDE;
   if (side_by_side) TRISPEC_CUDA_OK(cudaEventRecord(hs->inputs, st));
   if (attn) {
     TRISPEC_CUDA_OK(cudaStreamWaitEvent(hs->copy, hs->fork, 0));

@@ -62,3 +62,29 @@ def test_lmhead_workspace_shows_the_kernel_choice():
     assert ts.trispec_lmhead_stats_workspace(args(1, 9, 64, 200)) == 13 * 64 * 32
     # unsupported shapes plan nothing
     assert ts.trispec_lmhead_stats_workspace(args(1, 65, 2048, 32000)) == 0
+
+
+def test_pass_form_follows_the_active_sequences_and_the_size_of_the_attention():
+    def lm_args(B, n_active=None):
+        a = ts.LmheadArgs()
+        a.B, a.T, a.d, a.V, a.logit_scale = B, 61, 2048, 151936, 1.0
+        a.B_active = 0 if n_active is None else n_active
+        a.seq_index = None if n_active is None else 1
+        return a
+    one = gen.small_variant
+    # batches: attention, then LM head
+    assert ts.trispec_verify_plan(_attn_args(gen.CONFIGS["proxy_tree"]), lm_args(8)) == "attention_first"
+    assert ts.trispec_verify_plan(None, lm_args(1)) == "attention_first"
+    # one sequence, 512 context tokens: 8 KV heads x 2 splits = 16 CTAs, an eighth of 148 SMs or less
+    assert ts.trispec_verify_plan(_attn_args(gen.CONFIGS["tiny_chain"]), lm_args(1)) == "side_by_side"
+    # one sequence, 4096 context tokens: 64 CTAs, more than a quarter of the chip
+    assert ts.trispec_verify_plan(_attn_args(one(gen.CONFIGS["proxy_tree"], B=1)), lm_args(1)) == "lm_first"
+    # one ACTIVE sequence of several, picked through an index list
+    a = _attn_args(one(gen.CONFIGS["tiny_chain"], B=4), n_active=1)
+    assert ts.trispec_verify_plan(a, lm_args(4, n_active=1)) == "side_by_side"
+    # ... unless the scan writes its escalation list over that index list: then in stream order
+    s = ts.ScanArgs()
+    s.esc_index = 1
+    assert ts.trispec_verify_plan(a, lm_args(4, n_active=1), s) == "attention_first"
+    s.esc_index = 2
+    assert ts.trispec_verify_plan(a, lm_args(4, n_active=1), s) == "side_by_side"
