@@ -78,11 +78,10 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
       nr1 = fabsf(f - a.lambda) < 1e-3f;
     }
   }
-  // the margin test of every node as one bit (Eq. 8), known to the whole warp
-  const unsigned long long trusted =
-      __ballot_sync(0xffffffffu, tr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, tr1)) << 32);
-  const unsigned long long near_bits =
-      __ballot_sync(0xffffffffu, nr0) | (static_cast<unsigned long long>(__ballot_sync(0xffffffffu, nr1)) << 32);
+  // the margin test (Eq. 8) and the near-threshold mark of this lane's two nodes as four bits; the walk
+  // fetches them from the current node's lane together with its top-1 (cur is the same in every lane, so
+  // each lane picks its low or high node BEFORE the shuffle: one shuffle per value and step)
+  const int flags = (tr0 ? 1 : 0) | (tr1 ? 2 : 0) | (nr0 ? 4 : 0) | (nr1 ? 8 : 0);
   // Bernoulli acceptance of Eq. 6 for every node at once: bit c = child c passes its test
   unsigned long long passes = ~0ull;
   if (stochastic) {
@@ -107,18 +106,18 @@ __device__ __forceinline__ int scan_sequence(const trispec_scan_args& a, const l
   // each accepted node has a larger index than the previous one: at most T iterations
   for (int it = 0; it < T; ++it) {
     const int src = cur & 31;
-    const int t_lo = __shfl_sync(0xffffffffu, top0, src), t_hi = __shfl_sync(0xffffffffu, top1v, src);
-    const int top1 = (cur < 32) ? t_lo : t_hi;
+    const bool hi = cur >= 32;
+    const int top1 = __shfl_sync(0xffffffffu, hi ? top1v : top0, src);
     if (proxy) {
-      near += static_cast<int>((near_bits >> cur) & 1ull);
-      if (!((trusted >> cur) & 1ull)) { esc = 1; break; }
+      const int fl = __shfl_sync(0xffffffffu, flags, src) >> (hi ? 1 : 0);
+      near += (fl >> 2) & 1;
+      if (!(fl & 1)) { esc = 1; break; }
     }
     // greedy: the child whose token is the arg-max; stochastic: the first child that passed its
     // Bernoulli test; token-specific: the first child at least (1 - alpha) as probable as the arg-max
     unsigned m0, m1;
     if (token_rule) {
-      const float p_lo = __shfl_sync(0xffffffffu, pt0, src), p_hi = __shfl_sync(0xffffffffu, pt1, src);
-      const float bar = (1.f - a.alpha) * ((cur < 32) ? p_lo : p_hi);
+      const float bar = (1.f - a.alpha) * __shfl_sync(0xffffffffu, hi ? pt1 : pt0, src);
       m0 = __ballot_sync(0xffffffffu, par0 == cur && pd0 >= bar);
       m1 = __ballot_sync(0xffffffffu, par1 == cur && pd1 >= bar);
     } else {
