@@ -516,6 +516,92 @@ struct LmRowsParams {
 
 struct LmColStats { float m, s, t, v1, v2; int i1, i2; };
 
+// One 32-column chunk of a tile in the epilogue of lmhead_rows_kernel: r[j] = logit of column col0 + j at this
+// lane's vocabulary entry my_v. Per column: top-2 (value, vocabulary index) and the sum of exponentials over
+// the warp's 32 vocabulary entries, folded into the running statistics `run` of column col0 + lane. A
+// transposing butterfly does all columns at once: in the step with distance o a lane keeps half of the
+// columns it still holds, hands the other half to its partner and merges what it receives, so that after
+// the steps lane l holds column l. NC = 32 columns take five steps; when the tree has at most 16 nodes
+// (NC = 16: chains), four steps leave lanes l and l + 16 with column l over one half of the entries each,
+// and one more exchange merges the halves (lanes 16-31 then hold copies, which nothing reads).
+template <bool kEntropy, int NC>
+__device__ __forceinline__ void lm_rows_chunk_nc(const uint32_t (&r)[32], bool valid, int my_v, int col0, int N, int lane,
+                                                 float c, LmColStats& run) {
+  float v1[NC], v2[NC];
+  int i1[NC], i2[NC];
+#pragma unroll
+  for (int j = 0; j < NC; ++j) {
+    const bool on = valid && (col0 + j < N);
+    v1[j] = on ? __uint_as_float(r[j]) : -INFINITY;
+    i1[j] = on ? my_v : -1;
+    v2[j] = -INFINITY;
+    i2[j] = -1;
+  }
+#pragma unroll
+  for (int o = NC / 2; o > 0; o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      const float sv1 = up ? v1[i] : v1[i + o], sv2 = up ? v2[i] : v2[i + o];
+      const int si1 = up ? i1[i] : i1[i + o], si2 = up ? i2[i] : i2[i + o];
+      float kv1 = up ? v1[i + o] : v1[i], kv2 = up ? v2[i + o] : v2[i];
+      int ki1 = up ? i1[i + o] : i1[i], ki2 = up ? i2[i + o] : i2[i];
+      const float rv1 = __shfl_xor_sync(0xffffffffu, sv1, o), rv2 = __shfl_xor_sync(0xffffffffu, sv2, o);
+      const int ri1 = __shfl_xor_sync(0xffffffffu, si1, o), ri2 = __shfl_xor_sync(0xffffffffu, si2, o);
+      lm_top2_insert(rv1, ri1, kv1, ki1, kv2, ki2);
+      lm_top2_insert(rv2, ri2, kv1, ki1, kv2, ki2);
+      v1[i] = kv1; v2[i] = kv2; i1[i] = ki1; i2[i] = ki2;
+    }
+  }
+  if (NC == 16) {   // lanes l and l ^ 16 hold the same column over different vocabulary entries
+    const float rv1 = __shfl_xor_sync(0xffffffffu, v1[0], 16), rv2 = __shfl_xor_sync(0xffffffffu, v2[0], 16);
+    const int ri1 = __shfl_xor_sync(0xffffffffu, i1[0], 16), ri2 = __shfl_xor_sync(0xffffffffu, i2[0], 16);
+    lm_top2_insert(rv1, ri1, v1[0], i1[0], v2[0], i2[0]);
+    lm_top2_insert(rv2, ri2, v1[0], i1[0], v2[0], i2[0]);
+  }
+  const float m_t = v1[0];                  // this lane's column: col0 + (lane mod NC)
+  // every lane needs every column's maximum for its exponentials
+  float es[NC], et[NC];
+#pragma unroll
+  for (int j = 0; j < NC; ++j) {
+    const float mj = __shfl_sync(0xffffffffu, m_t, j);
+    const bool on = valid && (col0 + j < N);
+    const float z = __uint_as_float(r[j]);
+    es[j] = on ? ex2f((z - mj) * c) : 0.f;
+    et[j] = (kEntropy && on) ? es[j] * z : 0.f;
+  }
+#pragma unroll
+  for (int o = NC / 2; o > 0; o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      const float ss = up ? es[i] : es[i + o], ks = up ? es[i + o] : es[i];
+      es[i] = ks + __shfl_xor_sync(0xffffffffu, ss, o);
+      if (kEntropy) {
+        const float st2 = up ? et[i] : et[i + o], kt = up ? et[i + o] : et[i];
+        et[i] = kt + __shfl_xor_sync(0xffffffffu, st2, o);
+      }
+    }
+  }
+  if (NC == 16) {
+    es[0] += __shfl_xor_sync(0xffffffffu, es[0], 16);
+    if (kEntropy) et[0] += __shfl_xor_sync(0xffffffffu, et[0], 16);
+  }
+  // fold the tile's statistics of this lane's column into the running ones
+  LmRowAcc a = {run.m, run.s, run.t};
+  lm_fold(a, m_t, es[0], et[0], c);
+  run.m = a.m; run.s = a.s; run.t = a.t;
+  lm_top2_insert(v1[0], i1[0], run.v1, run.i1, run.v2, run.i2);
+  lm_top2_insert(v2[0], i2[0], run.v1, run.i1, run.v2, run.i2);
+}
+template <bool kEntropy>
+__device__ __forceinline__ void lm_rows_chunk(const uint32_t (&r)[32], bool valid, int my_v, int col0, int N, int lane,
+                                              float c, LmColStats& run) {
+  if (N <= 16) lm_rows_chunk_nc<kEntropy, 16>(r, valid, my_v, col0, N, lane, c, run);
+  else lm_rows_chunk_nc<kEntropy, 32>(r, valid, my_v, col0, N, lane, c, run);
+}
+
+
 template <bool kEntropy, int KPS>
 __global__ void __launch_bounds__(LW_THREADS, 1)
 lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_wt,
@@ -636,69 +722,7 @@ lmhead_rows_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
           __syncwarp();
           if (lane == 0) mbar_arrive(tmem_empty + buf);
         }
-        // Per column: top-2 (value, vocabulary index) and the sum of exponentials over this warp's 32
-        // vocabulary entries. A transposing butterfly does all 32 columns at once: in the step with
-        // distance o a lane keeps half of the columns it still holds, hands the other half to its
-        // partner and merges what it receives, so that after five steps lane l holds column l.
-        const int my_v = v_lane0 + lane;
-        float v1[32], v2[32];
-        int i1[32], i2[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const bool on = valid && (h * 32 + j < sp.N);
-          v1[j] = on ? __uint_as_float(r[j]) : -INFINITY;
-          i1[j] = on ? my_v : -1;
-          v2[j] = -INFINITY;
-          i2[j] = -1;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const bool up = (lane & o) != 0;
-#pragma unroll
-          for (int i = 0; i < o; ++i) {
-            const float sv1 = up ? v1[i] : v1[i + o], sv2 = up ? v2[i] : v2[i + o];
-            const int si1 = up ? i1[i] : i1[i + o], si2 = up ? i2[i] : i2[i + o];
-            float kv1 = up ? v1[i + o] : v1[i], kv2 = up ? v2[i + o] : v2[i];
-            int ki1 = up ? i1[i + o] : i1[i], ki2 = up ? i2[i + o] : i2[i];
-            const float rv1 = __shfl_xor_sync(0xffffffffu, sv1, o), rv2 = __shfl_xor_sync(0xffffffffu, sv2, o);
-            const int ri1 = __shfl_xor_sync(0xffffffffu, si1, o), ri2 = __shfl_xor_sync(0xffffffffu, si2, o);
-            lm_top2_insert(rv1, ri1, kv1, ki1, kv2, ki2);
-            lm_top2_insert(rv2, ri2, kv1, ki1, kv2, ki2);
-            v1[i] = kv1; v2[i] = kv2; i1[i] = ki1; i2[i] = ki2;
-          }
-        }
-        const float m_t = v1[0];                  // this lane's column: h * 32 + lane
-        // every lane needs every column's maximum for its exponentials
-        float es[32], et[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float mj = __shfl_sync(0xffffffffu, m_t, j);
-          const bool on = valid && (h * 32 + j < sp.N);
-          const float z = __uint_as_float(r[j]);
-          es[j] = on ? ex2f((z - mj) * c) : 0.f;
-          et[j] = (kEntropy && on) ? es[j] * z : 0.f;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const bool up = (lane & o) != 0;
-#pragma unroll
-          for (int i = 0; i < o; ++i) {
-            const float ss = up ? es[i] : es[i + o], ks = up ? es[i + o] : es[i];
-            es[i] = ks + __shfl_xor_sync(0xffffffffu, ss, o);
-            if (kEntropy) {
-              const float st2 = up ? et[i] : et[i + o], kt = up ? et[i + o] : et[i];
-              et[i] = kt + __shfl_xor_sync(0xffffffffu, st2, o);
-            }
-          }
-        }
-        // fold the tile's statistics of column h * 32 + lane into the running ones
-        {
-          LmRowAcc a = {run[h].m, run[h].s, run[h].t};
-          lm_fold(a, m_t, es[0], et[0], c);
-          run[h].m = a.m; run[h].s = a.s; run[h].t = a.t;
-          lm_top2_insert(v1[0], i1[0], run[h].v1, run[h].i1, run[h].v2, run[h].i2);
-          lm_top2_insert(v2[0], i2[0], run[h].v1, run[h].i1, run[h].v2, run[h].i2);
-        }
+        lm_rows_chunk<kEntropy>(r, valid, v_lane0 + lane, h * 32, sp.N, lane, c, run[h]);
       }
     }
     // the four warps covered different vocabulary entries of every tile: merge through shared memory
