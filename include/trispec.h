@@ -365,8 +365,8 @@ int trispec_sample_bonus(const trispec_sample_args* a, void* stream);
  * Fused pass: the four calls above on `stream` (one verification round of Algorithm 1 for
  * one verifier): tree mask first, acceptance scan last; the attention and the LM-head
  * statistics, which do not read each other's results, in the order the library finds faster
- * for the shape. `attn` may be NULL to skip attention. For one active sequence and a short
- * context the library runs mask + attention on an internal second stream beside the LM head and
+ * for the shape. `attn` may be NULL to skip attention. For one active sequence whose attention
+ * needs few CTAs the library runs mask + attention on an internal second stream beside the LM head and
  * the scan, and `stream` waits for that stream before the call returns its place in the queue:
  * what the caller sees is unchanged (everything the call enqueues has completed before anything
  * enqueued on `stream` afterwards starts), but no output buffer of the call may overlap an input
@@ -376,9 +376,10 @@ int trispec_sample_bonus(const trispec_sample_args* a, void* stream);
 int trispec_verify(const trispec_tree_args* tree, const trispec_attn_args* attn,
                    const trispec_lmhead_args* lm, const trispec_scan_args* scan, void* stream);
 /* How a pass with these arguments arranges its attention and its LM head (a diagnostic; host only,
- * nothing is launched; `attn` and `scan` may be NULL): "attention_first", "lm_first" (one active
- * sequence behind a chip-filling attention) or "side_by_side" (one active sequence, short context:
- * the second-stream form described above); "none" without `lm`. */
+ * nothing is launched; `attn` and `scan` may be NULL): "attention_first" (batches), "lm_first" or
+ * "side_by_side" (one active sequence: the second-stream form described above where the LM head can
+ * spare the attention's SMs); "none" without `lm`. The environment variable TRISPEC_PASS_FORM =
+ * attention_first | lm_first | side_by_side overrides the choice for one active sequence. */
 const char* trispec_verify_plan(const trispec_attn_args* attn, const trispec_lmhead_args* lm,
                                 const trispec_scan_args* scan);
 

@@ -1,6 +1,7 @@
 // Fused verify pass: tree mask -> attention -> LM-head statistics -> acceptance scan on one
 // stream (one verification round of Algorithm 1 for one verifier).
 #include <mutex>
+#include <stdlib.h>
 
 #include "host_common.h"
 
@@ -41,12 +42,27 @@ static PassForm pass_form(const trispec_attn_args* attn, const trispec_lmhead_ar
   const int attn_ctas = attn ? attn_planned_ctas(attn) : 0;
   if (attn_ctas_out) *attn_ctas_out = attn_ctas;
   if (!attn || lm_seqs != 1 || attn_ctas <= 0) return PASS_ATTENTION_FIRST;
+  // TRISPEC_PASS_FORM = attention_first | lm_first | side_by_side overrides the rule below for one active
+  // sequence (a tuning and testing aid, read at every call; side by side still needs at most SMs / 2 CTAs)
+  if (const char* e = getenv("TRISPEC_PASS_FORM")) {
+    if (e[0] == 'a') return PASS_ATTENTION_FIRST;
+    if (e[0] == 'l') return PASS_LM_FIRST;
+    if (e[0] == 's' && attn_ctas * 2 <= device_sm_count() &&
+        !(attn->seq_index && scan && scan->esc_index == attn->seq_index)) return PASS_SIDE_BY_SIDE;
+  }
   // not side by side when the scan's escalation list is written over the index list the attention reads:
   // in stream order the scan comes last, side by side it would not
   const bool in_place_list = attn->seq_index && scan && scan->esc_index == attn->seq_index;
-  if (attn_ctas * 8 <= device_sm_count() && !in_place_list) return PASS_SIDE_BY_SIDE;
-  if (attn_ctas * 4 > device_sm_count()) return PASS_LM_FIRST;
-  return PASS_ATTENTION_FIRST;
+  // Side by side the LM head gives up one SM per attention CTA and takes SMs / (SMs - CTAs) times as long;
+  // one after the other the pass pays the attention (15-25 us at these sizes) and a launch boundary. With the
+  // LM head's time estimated as its bytes of W at 5 TB/s, side by side wins while that extra time stays below
+  // about 40 us (measured on one sequence: 32000 x 2048 weights with 16 and 64 CTAs, 151936 x 2048 with 16 and
+  // 32 CTAs win; 151936 x 2048 with 64 CTAs loses 180 against 152 us; 128256 x 4096 with 32 CTAs is even).
+  // Otherwise the LM head goes first: behind the attention it would stall as a programmatic dependent.
+  const int sms = device_sm_count();
+  const double lm_us = static_cast<double>(lm->V) * lm->d * 2.0 / 5.0e6;
+  if (attn_ctas * 2 <= sms && !in_place_list && lm_us * attn_ctas <= 40.0 * (sms - attn_ctas)) return PASS_SIDE_BY_SIDE;
+  return PASS_LM_FIRST;
 }
 }  // namespace trispec
 
@@ -68,15 +84,15 @@ extern "C" int trispec_verify(const trispec_tree_args* tree, const trispec_attn_
   // a programmatic dependent gets its launch latency and prologue hidden, but its loads make almost no
   // progress while the kernel before it still runs (measured: the stages of the single-sequence LM head
   // arrive within a microsecond of the attention's end, whenever it started). For one active sequence the
-  // LM head is a pure stream of W: behind an attention that fills a good part of the chip it loses more
-  // than the hidden latency (one sequence of 4096 context tokens: 166 us against 156 us the other way
-  // round), so there the LM head goes first.
+  // LM head is a pure stream of W and loses more behind an attention than the hidden latency is worth (one
+  // sequence of 4096 context tokens: 166 us against 156 us the other way round), so there the LM head goes
+  // first, or the two run side by side (pass_form above).
   int attn_ctas = 0;
   const trispec::PassForm form = trispec::pass_form(attn, lm, scan, &attn_ctas);
   const bool lm_first = form == trispec::PASS_LM_FIRST;
   int rc;
-  // One active sequence and a small attention (a short context: a few CTAs for 10-20 us, all latency): the
-  // two run side by side. Mask and attention go to a second stream behind an event recorded on `stream` at the
+  // One active sequence and an attention small enough beside the LM head (pass_form): the two run side by
+  // side. Mask and attention go to a second stream behind an event recorded on `stream` at the
   // start of the call; the LM head, whose grid is one persistent CTA per SM, leaves them one SM per attention
   // CTA and starts at once, the scan follows it, and `stream` then waits for the second stream: everything
   // the call enqueues is complete before anything enqueued on `stream` after it.

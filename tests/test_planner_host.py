@@ -75,9 +75,9 @@ def test_pass_form_follows_the_active_sequences_and_the_size_of_the_attention():
     # batches: attention, then LM head
     assert ts.trispec_verify_plan(_attn_args(gen.CONFIGS["proxy_tree"]), lm_args(8)) == "attention_first"
     assert ts.trispec_verify_plan(None, lm_args(1)) == "attention_first"
-    # one sequence, 512 context tokens: 8 KV heads x 2 splits = 16 CTAs, an eighth of 148 SMs or less
+    # one sequence, 512 context tokens: 8 KV heads x 2 splits = 16 CTAs: the LM head can spare their SMs
     assert ts.trispec_verify_plan(_attn_args(gen.CONFIGS["tiny_chain"]), lm_args(1)) == "side_by_side"
-    # one sequence, 4096 context tokens: 64 CTAs, more than a quarter of the chip
+    # one sequence, 4096 context tokens: 64 CTAs would cost the LM head (151936 x 2048 weights) too many SMs
     assert ts.trispec_verify_plan(_attn_args(one(gen.CONFIGS["proxy_tree"], B=1)), lm_args(1)) == "lm_first"
     # one ACTIVE sequence of several, picked through an index list
     a = _attn_args(one(gen.CONFIGS["tiny_chain"], B=4), n_active=1)
@@ -85,6 +85,6 @@ def test_pass_form_follows_the_active_sequences_and_the_size_of_the_attention():
     # ... unless the scan writes its escalation list over that index list: then in stream order
     s = ts.ScanArgs()
     s.esc_index = 1
-    assert ts.trispec_verify_plan(a, lm_args(4, n_active=1), s) == "attention_first"
+    assert ts.trispec_verify_plan(a, lm_args(4, n_active=1), s) == "lm_first"
     s.esc_index = 2
     assert ts.trispec_verify_plan(a, lm_args(4, n_active=1), s) == "side_by_side"
